@@ -1,0 +1,161 @@
+/*
+ * adadecode.h - C ABI of the B200 (sm_100a) layer-parallel decode library.
+ *
+ * The library implements the decoding loop of AdaDecode (Algorithm 1 of the paper): the newest
+ * token climbs the decoder layers while the deferred upper layers of earlier early-predicted
+ * tokens are processed alongside it; at chosen intermediate layers a lightweight head
+ * (Section 2.1) predicts the next token and, if its probability exceeds a threshold (Eq. 1),
+ * the token is emitted early; when the newest token reaches the last layer every early token
+ * is verified against the full-depth argmax (Eq. 2 at temperature zero, Appendix D) and the
+ * first mismatch rolls the sequence and the KV cache back.  Plain greedy decoding (Table 2,
+ * "Vanilla Decoding") runs through the same kernels with one row and no heads.
+ *
+ * Conventions
+ *   - Every function returns 0 (ADA_OK) or a negative ADA_E* code; nothing throws, aborts or
+ *     traps the GPU.  ada_strerror() names a code; ada_last_cuda_error() returns the CUDA error
+ *     string saved by the last ADA_ECUDA on the calling thread.
+ *   - "dev" pointers are device memory owned by the CALLER (allocated e.g. through PyTorch); the
+ *     library borrows them and they must outlive the object they were given to.  "host" pointers
+ *     are ordinary host memory.  The library never allocates device memory itself, except in
+ *     ada_*_create for tensor-map/handle bookkeeping on the host.
+ *   - All matrices are row-major [out_features, in_features]; every tensor of a model has the
+ *     model's dtype (fp32 or bf16 bit patterns).
+ *   - One session is used from one host thread at a time.  All device work of a session is issued
+ *     on the CUDA stream given at creation.
+ */
+#ifndef ADADECODE_H
+#define ADADECODE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ADA_OK 0
+#define ADA_EINVAL (-1)       /* bad argument */
+#define ADA_ESTATE (-2)       /* call order (e.g. decode before prefill, tensor missing) */
+#define ADA_ECAPACITY (-3)    /* KV pool, max_seq_len, max_early or scratch too small */
+#define ADA_ECUDA (-4)        /* a CUDA call failed; see ada_last_cuda_error() */
+#define ADA_ETIMEOUT (-5)     /* a bounded device-side wait expired */
+#define ADA_EUNSUPPORTED (-6) /* shape or dtype outside what the kernels are built for */
+
+#define ADA_DTYPE_FP32 0
+#define ADA_DTYPE_BF16 1
+
+#define ADA_MAX_BATCH 16
+#define ADA_MAX_LAYERS 256
+
+typedef struct ada_model ada_model;     /* opaque */
+typedef struct ada_session ada_session; /* opaque: sequences, paged KV metadata, in-flight state */
+
+/* Decoder shape (the Llama family the paper evaluates, Section 3).  d_model, d_ff and
+   n_q_heads*head_dim must be multiples of 8; head_dim a multiple of 32, at most 256;
+   n_q_heads a multiple of n_kv_heads. */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+    int32_t dtype;        /* ADA_DTYPE_* of every tensor, of the activations fed to the GEMMs and of the KV cache */
+    int32_t tied_lm_head; /* 1: the LM head E* aliases tok_embed */
+    float rope_base, rms_eps;
+} ada_config;
+
+/* Counters of one or more decode calls (accumulated into the struct the caller passes).
+   Definitions: a "step" is one iteration of Algorithm 1's while loop for one sequence; the
+   early-exit rate is early_exits / steps; the rejection rate is rejected / (accepted + rejected);
+   early predictions behind a rejection were never examined and count as discarded. */
+typedef struct {
+    int64_t steps, head_evals, early_exits, verify_steps, accepted, rejected, discarded;
+    int64_t row_layers;      /* sum over processed layers of the rows processed there */
+    int64_t truncated;       /* verified tokens dropped to end a call on the requested count */
+    int64_t exits_at_layer[ADA_MAX_LAYERS]; /* indexed by 1-based exit layer */
+    int64_t host_syncs;      /* stream synchronisations the decode loop needed */
+    int64_t kernel_launches; /* kernels of this library launched by the decode calls */
+    double decode_ms;        /* device time of the decode calls (CUDA events on the session stream) */
+} ada_stats;
+
+const char *ada_strerror(int code);
+const char *ada_last_cuda_error(void);
+
+/* ---- model: "load weights" -------------------------------------------------------------- */
+
+int ada_model_create(const ada_config *cfg, ada_model **out);
+
+/* Lend one tensor (device pointer, exact byte size checked).  Names:
+ *   tok_embed [vocab, d]         final_norm [d]          lm_head [vocab, d] (only if not tied)
+ *   layers.N.attn_norm [d]       layers.N.ffn_norm [d]
+ *   layers.N.wqkv [(n_q+2 n_kv) head_dim, d]   rows: all q heads, then all k heads, then all v heads
+ *   layers.N.wo [d, n_q head_dim]
+ *   layers.N.w_gate_up [2 d_ff, d]             rows: gate, then up
+ *   layers.N.w_down [d, d_ff]
+ * Pointers must be 16-byte aligned. */
+int ada_model_set_tensor(ada_model *m, const char *name, const void *dev_ptr, size_t bytes);
+
+/* Register the intermediate head of Section 2.1 at 1-based `layer` (1 <= layer < n_layers):
+ * logits = logit_scale * E* (T RMSNorm_f(h)), E^(i) = E* T^(i).  T_dev is a dense [d, d] matrix in
+ * the model dtype, or NULL for T = I. */
+int ada_model_set_exit_head(ada_model *m, int32_t layer, const void *T_dev, float logit_scale);
+
+int ada_model_finalize(ada_model *m); /* ADA_ESTATE if a tensor is missing */
+void ada_model_destroy(ada_model *m);
+
+/* ---- session ------------------------------------------------------------------------------ */
+
+/* Device bytes of scratch a session needs (activations, partial results, state; no KV). */
+size_t ada_session_scratch_bytes(const ada_model *m, int32_t batch, int32_t max_seq_len, int32_t max_early);
+/* Device bytes of one KV page (page_tokens positions, all layers, K and V). */
+size_t ada_kv_page_bytes(const ada_model *m, int32_t page_tokens);
+
+/* Create a session of `batch` independent sequences.  kv_pool_dev holds kv_pool_bytes /
+ * ada_kv_page_bytes() pages that the session hands to sequences on demand; page_tokens is a power
+ * of two in [16, 256].  max_early bounds the early predictions in flight per sequence (the paper
+ * uses 5).  scratch_dev must be 256-byte aligned and at least ada_session_scratch_bytes() long;
+ * the session zero-fills what it needs of it.  cuda_stream is a cudaStream_t (0 = default). */
+int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, int32_t page_tokens,
+                       int32_t max_early, void *kv_pool_dev, size_t kv_pool_bytes, void *scratch_dev,
+                       size_t scratch_bytes, void *cuda_stream, ada_session **out);
+void ada_session_destroy(ada_session *s);
+/* Forget sequence `seq` (or all sequences if seq < 0) and return its pages to the pool. */
+int ada_session_reset(ada_session *s, int32_t seq);
+
+/* KV cache <- LM(x) (first line of Algorithm 1): runs the n_prompt tokens of sequence `seq`
+ * through all layers.  The first generated token (full-depth argmax at the last prompt token)
+ * becomes the sequence's pending token.  ADA_ECAPACITY if pages or max_seq_len do not suffice. */
+int ada_prefill(ada_session *s, int32_t seq, const int32_t *prompt_host, int32_t n_prompt);
+
+/* Both decode calls return the NEXT n_tokens verified generated tokens of every sequence into
+ * out_host[batch][n_tokens] (counting from the first generated token, which prefill produced),
+ * synchronise the stream before returning, and leave the same logical state: K/V present at all
+ * layers for every token before the last returned one, which stays pending.  Calls can be chained
+ * and mixed.  Every sequence must have been prefilled. */
+int ada_plain_decode(ada_session *s, int32_t n_tokens, int32_t *out_host, ada_stats *stats /* nullable */);
+
+/* Algorithm 1.  threshold = gamma of Eq. 1 (strict: exit iff p > gamma).  exit_layers: ascending
+ * 1-based layers, each < n_layers, each with a registered head.  max_early <= the session's. */
+int ada_adaptive_decode(ada_session *s, int32_t n_tokens, float threshold, const int32_t *exit_layers,
+                        int32_t n_exit_layers, int32_t max_early, int32_t *out_host, ada_stats *stats);
+
+/* ---- test hooks --------------------------------------------------------------------------- */
+
+/* Record the final-layer logits of every verified generated token of sequence 0 into dev_buf
+ * [max_tokens][vocab] fp32 (device memory), from the next prefill/decode on; NULL stops. */
+int ada_debug_capture_logits(ada_session *s, float *dev_buf, int32_t max_tokens);
+int ada_debug_logits_captured(ada_session *s, int32_t *n_out);
+/* Record every intermediate-head evaluation as 4 floats (step, layer, token, p) into host_buf
+ * (copied at the end of each adaptive call); NULL stops. */
+int ada_debug_capture_heads(ada_session *s, float *host_buf, int32_t max_evals, int32_t *n_out);
+/* Force exit decisions: entry i is consumed by the i-th head evaluation of sequence 0 of the next
+ * adaptive call; 0 = continue, 1 = exit, other = follow Eq. 1.  Past the end: Eq. 1. */
+int ada_debug_set_exit_tape(ada_session *s, const uint8_t *tape_host, int32_t n);
+/* Read back per-layer fill levels (positions with valid K/V) and the length of sequence seq. */
+int ada_debug_get_state(ada_session *s, int32_t seq, int32_t *len_out, int32_t *fill_out /*[n_layers]*/);
+/* Copy K (which=0) or V (which=1) of one cached position of one layer into host_out
+ * [n_kv_heads*head_dim] as fp32. */
+int ada_debug_read_kv(ada_session *s, int32_t seq, int32_t which, int32_t layer0, int32_t pos, float *host_out);
+/* Select the GEMM path: 0 = CUDA-core kernels (any dtype), 1 = tensor-core kernels (bf16 only). */
+int ada_debug_set_path(ada_session *s, int32_t path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADADECODE_H */

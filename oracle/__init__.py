@@ -32,7 +32,7 @@ def build(force: bool = False) -> str:
 class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ff", C.c_int32),
-                ("vocab", C.c_int32), ("wdtype", C.c_int32), ("rope_base", C.c_double),
+                ("vocab", C.c_int32), ("wdtype", C.c_int32), ("kv_bf16", C.c_int32), ("rope_base", C.c_double),
                 ("rms_eps", C.c_double)]
 
 
@@ -99,7 +99,7 @@ class Model:
     """Borrowed-weights oracle model.  `weights` uses the fused layout names
     (tok_embed, final_norm, [lm_head], layers.N.{attn_norm,wqkv,wo,ffn_norm,w_gate_up,w_down})."""
 
-    def __init__(self, cfg, weights: Dict[str, np.ndarray]):
+    def __init__(self, cfg, weights: Dict[str, np.ndarray], kv_bf16: Optional[bool] = None):
         lib = _lib()
         self.cfg = cfg
         self._keep = []
@@ -113,7 +113,7 @@ class Model:
             return a.ctypes.data
 
         c = Config(cfg.n_layers, cfg.d_model, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ff,
-                   cfg.vocab, 1 if bf16 else 0, cfg.rope_base, cfg.rms_eps)
+                   cfg.vocab, 1 if bf16 else 0, int(bf16 if kv_bf16 is None else kv_bf16), cfg.rope_base, cfg.rms_eps)
         nq, nkv = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
         layers = (LayerW * cfg.n_layers)()
         for l in range(cfg.n_layers):
@@ -270,6 +270,7 @@ class Session:
             pass
 
 
-def model_from_torch(cfg, weights) -> Model:
-    """Build an oracle model from the torch tensors of the input generator (moved to the CPU)."""
-    return Model(cfg, {k: to_numpy(v) for k, v in weights.items()})
+def model_from_torch(cfg, weights, kv_bf16: Optional[bool] = None) -> Model:
+    """Build an oracle model from the torch tensors of the input generator (moved to the CPU).
+    kv_bf16 None: the cache holds bf16 exactly when the model is a bf16 model."""
+    return Model(cfg, {k: to_numpy(v) for k, v in weights.items()}, kv_bf16=kv_bf16)

@@ -36,6 +36,8 @@
 typedef struct {
     int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
     int32_t wdtype; /* storage of every tensor: 0 = fp32, 1 = bf16 */
+    int32_t kv_bf16; /* 1: the KV cache holds bf16: K (after rotation) and V are rounded once, to
+                        nearest-even, when they are written; everything else stays double */
     double rope_base, rms_eps;
 } orc_config;
 
@@ -146,6 +148,18 @@ static void rope(double *v, int hd, int pos, double base) {
 
 static double silu(double x) { return x / (1.0 + exp(-x)); }
 
+/* Round a double to the nearest bf16 (ties to even), returned as a double.  The double is first
+   rounded to fp32 (the type the cache writer holds it in), then the low 16 bits are rounded away. */
+static double round_bf16(double x) {
+    float f = (float)x;
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) != 0x7f800000u) u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
 /* ---------------------------------------------------------------- model */
 
 orc_model *orc_model_create(const orc_config *c, const void *tok_embed, const void *lm_head,
@@ -246,6 +260,9 @@ static int layer_forward(orc_session *s, int l, int pos0, int n_rows, double *H)
         int pos = pos0 + r;
         for (int h = 0; h < nq; ++h) rope(q + (size_t)r * qd + h * hd, hd, pos, c->rope_base);
         for (int h = 0; h < nkv; ++h) rope(k + (size_t)r * kvd + h * hd, hd, pos, c->rope_base);
+        if (c->kv_bf16) {
+            for (int i = 0; i < kvd; ++i) { k[(size_t)r * kvd + i] = round_bf16(k[(size_t)r * kvd + i]); v[(size_t)r * kvd + i] = round_bf16(v[(size_t)r * kvd + i]); }
+        }
         memcpy(kc + (size_t)pos * kvd, k + (size_t)r * kvd, sizeof(double) * kvd);
         memcpy(vc + (size_t)pos * kvd, v + (size_t)r * kvd, sizeof(double) * kvd);
     }

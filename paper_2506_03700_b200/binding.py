@@ -1,0 +1,253 @@
+"""ctypes binding of the C-ABI decode library (`include/adadecode.h`).
+
+Argument marshalling only: every step of the decode path runs in the library's CUDA kernels.
+PyTorch is used for device memory and the CUDA stream.  There is no CPU fallback: loading fails
+loudly when the compiled library is missing.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libadadecode.so")
+_LIB = None
+
+ADA_MAX_LAYERS = 256
+ERRORS = {0: "ADA_OK", -1: "ADA_EINVAL", -2: "ADA_ESTATE", -3: "ADA_ECAPACITY", -4: "ADA_ECUDA",
+          -5: "ADA_ETIMEOUT", -6: "ADA_EUNSUPPORTED"}
+
+EXPORTS = [
+    "ada_strerror", "ada_last_cuda_error", "ada_model_create", "ada_model_set_tensor", "ada_model_set_exit_head",
+    "ada_model_finalize", "ada_model_destroy", "ada_session_scratch_bytes", "ada_kv_page_bytes",
+    "ada_session_create", "ada_session_destroy", "ada_session_reset", "ada_prefill", "ada_plain_decode",
+    "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
+    "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
+]
+
+
+class AdaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = f"{where}: {ERRORS.get(code, code)}"
+        try:
+            lib = _LIB
+            if lib is not None:
+                msg += f" ({lib.ada_strerror(code).decode()})"
+                if code == -4:
+                    msg += f" [{lib.ada_last_cuda_error().decode()}]"
+        except Exception:
+            pass
+        super().__init__(msg)
+
+
+class Config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32),
+                ("dtype", C.c_int32), ("tied_lm_head", C.c_int32), ("rope_base", C.c_float), ("rms_eps", C.c_float)]
+
+
+class Stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in
+                ("steps", "head_evals", "early_exits", "verify_steps", "accepted", "rejected", "discarded",
+                 "row_layers", "truncated")] + \
+               [("exits_at_layer", C.c_int64 * ADA_MAX_LAYERS), ("host_syncs", C.c_int64),
+                ("kernel_launches", C.c_int64), ("decode_ms", C.c_double)]
+
+    def as_dict(self) -> dict:
+        d = {n: getattr(self, n) for n, _ in self._fields_ if n != "exits_at_layer"}
+        d["exits_at_layer"] = {i: int(v) for i, v in enumerate(self.exits_at_layer) if v}
+        return d
+
+
+def load() -> C.CDLL:
+    """Load the compiled library; raises if it has not been built."""
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2506_03700_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+        L.ada_strerror.restype = C.c_char_p
+        L.ada_strerror.argtypes = [C.c_int]
+        L.ada_last_cuda_error.restype = C.c_char_p
+        L.ada_model_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+        L.ada_model_set_tensor.argtypes = [vp, C.c_char_p, vp, sz]
+        L.ada_model_set_exit_head.argtypes = [vp, i32, vp, C.c_float]
+        L.ada_model_finalize.argtypes = [vp]
+        L.ada_model_destroy.argtypes = [vp]
+        L.ada_model_destroy.restype = None
+        L.ada_session_scratch_bytes.restype = sz
+        L.ada_session_scratch_bytes.argtypes = [vp, i32, i32, i32]
+        L.ada_kv_page_bytes.restype = sz
+        L.ada_kv_page_bytes.argtypes = [vp, i32]
+        L.ada_session_create.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, sz, vp, C.POINTER(vp)]
+        L.ada_session_destroy.argtypes = [vp]
+        L.ada_session_destroy.restype = None
+        L.ada_session_reset.argtypes = [vp, i32]
+        L.ada_prefill.argtypes = [vp, i32, vp, i32]
+        L.ada_plain_decode.argtypes = [vp, i32, vp, C.POINTER(Stats)]
+        L.ada_adaptive_decode.argtypes = [vp, i32, C.c_float, vp, i32, i32, vp, C.POINTER(Stats)]
+        L.ada_debug_capture_logits.argtypes = [vp, vp, i32]
+        L.ada_debug_logits_captured.argtypes = [vp, C.POINTER(i32)]
+        L.ada_debug_capture_heads.argtypes = [vp, vp, i32, C.POINTER(i32)]
+        L.ada_debug_set_exit_tape.argtypes = [vp, vp, i32]
+        L.ada_debug_get_state.argtypes = [vp, i32, C.POINTER(i32), vp]
+        L.ada_debug_read_kv.argtypes = [vp, i32, i32, i32, i32, vp]
+        L.ada_debug_set_path.argtypes = [vp, i32]
+        _LIB = L
+    return _LIB
+
+
+def _ck(rc: int, where: str):
+    if rc != 0:
+        raise AdaError(rc, where)
+
+
+class Model:
+    """ada_model over borrowed torch CUDA tensors (fused layout of `synth.make_weights`)."""
+
+    def __init__(self, cfg, weights: Dict[str, "torch.Tensor"], tied: Optional[bool] = None):
+        import torch
+        lib = load()
+        self.cfg = cfg
+        tied = ("lm_head" not in weights) if tied is None else tied
+        c = Config(cfg.n_layers, cfg.d_model, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ff, cfg.vocab,
+                   1 if cfg.dtype == "bf16" else 0, 1 if tied else 0, cfg.rope_base, cfg.rms_eps)
+        h = C.c_void_p()
+        _ck(lib.ada_model_create(C.byref(c), C.byref(h)), "ada_model_create")
+        self.h = h
+        self._keep = []
+        for name, t in weights.items():
+            assert t.is_cuda and t.is_contiguous() and t.dtype == cfg.torch_dtype, name
+            self._keep.append(t)
+            _ck(lib.ada_model_set_tensor(h, name.encode(), t.data_ptr(), t.numel() * t.element_size()),
+                f"ada_model_set_tensor({name})")
+        self._finalized = False
+
+    def set_exit_head(self, layer: int, T=None, logit_scale: float = 1.0):
+        ptr = None
+        if T is not None:
+            assert T.is_cuda and T.is_contiguous() and T.dtype == self.cfg.torch_dtype
+            self._keep.append(T)
+            ptr = T.data_ptr()
+        _ck(load().ada_model_set_exit_head(self.h, layer, ptr, logit_scale), f"ada_model_set_exit_head({layer})")
+
+    def finalize(self):
+        if not self._finalized:
+            _ck(load().ada_model_finalize(self.h), "ada_model_finalize")
+            self._finalized = True
+
+    def __del__(self):
+        try:
+            if self.h:
+                load().ada_model_destroy(self.h)
+                self.h = None
+        except Exception:
+            pass
+
+
+class Session:
+    """ada_session with its KV pool and scratch allocated through torch on the current device."""
+
+    def __init__(self, model: Model, batch: int = 1, max_seq_len: int = 4096, page_tokens: int = 64,
+                 max_early: int = 5, kv_pages: Optional[int] = None, stream=None):
+        import torch
+        lib = load()
+        model.finalize()
+        self.model = model
+        self.batch = batch
+        self.max_seq_len = max_seq_len
+        self.vocab = model.cfg.vocab
+        page_bytes = lib.ada_kv_page_bytes(model.h, page_tokens)
+        if kv_pages is None:
+            kv_pages = batch * ((max_seq_len + page_tokens - 1) // page_tokens)
+        self.kv_pool = torch.empty(kv_pages * page_bytes, dtype=torch.uint8, device="cuda")
+        sb = lib.ada_session_scratch_bytes(model.h, batch, max_seq_len, max_early)
+        self.scratch = torch.empty(sb + 256, dtype=torch.uint8, device="cuda")
+        off = (-self.scratch.data_ptr()) % 256
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        h = C.c_void_p()
+        _ck(lib.ada_session_create(model.h, batch, max_seq_len, page_tokens, max_early, self.kv_pool.data_ptr(),
+                                   self.kv_pool.numel(), self.scratch.data_ptr() + off, sb,
+                                   self.stream.cuda_stream, C.byref(h)), "ada_session_create")
+        self.h = h
+        self._capture = None
+        self._heads = None
+        self._heads_n = C.c_int32(0)
+
+    # ---- the calls of the boundary
+    def reset(self, seq: int = -1):
+        _ck(load().ada_session_reset(self.h, seq), "ada_session_reset")
+
+    def prefill(self, prompt: Sequence[int], seq: int = 0):
+        p = np.ascontiguousarray(np.asarray(prompt, dtype=np.int32))
+        _ck(load().ada_prefill(self.h, seq, p.ctypes.data, len(p)), "ada_prefill")
+
+    def plain_decode(self, n_tokens: int, stats: Optional[Stats] = None, out: Optional[np.ndarray] = None) -> np.ndarray:
+        out = np.empty((self.batch, n_tokens), dtype=np.int32) if out is None else out
+        _ck(load().ada_plain_decode(self.h, n_tokens, out.ctypes.data, C.byref(stats) if stats is not None else None),
+            "ada_plain_decode")
+        return out
+
+    def adaptive_decode(self, n_tokens: int, threshold: float, exit_layers: Sequence[int], max_early: int = 5,
+                        stats: Optional[Stats] = None, out: Optional[np.ndarray] = None) -> np.ndarray:
+        out = np.empty((self.batch, n_tokens), dtype=np.int32) if out is None else out
+        ex = np.ascontiguousarray(np.asarray(exit_layers, dtype=np.int32))
+        _ck(load().ada_adaptive_decode(self.h, n_tokens, threshold, ex.ctypes.data if len(ex) else None, len(ex),
+                                       max_early, out.ctypes.data, C.byref(stats) if stats is not None else None),
+            "ada_adaptive_decode")
+        return out
+
+    # ---- test hooks
+    def capture_logits(self, max_tokens: int):
+        import torch
+        self._capture = torch.zeros(max_tokens, self.vocab, dtype=torch.float32, device="cuda")
+        _ck(load().ada_debug_capture_logits(self.h, self._capture.data_ptr(), max_tokens), "ada_debug_capture_logits")
+
+    def captured_logits(self):
+        n = C.c_int32(0)
+        _ck(load().ada_debug_logits_captured(self.h, C.byref(n)), "ada_debug_logits_captured")
+        return self._capture[:min(n.value, self._capture.shape[0])]
+
+    def capture_heads(self, max_evals: int = 1 << 16):
+        self._heads = np.zeros((max_evals, 4), dtype=np.float32)
+        _ck(load().ada_debug_capture_heads(self.h, self._heads.ctypes.data, max_evals, C.byref(self._heads_n)),
+            "ada_debug_capture_heads")
+
+    def captured_heads(self) -> np.ndarray:
+        """Rows (step, layer, token, p) of the last adaptive call."""
+        return self._heads[:min(self._heads_n.value, len(self._heads))]
+
+    def set_exit_tape(self, tape: Sequence[int]):
+        t = np.ascontiguousarray(np.asarray(tape, dtype=np.uint8))
+        _ck(load().ada_debug_set_exit_tape(self.h, t.ctypes.data if len(t) else None, len(t)), "ada_debug_set_exit_tape")
+
+    def state(self, seq: int = 0):
+        ln = C.c_int32(0)
+        fill = np.zeros(self.model.cfg.n_layers, dtype=np.int32)
+        _ck(load().ada_debug_get_state(self.h, seq, C.byref(ln), fill.ctypes.data), "ada_debug_get_state")
+        return ln.value, fill
+
+    def read_kv(self, which: int, layer0: int, pos: int, seq: int = 0) -> np.ndarray:
+        c = self.model.cfg
+        out = np.zeros(c.n_kv_heads * c.head_dim, dtype=np.float32)
+        _ck(load().ada_debug_read_kv(self.h, seq, which, layer0, pos, out.ctypes.data), "ada_debug_read_kv")
+        return out
+
+    def set_path(self, path: int):
+        _ck(load().ada_debug_set_path(self.h, path), "ada_debug_set_path")
+
+    def __del__(self):
+        try:
+            if self.h:
+                load().ada_session_destroy(self.h)
+                self.h = None
+        except Exception:
+            pass

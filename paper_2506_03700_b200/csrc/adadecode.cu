@@ -1,0 +1,719 @@
+// Host side of the decode library: C ABI, model/session bookkeeping, paged KV allocator, and the
+// loops that issue the kernels of Algorithm 1.  All decoding state lives on the device; the host
+// only decides how far to launch and reads back a few counters.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "kernels.cuh"
+
+using namespace ada;
+
+namespace {
+
+thread_local std::string g_cuda_err;
+
+#define CK(expr)                                                                                    \
+    do {                                                                                            \
+        cudaError_t e__ = (expr);                                                                   \
+        if (e__ != cudaSuccess) {                                                                   \
+            g_cuda_err = std::string(#expr) + ": " + cudaGetErrorString(e__);                       \
+            return ADA_ECUDA;                                                                       \
+        }                                                                                           \
+    } while (0)
+
+struct LayerW {
+    const void *attn_norm = nullptr, *wqkv = nullptr, *wo = nullptr, *ffn_norm = nullptr, *w_gate_up = nullptr,
+               *w_down = nullptr;
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+struct ada_model {
+    ada_config cfg;
+    size_t esz;
+    const void *tok_embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+    std::vector<LayerW> layers;
+    std::vector<int> has_head;
+    std::vector<const void *> head_T;
+    std::vector<float> head_scale;
+    bool finalized = false;
+};
+
+struct ada_session {
+    const ada_model *m;
+    int batch, max_seq, page_tokens, max_early, slots, rows_alloc, n_pages, max_pages, n_chunks, head_blocks;
+    cudaStream_t stream;
+    Ctx c;
+    void *scratch;
+    size_t scratch_bytes;
+    float *t_out; // [R][d] output of the head transformation
+    std::vector<int> free_pages;
+    std::vector<std::vector<int>> seq_pages;
+    std::vector<int> h_len, h_prompt, h_reported;
+    std::vector<char> prefilled;
+    int32_t *pinned = nullptr; // small read-back area
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    int path = 0;
+    int64_t launches = 0, syncs = 0;
+    // debug
+    float *capture_dev = nullptr;
+    int capture_cap = 0;
+    float *head_log_host = nullptr;
+    int head_log_cap = 0;
+    int32_t *head_log_n_out = nullptr;
+    std::vector<uint8_t> tape;
+};
+
+namespace {
+
+// Scratch layout (all offsets 256-byte aligned).
+struct Layout {
+    size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
+        head_part, logit_stage, head_log, t_out, total;
+};
+
+int rows_alloc_for(int batch, int max_early) { return std::max(batch * (max_early + 1), 32); }
+
+Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, int head_blocks) {
+    Layout L;
+    const int R = rows_alloc_for(batch, max_early);
+    const int qd = g.n_q_heads * g.head_dim, qkv_rows = (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim;
+    const int n_chunks = (max_seq + kAttnChunk - 1) / kAttnChunk;
+    const int max_pages = (max_seq + 15) / 16;  // upper bound for any page size >= 16
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    L.st = take(sizeof(DevState));
+    L.rt = take(sizeof(RowTable));
+    L.fill = take(sizeof(int32_t) * batch * g.n_layers);
+    L.tokens = take(sizeof(int32_t) * (size_t)batch * max_seq);
+    L.page_table = take(sizeof(int32_t) * (size_t)batch * max_pages);
+    L.head_res = take(sizeof(HeadResult) * kMaxRows);
+    L.resid = take(sizeof(float) * (size_t)R * g.d_model);
+    L.xn = take(sizeof(float) * (size_t)R * g.d_model);
+    L.qkv = take(sizeof(float) * (size_t)R * qkv_rows);
+    L.q = take(sizeof(float) * (size_t)R * qd);
+    L.attn_out = take(sizeof(float) * (size_t)R * qd);
+    L.gu = take(sizeof(float) * (size_t)R * 2 * g.d_ff);
+    L.hact = take(sizeof(float) * (size_t)R * g.d_ff);
+    L.rope_cs = take(sizeof(float) * (size_t)R * g.head_dim);
+    L.attn_part = take(sizeof(float) * (size_t)R * g.n_q_heads * n_chunks * (g.head_dim + 2));
+    L.head_part = take(sizeof(float) * (size_t)head_blocks * kMaxRows * 4);
+    L.logit_stage = take(sizeof(float) * (size_t)R * g.vocab);
+    L.head_log = take(sizeof(float) * 4 * kHeadLogCap);
+    L.t_out = take(sizeof(float) * (size_t)R * g.d_model);
+    L.total = o;
+    return L;
+}
+
+constexpr int kHeadBlocks = 148 * 4;
+
+int check_cfg(const ada_config &g) {
+    if (g.n_layers < 1 || g.n_layers > ADA_MAX_LAYERS - 1 || g.d_model < 8 || g.vocab < 2) return ADA_EINVAL;
+    if (g.dtype != ADA_DTYPE_FP32 && g.dtype != ADA_DTYPE_BF16) return ADA_EINVAL;
+    if (g.n_q_heads < 1 || g.n_kv_heads < 1 || g.n_q_heads % g.n_kv_heads) return ADA_EINVAL;
+    if (g.d_model % 8 || g.d_ff % 8 || (g.n_q_heads * g.head_dim) % 8) return ADA_EUNSUPPORTED;
+    if (g.head_dim % 32 || g.head_dim > 256 || g.head_dim < 32) return ADA_EUNSUPPORTED;
+    return ADA_OK;
+}
+
+// ---- typed launch helpers --------------------------------------------------------------------
+
+template <typename T>
+int launch_gemv(ada_session *S, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy, int sel) {
+    int blocks = std::min((N + 7) / 8, 148 * 4);
+    if (epi == 0)
+        k_gemv<T, 0><<<blocks, 256, 0, S->stream>>>(S->c, (const T *)W, N, K, X, ldx, Y, ldy, sel);
+    else
+        k_gemv<T, 1><<<blocks, 256, 0, S->stream>>>(S->c, (const T *)W, N, K, X, ldx, Y, ldy, sel);
+    S->launches++;
+    CK(cudaGetLastError());
+    return ADA_OK;
+}
+
+template <typename T>
+int launch_attn(ada_session *S, int layer, int rows) {
+    const ada_config &g = S->m->cfg;
+    dim3 grid(S->n_chunks, g.n_q_heads, rows);
+    switch (g.head_dim / 32) {
+        case 1: k_attn_partial<T, 1><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        case 2: k_attn_partial<T, 2><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        case 3: k_attn_partial<T, 3><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        case 4: k_attn_partial<T, 4><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        case 5: k_attn_partial<T, 5><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        case 6: k_attn_partial<T, 6><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        case 7: k_attn_partial<T, 7><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+        default: k_attn_partial<T, 8><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
+    }
+    CK(cudaGetLastError());
+    k_attn_combine<<<dim3(g.n_q_heads, rows), 64, 0, S->stream>>>(S->c, layer);
+    CK(cudaGetLastError());
+    S->launches += 2;
+    return ADA_OK;
+}
+
+// One decoder layer over the rows active at `layer` (0-based); `rows` bounds the row indices.
+template <typename T>
+int run_layer_t(ada_session *S, int layer, int rows) {
+    const ada_model *m = S->m;
+    const ada_config &g = m->cfg;
+    const LayerW &w = m->layers[layer];
+    const int d = g.d_model, qd = g.n_q_heads * g.head_dim, qkv_rows = S->c.qkv_rows;
+    const int ldx = d;
+    int rc;
+    k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)w.attn_norm, layer, S->c.xn, ldx);
+    CK(cudaGetLastError());
+    S->launches++;
+    if ((rc = launch_gemv<T>(S, 0, w.wqkv, qkv_rows, d, S->c.xn, ldx, S->c.qkv, qkv_rows, layer))) return rc;
+    k_rope_kv<T><<<rows, 128, 0, S->stream>>>(S->c, layer);
+    CK(cudaGetLastError());
+    S->launches++;
+    if ((rc = launch_attn<T>(S, layer, rows))) return rc;
+    if ((rc = launch_gemv<T>(S, 1, w.wo, d, qd, S->c.attn_out, qd, S->c.resid, d, layer))) return rc;
+    k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)w.ffn_norm, layer, S->c.xn, ldx);
+    CK(cudaGetLastError());
+    S->launches++;
+    if ((rc = launch_gemv<T>(S, 0, w.w_gate_up, 2 * g.d_ff, d, S->c.xn, ldx, S->c.gu, 2 * g.d_ff, layer))) return rc;
+    k_swiglu<<<dim3((g.d_ff + 255) / 256, rows), 256, 0, S->stream>>>(S->c, layer);
+    CK(cudaGetLastError());
+    S->launches++;
+    if ((rc = launch_gemv<T>(S, 1, w.w_down, d, g.d_ff, S->c.hact, g.d_ff, S->c.resid, d, layer))) return rc;
+    return ADA_OK;
+}
+
+// Head over the rows picked by `sel`: layer1 >= 1 is the intermediate head registered there,
+// layer1 == 0 the final LM head (unscaled, T = I).
+template <typename T>
+int run_head_t(ada_session *S, int layer1, int sel, int rows) {
+    const ada_model *m = S->m;
+    const ada_config &g = m->cfg;
+    const int d = g.d_model;
+    int rc;
+    k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)m->final_norm, sel, S->c.xn, d);
+    CK(cudaGetLastError());
+    S->launches++;
+    const float *x = S->c.xn;
+    float scale = 1.0f;
+    if (layer1 > 0) {
+        scale = m->head_scale[layer1];
+        if (m->head_T[layer1]) {
+            if ((rc = launch_gemv<T>(S, 0, m->head_T[layer1], d, d, S->c.xn, d, S->t_out, d, sel))) return rc;
+            x = S->t_out;
+        }
+    }
+    const int store = (layer1 == 0 && S->capture_dev) ? 1 : 0;
+    k_head_partial<T><<<S->head_blocks, 256, 0, S->stream>>>(S->c, (const T *)m->lm_head, x, d, scale, sel, store);
+    CK(cudaGetLastError());
+    k_head_final<<<rows, 32, 0, S->stream>>>(S->c, S->head_blocks, sel);
+    CK(cudaGetLastError());
+    S->launches += 2;
+    return ADA_OK;
+}
+
+int run_layer(ada_session *S, int layer, int rows) {
+    return S->m->cfg.dtype == ADA_DTYPE_BF16 ? run_layer_t<__nv_bfloat16>(S, layer, rows) : run_layer_t<float>(S, layer, rows);
+}
+int run_head(ada_session *S, int layer1, int sel, int rows) {
+    return S->m->cfg.dtype == ADA_DTYPE_BF16 ? run_head_t<__nv_bfloat16>(S, layer1, sel, rows) : run_head_t<float>(S, layer1, sel, rows);
+}
+
+int step_begin(ada_session *S) {
+    const ada_model *m = S->m;
+    if (m->cfg.dtype == ADA_DTYPE_BF16)
+        k_step_begin<__nv_bfloat16><<<1, 256, 0, S->stream>>>(S->c, (const __nv_bfloat16 *)m->tok_embed, m->cfg.rope_base);
+    else
+        k_step_begin<float><<<1, 256, 0, S->stream>>>(S->c, (const float *)m->tok_embed, m->cfg.rope_base);
+    CK(cudaGetLastError());
+    S->launches++;
+    return ADA_OK;
+}
+
+int capture_rows(ada_session *S, int row0) {
+    if (!S->capture_dev) return ADA_OK;
+    k_capture<<<64, 256, 0, S->stream>>>(S->c, row0);
+    CK(cudaGetLastError());
+    k_capture_advance<<<1, 32, 0, S->stream>>>(S->c);
+    CK(cudaGetLastError());
+    S->launches += 2;
+    return ADA_OK;
+}
+
+// Read n_climbing / n_done (one stream synchronisation).
+int read_progress(ada_session *S, int *n_climbing, int *n_done) {
+    CK(cudaMemcpyAsync(S->pinned, &S->c.st->n_climbing, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+    CK(cudaStreamSynchronize(S->stream));
+    S->syncs++;
+    *n_climbing = S->pinned[0];
+    *n_done = S->pinned[1];
+    return ADA_OK;
+}
+
+int ensure_pages(ada_session *S, int seq, int positions) {
+    int need = (positions + S->page_tokens - 1) / S->page_tokens;
+    if (need > S->max_pages) return ADA_ECAPACITY;
+    std::vector<int> &pg = S->seq_pages[seq];
+    if ((int)pg.size() >= need) return ADA_OK;
+    if ((int)S->free_pages.size() < need - (int)pg.size()) return ADA_ECAPACITY;
+    size_t first = pg.size();
+    while ((int)pg.size() < need) { pg.push_back(S->free_pages.back()); S->free_pages.pop_back(); }
+    CK(cudaMemcpyAsync(S->c.page_table + (size_t)seq * S->c.max_pages + first, pg.data() + first,
+                       sizeof(int32_t) * (pg.size() - first), cudaMemcpyHostToDevice, S->stream));
+    CK(cudaStreamSynchronize(S->stream));  // pg may reallocate before the copy is consumed
+    return ADA_OK;
+}
+
+void add_stats(ada_session *S, const DevStats &d, ada_stats *out, float ms, int64_t l0, int64_t s0) {
+    if (!out) return;
+    out->steps += d.steps; out->head_evals += d.head_evals; out->early_exits += d.early_exits;
+    out->verify_steps += d.verify_steps; out->accepted += d.accepted; out->rejected += d.rejected;
+    out->discarded += d.discarded; out->row_layers += d.row_layers; out->truncated += d.truncated;
+    for (int i = 0; i < ADA_MAX_LAYERS; ++i) out->exits_at_layer[i] += d.exits_at_layer[i];
+    out->host_syncs += S->syncs - s0;
+    out->kernel_launches += S->launches - l0;
+    out->decode_ms += ms;
+}
+
+// Shared body of both decode calls.
+int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers, int n_exit, int max_early,
+           int32_t *out_host, ada_stats *stats) {
+    const ada_model *m = S->m;
+    const int L = m->cfg.n_layers;
+    if (!out_host || n_tokens < 1) return ADA_EINVAL;
+    for (int s = 0; s < S->batch; ++s) if (!S->prefilled[s]) return ADA_ESTATE;
+    if (max_early < 0 || max_early > S->max_early) return ADA_ECAPACITY;
+    for (int e = 0; e < n_exit; ++e) {
+        if (exit_layers[e] < 1 || exit_layers[e] >= L || !m->has_head[exit_layers[e]]) return ADA_EINVAL;
+        if (e && exit_layers[e] <= exit_layers[e - 1]) return ADA_EINVAL;
+    }
+    CallTargets tg;
+    memset(&tg, 0, sizeof(tg));
+    int max_steps_plain = 0;
+    for (int s = 0; s < S->batch; ++s) {
+        int target = S->h_prompt[s] + S->h_reported[s] + n_tokens;
+        if (target + 1 > S->max_seq) return ADA_ECAPACITY;
+        int rc = ensure_pages(S, s, target + 1);
+        if (rc) return rc;
+        tg.target_len[s] = target;
+        max_steps_plain = std::max(max_steps_plain, target - S->h_len[s]);
+    }
+    const int64_t l0 = S->launches, s0 = S->syncs;
+    const int rows = S->batch * S->slots;
+    int rc;
+    // zero the device counters, set targets
+    CK(cudaMemsetAsync(&S->c.st->st, 0, sizeof(DevStats), S->stream));
+    int tape_n = (int)std::min<size_t>(S->tape.size(), kMaxTape);
+    if (tape_n) CK(cudaMemcpyAsync(S->c.st->tape, S->tape.data(), tape_n, cudaMemcpyHostToDevice, S->stream));
+    CK(cudaEventRecord(S->ev0, S->stream));
+    k_call_begin<<<1, 32, 0, S->stream>>>(S->c, tg, gamma, max_early, tape_n);
+    CK(cudaGetLastError());
+    S->launches++;
+
+    const bool plain = (n_exit == 0 || max_early == 0);
+    if (plain) {
+        // every step is one token through all layers; the step count is known, no read-back needed
+        for (int it = 0; it < max_steps_plain; ++it) {
+            if ((rc = step_begin(S))) return rc;
+            for (int l = 0; l < L; ++l) if ((rc = run_layer(S, l, rows))) return rc;
+            if ((rc = run_head(S, 0, SEL_FINAL, rows))) return rc;
+            k_verify<<<1, 32, 0, S->stream>>>(S->c);
+            CK(cudaGetLastError());
+            S->launches++;
+            if ((rc = capture_rows(S, 0))) return rc;
+        }
+    } else {
+        int n_done = 0, n_climbing = 0;
+        if ((rc = read_progress(S, &n_climbing, &n_done))) return rc;
+        // generous bound on the loop: every step emits or verifies at least one token
+        long long guard = (long long)(n_tokens + 2) * (max_early + 2) * 4 + 16;
+        while (n_done < S->batch) {
+            if (--guard < 0) return ADA_ETIMEOUT;
+            if ((rc = step_begin(S))) return rc;
+            int e_i = 0;
+            bool reached_top = true;
+            for (int l = 0; l < L; ++l) {
+                if ((rc = run_layer(S, l, rows))) return rc;
+                if (e_i < n_exit && exit_layers[e_i] == l + 1) {
+                    if ((rc = run_head(S, l + 1, SEL_HEAD, rows))) return rc;
+                    k_exit_control<<<1, 32, 0, S->stream>>>(S->c, l + 1);
+                    CK(cudaGetLastError());
+                    S->launches++;
+                    ++e_i;
+                    if ((rc = read_progress(S, &n_climbing, &n_done))) return rc;
+                    if (n_climbing == 0) { reached_top = false; break; }
+                }
+            }
+            if (reached_top) {
+                if ((rc = run_head(S, 0, SEL_FINAL, rows))) return rc;
+                k_verify<<<1, 32, 0, S->stream>>>(S->c);
+                CK(cudaGetLastError());
+                S->launches++;
+                if ((rc = capture_rows(S, 0))) return rc;
+                if ((rc = read_progress(S, &n_climbing, &n_done))) return rc;
+            }
+        }
+    }
+    CK(cudaEventRecord(S->ev1, S->stream));
+    // results
+    for (int s = 0; s < S->batch; ++s) {
+        CK(cudaMemcpyAsync(out_host + (size_t)s * n_tokens,
+                           S->c.tokens + (size_t)s * S->max_seq + S->h_prompt[s] + S->h_reported[s],
+                           sizeof(int32_t) * n_tokens, cudaMemcpyDeviceToHost, S->stream));
+    }
+    DevStats ds;
+    CK(cudaMemcpyAsync(&ds, &S->c.st->st, sizeof(DevStats), cudaMemcpyDeviceToHost, S->stream));
+    int32_t hl_n = 0;
+    if (S->head_log_host) {
+        CK(cudaMemcpyAsync(&hl_n, &S->c.st->head_log_n, sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+    }
+    CK(cudaStreamSynchronize(S->stream));
+    S->syncs++;
+    if (S->head_log_host) {
+        int n = std::min(hl_n, S->head_log_cap);
+        if (n > 0) CK(cudaMemcpy(S->head_log_host, S->c.head_log, sizeof(float) * 4 * n, cudaMemcpyDeviceToHost));
+        if (S->head_log_n_out) *S->head_log_n_out = hl_n;
+    }
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, S->ev0, S->ev1));
+    for (int s = 0; s < S->batch; ++s) {
+        S->h_reported[s] += n_tokens;
+        S->h_len[s] = tg.target_len[s];
+    }
+    S->tape.clear();
+    add_stats(S, ds, stats, ms, l0, s0);
+    return ADA_OK;
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+
+extern "C" {
+
+const char *ada_strerror(int code) {
+    switch (code) {
+        case ADA_OK: return "ok";
+        case ADA_EINVAL: return "invalid argument";
+        case ADA_ESTATE: return "wrong call order or missing tensor";
+        case ADA_ECAPACITY: return "capacity exceeded (KV pages, max_seq_len, max_early or scratch)";
+        case ADA_ECUDA: return "CUDA error";
+        case ADA_ETIMEOUT: return "bounded wait expired";
+        case ADA_EUNSUPPORTED: return "unsupported shape or dtype";
+        default: return "unknown error";
+    }
+}
+
+const char *ada_last_cuda_error(void) { return g_cuda_err.c_str(); }
+
+int ada_model_create(const ada_config *cfg, ada_model **out) {
+    if (!cfg || !out) return ADA_EINVAL;
+    int rc = check_cfg(*cfg);
+    if (rc) return rc;
+    ada_model *m = new ada_model();
+    m->cfg = *cfg;
+    m->esz = cfg->dtype == ADA_DTYPE_BF16 ? 2 : 4;
+    m->layers.resize(cfg->n_layers);
+    m->has_head.assign(cfg->n_layers + 1, 0);
+    m->head_T.assign(cfg->n_layers + 1, nullptr);
+    m->head_scale.assign(cfg->n_layers + 1, 1.0f);
+    *out = m;
+    return ADA_OK;
+}
+
+int ada_model_set_tensor(ada_model *m, const char *name, const void *dev_ptr, size_t bytes) {
+    if (!m || !name || !dev_ptr) return ADA_EINVAL;
+    if (m->finalized) return ADA_ESTATE;
+    if ((uintptr_t)dev_ptr % 16) return ADA_EINVAL;
+    const ada_config &g = m->cfg;
+    const size_t d = g.d_model, qd = (size_t)g.n_q_heads * g.head_dim;
+    const size_t qkv_rows = (size_t)(g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim;
+    size_t want = 0;
+    const void **slot = nullptr;
+    std::string n(name);
+    if (n == "tok_embed") { want = (size_t)g.vocab * d; slot = &m->tok_embed; }
+    else if (n == "lm_head") { if (g.tied_lm_head) return ADA_EINVAL; want = (size_t)g.vocab * d; slot = &m->lm_head; }
+    else if (n == "final_norm") { want = d; slot = &m->final_norm; }
+    else if (n.rfind("layers.", 0) == 0) {
+        size_t dot = n.find('.', 7);
+        if (dot == std::string::npos) return ADA_EINVAL;
+        int l = -1;
+        try { l = std::stoi(n.substr(7, dot - 7)); } catch (...) { return ADA_EINVAL; }
+        if (l < 0 || l >= g.n_layers) return ADA_EINVAL;
+        std::string f = n.substr(dot + 1);
+        LayerW &w = m->layers[l];
+        if (f == "attn_norm") { want = d; slot = &w.attn_norm; }
+        else if (f == "ffn_norm") { want = d; slot = &w.ffn_norm; }
+        else if (f == "wqkv") { want = qkv_rows * d; slot = &w.wqkv; }
+        else if (f == "wo") { want = d * qd; slot = &w.wo; }
+        else if (f == "w_gate_up") { want = 2 * (size_t)g.d_ff * d; slot = &w.w_gate_up; }
+        else if (f == "w_down") { want = d * (size_t)g.d_ff; slot = &w.w_down; }
+        else return ADA_EINVAL;
+    } else return ADA_EINVAL;
+    if (bytes != want * m->esz) return ADA_EINVAL;
+    *slot = dev_ptr;
+    return ADA_OK;
+}
+
+int ada_model_set_exit_head(ada_model *m, int32_t layer, const void *T_dev, float logit_scale) {
+    if (!m) return ADA_EINVAL;
+    if (layer < 1 || layer >= m->cfg.n_layers) return ADA_EINVAL;
+    if (!(logit_scale > 0.0f)) return ADA_EINVAL;
+    if (T_dev && (uintptr_t)T_dev % 16) return ADA_EINVAL;
+    m->has_head[layer] = 1;
+    m->head_T[layer] = T_dev;
+    m->head_scale[layer] = logit_scale;
+    return ADA_OK;
+}
+
+int ada_model_finalize(ada_model *m) {
+    if (!m) return ADA_EINVAL;
+    if (!m->tok_embed || !m->final_norm) return ADA_ESTATE;
+    if (m->cfg.tied_lm_head) m->lm_head = m->tok_embed;
+    if (!m->lm_head) return ADA_ESTATE;
+    for (const LayerW &w : m->layers)
+        if (!w.attn_norm || !w.wqkv || !w.wo || !w.ffn_norm || !w.w_gate_up || !w.w_down) return ADA_ESTATE;
+    m->finalized = true;
+    return ADA_OK;
+}
+
+void ada_model_destroy(ada_model *m) { delete m; }
+
+size_t ada_session_scratch_bytes(const ada_model *m, int32_t batch, int32_t max_seq_len, int32_t max_early) {
+    if (!m || batch < 1 || max_seq_len < 2 || max_early < 0) return 0;
+    return make_layout(m->cfg, batch, max_seq_len, max_early, kHeadBlocks).total;
+}
+
+size_t ada_kv_page_bytes(const ada_model *m, int32_t page_tokens) {
+    if (!m || page_tokens < 1) return 0;
+    const ada_config &g = m->cfg;
+    return (size_t)g.n_layers * 2 * g.n_kv_heads * page_tokens * g.head_dim * m->esz;
+}
+
+int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, int32_t page_tokens, int32_t max_early,
+                       void *kv_pool_dev, size_t kv_pool_bytes, void *scratch_dev, size_t scratch_bytes,
+                       void *cuda_stream, ada_session **out) {
+    if (!m || !out || !kv_pool_dev || !scratch_dev) return ADA_EINVAL;
+    if (!m->finalized) return ADA_ESTATE;
+    if (batch < 1 || batch > ADA_MAX_BATCH || max_seq_len < 2 || max_early < 0) return ADA_EINVAL;
+    if (page_tokens < 16 || page_tokens > 256 || (page_tokens & (page_tokens - 1))) return ADA_EINVAL;
+    if (batch * (max_early + 1) > kMaxRows) return ADA_ECAPACITY;
+    if ((uintptr_t)scratch_dev % 256 || (uintptr_t)kv_pool_dev % 256) return ADA_EINVAL;
+    const ada_config &g = m->cfg;
+    Layout lay = make_layout(g, batch, max_seq_len, max_early, kHeadBlocks);
+    if (scratch_bytes < lay.total) return ADA_ECAPACITY;
+    size_t page_bytes = ada_kv_page_bytes(m, page_tokens);
+    int n_pages = (int)std::min<size_t>(kv_pool_bytes / page_bytes, 1u << 30);
+    if (n_pages < 1) return ADA_ECAPACITY;
+
+    ada_session *S = new ada_session();
+    S->m = m;
+    S->batch = batch; S->max_seq = max_seq_len; S->page_tokens = page_tokens; S->max_early = max_early;
+    S->slots = max_early + 1;
+    S->rows_alloc = rows_alloc_for(batch, max_early);
+    S->n_pages = n_pages;
+    S->max_pages = (max_seq_len + 15) / 16;
+    S->n_chunks = (max_seq_len + kAttnChunk - 1) / kAttnChunk;
+    S->head_blocks = kHeadBlocks;
+    S->stream = (cudaStream_t)cuda_stream;
+    S->scratch = scratch_dev;
+    S->scratch_bytes = scratch_bytes;
+    char *b = (char *)scratch_dev;
+    Ctx &c = S->c;
+    c.d = g.d_model; c.nq = g.n_q_heads; c.nkv = g.n_kv_heads; c.hd = g.head_dim; c.dff = g.d_ff; c.vocab = g.vocab;
+    c.L = g.n_layers; c.qkv_rows = (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim; c.group = g.n_q_heads / g.n_kv_heads;
+    c.eps = g.rms_eps;
+    c.page_tokens = page_tokens;
+    c.page_shift = 0;
+    while ((1 << c.page_shift) < page_tokens) c.page_shift++;
+    c.max_pages = S->max_pages; c.max_seq = max_seq_len; c.slots = S->slots; c.n_chunks = S->n_chunks;
+    c.st = (DevState *)(b + lay.st); c.rt = (RowTable *)(b + lay.rt); c.fill = (int32_t *)(b + lay.fill);
+    c.tokens = (int32_t *)(b + lay.tokens); c.page_table = (int32_t *)(b + lay.page_table);
+    c.head_res = (HeadResult *)(b + lay.head_res); c.resid = (float *)(b + lay.resid); c.xn = (float *)(b + lay.xn);
+    c.qkv = (float *)(b + lay.qkv); c.q = (float *)(b + lay.q); c.attn_out = (float *)(b + lay.attn_out);
+    c.gu = (float *)(b + lay.gu); c.hact = (float *)(b + lay.hact); c.rope_cs = (float *)(b + lay.rope_cs);
+    c.attn_part = (float *)(b + lay.attn_part); c.head_part = (float *)(b + lay.head_part);
+    c.logit_stage = (float *)(b + lay.logit_stage); c.capture = nullptr; c.head_log = (float *)(b + lay.head_log);
+    c.kv_pool = kv_pool_dev;
+    S->t_out = (float *)(b + lay.t_out);
+
+    auto fail = [&](int code) { ada_session_destroy(S); return code; };
+#define CKS(expr)                                                                   \
+    do {                                                                            \
+        cudaError_t e__ = (expr);                                                   \
+        if (e__ != cudaSuccess) {                                                   \
+            g_cuda_err = std::string(#expr) + ": " + cudaGetErrorString(e__);       \
+            return fail(ADA_ECUDA);                                                 \
+        }                                                                           \
+    } while (0)
+    CKS(cudaMallocHost((void **)&S->pinned, 256));
+    CKS(cudaEventCreate(&S->ev0));
+    CKS(cudaEventCreate(&S->ev1));
+    CKS(cudaMemsetAsync(scratch_dev, 0, lay.total, S->stream));
+    DevState hs;
+    memset(&hs, 0, sizeof(hs));
+    hs.batch = batch; hs.slots = S->slots; hs.n_layers = g.n_layers; hs.max_seq = max_seq_len;
+    CKS(cudaMemcpyAsync(c.st, &hs, offsetof(DevState, len), cudaMemcpyHostToDevice, S->stream));
+    CKS(cudaStreamSynchronize(S->stream));
+#undef CKS
+    // free list: pages are handed out from the back, in a scrambled order so that the page-table
+    // indirection is always exercised
+    S->free_pages.resize(n_pages);
+    for (int i = 0; i < n_pages; ++i) S->free_pages[i] = (int)(((long long)i * 7919 + 13) % n_pages);
+    {
+        std::vector<char> seen(n_pages, 0);
+        bool perm = true;
+        for (int p : S->free_pages) { if (seen[p]) perm = false; seen[p] = 1; }
+        if (!perm) for (int i = 0; i < n_pages; ++i) S->free_pages[i] = n_pages - 1 - i;
+    }
+    S->seq_pages.resize(batch);
+    S->h_len.assign(batch, 0); S->h_prompt.assign(batch, 0); S->h_reported.assign(batch, 0);
+    S->prefilled.assign(batch, 0);
+    *out = S;
+    return ADA_OK;
+}
+
+void ada_session_destroy(ada_session *S) {
+    if (!S) return;
+    if (S->pinned) cudaFreeHost(S->pinned);
+    if (S->ev0) cudaEventDestroy(S->ev0);
+    if (S->ev1) cudaEventDestroy(S->ev1);
+    delete S;
+}
+
+int ada_session_reset(ada_session *S, int32_t seq) {
+    if (!S || seq >= S->batch) return ADA_EINVAL;
+    for (int s = 0; s < S->batch; ++s) {
+        if (seq >= 0 && s != seq) continue;
+        for (int p : S->seq_pages[s]) S->free_pages.push_back(p);
+        S->seq_pages[s].clear();
+        S->prefilled[s] = 0;
+        S->h_len[s] = S->h_prompt[s] = S->h_reported[s] = 0;
+    }
+    return ADA_OK;
+}
+
+int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t n_prompt) {
+    if (!S || !prompt_host || seq < 0 || seq >= S->batch || n_prompt < 1) return ADA_EINVAL;
+    const ada_model *m = S->m;
+    const ada_config &g = m->cfg;
+    if (n_prompt + 2 > S->max_seq) return ADA_ECAPACITY;
+    for (int i = 0; i < n_prompt; ++i) if (prompt_host[i] < 0 || prompt_host[i] >= g.vocab) return ADA_EINVAL;
+    int rc = ada_session_reset(S, seq);
+    if (rc) return rc;
+    if ((rc = ensure_pages(S, seq, n_prompt + 1))) return rc;
+    CK(cudaMemcpyAsync(S->c.tokens + (size_t)seq * S->max_seq, prompt_host, sizeof(int32_t) * n_prompt,
+                       cudaMemcpyHostToDevice, S->stream));
+    if (seq == 0 && S->capture_dev) {
+        int32_t zero = 0;
+        CK(cudaMemcpyAsync(&S->c.st->capture_n, &zero, sizeof(int32_t), cudaMemcpyHostToDevice, S->stream));
+    }
+    const int chunk = std::min(S->rows_alloc, kMaxRows);
+    for (int p0 = 0; p0 < n_prompt; p0 += chunk) {
+        const int n = std::min(chunk, n_prompt - p0);
+        const int last = p0 + n == n_prompt;
+        if (g.dtype == ADA_DTYPE_BF16)
+            k_prefill_begin<__nv_bfloat16><<<1, 256, 0, S->stream>>>(S->c, (const __nv_bfloat16 *)m->tok_embed, g.rope_base, seq, p0, n);
+        else
+            k_prefill_begin<float><<<1, 256, 0, S->stream>>>(S->c, (const float *)m->tok_embed, g.rope_base, seq, p0, n);
+        CK(cudaGetLastError());
+        for (int l = 0; l < g.n_layers; ++l) if ((rc = run_layer(S, l, n))) return rc;
+        if (last && (rc = run_head(S, 0, SEL_LAST, n))) return rc;
+        k_prefill_end<<<1, 32, 0, S->stream>>>(S->c, seq, p0 + n, last, n_prompt);
+        CK(cudaGetLastError());
+        if (last && seq == 0 && (rc = capture_rows(S, n - 1))) return rc;
+    }
+    CK(cudaStreamSynchronize(S->stream));
+    S->prefilled[seq] = 1;
+    S->h_prompt[seq] = n_prompt;
+    S->h_len[seq] = n_prompt + 1;
+    S->h_reported[seq] = 0;
+    return ADA_OK;
+}
+
+int ada_plain_decode(ada_session *S, int32_t n_tokens, int32_t *out_host, ada_stats *stats) {
+    if (!S) return ADA_EINVAL;
+    return decode(S, n_tokens, 2.0f, nullptr, 0, 0, out_host, stats);
+}
+
+int ada_adaptive_decode(ada_session *S, int32_t n_tokens, float threshold, const int32_t *exit_layers,
+                        int32_t n_exit_layers, int32_t max_early, int32_t *out_host, ada_stats *stats) {
+    if (!S || n_exit_layers < 0 || (n_exit_layers > 0 && !exit_layers)) return ADA_EINVAL;
+    return decode(S, n_tokens, threshold, exit_layers, n_exit_layers, max_early, out_host, stats);
+}
+
+int ada_debug_capture_logits(ada_session *S, float *dev_buf, int32_t max_tokens) {
+    if (!S || (dev_buf && max_tokens < 1)) return ADA_EINVAL;
+    S->capture_dev = dev_buf;
+    S->capture_cap = dev_buf ? max_tokens : 0;
+    S->c.capture = dev_buf;
+    int32_t v[2] = {S->capture_cap, 0};
+    CK(cudaMemcpyAsync(&S->c.st->capture_cap, v, sizeof(v), cudaMemcpyHostToDevice, S->stream));
+    CK(cudaStreamSynchronize(S->stream));
+    return ADA_OK;
+}
+
+int ada_debug_logits_captured(ada_session *S, int32_t *n_out) {
+    if (!S || !n_out) return ADA_EINVAL;
+    CK(cudaMemcpyAsync(n_out, &S->c.st->capture_n, sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+    CK(cudaStreamSynchronize(S->stream));
+    return ADA_OK;
+}
+
+int ada_debug_capture_heads(ada_session *S, float *host_buf, int32_t max_evals, int32_t *n_out) {
+    if (!S || (host_buf && max_evals < 1)) return ADA_EINVAL;
+    S->head_log_host = host_buf;
+    S->head_log_cap = host_buf ? std::min(max_evals, kHeadLogCap) : 0;
+    S->head_log_n_out = n_out;
+    return ADA_OK;
+}
+
+int ada_debug_set_exit_tape(ada_session *S, const uint8_t *tape_host, int32_t n) {
+    if (!S || n < 0 || n > kMaxTape || (n > 0 && !tape_host)) return ADA_EINVAL;
+    S->tape.assign(tape_host, tape_host + n);
+    return ADA_OK;
+}
+
+int ada_debug_get_state(ada_session *S, int32_t seq, int32_t *len_out, int32_t *fill_out) {
+    if (!S || seq < 0 || seq >= S->batch) return ADA_EINVAL;
+    if (len_out) CK(cudaMemcpyAsync(len_out, &S->c.st->len[seq], sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+    if (fill_out)
+        CK(cudaMemcpyAsync(fill_out, S->c.fill + (size_t)seq * S->m->cfg.n_layers, sizeof(int32_t) * S->m->cfg.n_layers,
+                           cudaMemcpyDeviceToHost, S->stream));
+    CK(cudaStreamSynchronize(S->stream));
+    return ADA_OK;
+}
+
+int ada_debug_read_kv(ada_session *S, int32_t seq, int32_t which, int32_t layer0, int32_t pos, float *host_out) {
+    if (!S || !host_out || seq < 0 || seq >= S->batch || which < 0 || which > 1) return ADA_EINVAL;
+    const ada_config &g = S->m->cfg;
+    if (layer0 < 0 || layer0 >= g.n_layers || pos < 0) return ADA_EINVAL;
+    int pi = pos / S->page_tokens;
+    if (pi >= (int)S->seq_pages[seq].size()) return ADA_EINVAL;
+    const int page = S->seq_pages[seq][pi], t = pos % S->page_tokens;
+    const size_t esz = S->m->esz;
+    std::vector<unsigned char> tmp((size_t)g.head_dim * esz);
+    for (int h = 0; h < g.n_kv_heads; ++h) {
+        size_t idx = ((((size_t)page * g.n_layers + layer0) * 2 + which) * g.n_kv_heads + h) *
+                         ((size_t)S->page_tokens * g.head_dim) + (size_t)t * g.head_dim;
+        CK(cudaMemcpy(tmp.data(), (const char *)S->c.kv_pool + idx * esz, tmp.size(), cudaMemcpyDeviceToHost));
+        for (int i = 0; i < g.head_dim; ++i) {
+            float f;
+            if (esz == 4) memcpy(&f, tmp.data() + 4 * i, 4);
+            else { uint32_t b = ((uint32_t)tmp[2 * i] | ((uint32_t)tmp[2 * i + 1] << 8)) << 16; memcpy(&f, &b, 4); }
+            host_out[h * g.head_dim + i] = f;
+        }
+    }
+    return ADA_OK;
+}
+
+int ada_debug_set_path(ada_session *S, int32_t path) {
+    if (!S || path < 0 || path > 1) return ADA_EINVAL;
+    if (path == 1) return ADA_EUNSUPPORTED;
+    S->path = path;
+    return ADA_OK;
+}
+
+}  // extern "C"

@@ -11,7 +11,12 @@ def widen(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().to(torch.float64).numpy()
 
 
-def np_decoder_logits(cfg, W, tokens, upto_layer=None, return_hidden=False):
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bf16 through torch's own conversion (fp64 -> fp32 -> bf16)."""
+    return torch.from_numpy(np.ascontiguousarray(x)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def np_decoder_logits(cfg, W, tokens, upto_layer=None, return_hidden=False, kv_bf16=False):
     """Final logits of every position, whole sequence at once, written with matrix ops, a
     causal mask and complex-number rotary embedding (a different formulation from the
     oracle's loops).  W: name -> float64 array in the fused layout."""
@@ -39,6 +44,8 @@ def np_decoder_logits(cfg, W, tokens, upto_layer=None, return_hidden=False):
         q = rope(qkv[:, :nq].reshape(n, Hq, hd))
         k = rope(qkv[:, nq:nq + nkv].reshape(n, Hkv, hd))
         v = qkv[:, nq + nkv:].reshape(n, Hkv, hd)
+        if kv_bf16:     # the cache holds bf16: K (rotated) and V are rounded when written
+            k, v = bf16_round(k), bf16_round(v)
         k = np.repeat(k, Hq // Hkv, axis=1)
         v = np.repeat(v, Hq // Hkv, axis=1)
         s = np.einsum("qhd,khd->hqk", q, k) / np.sqrt(hd)
@@ -57,11 +64,11 @@ def np_decoder_logits(cfg, W, tokens, upto_layer=None, return_hidden=False):
     return rms(x, W["final_norm"]) @ E.T
 
 
-def make_oracle(cfg, seed=1234, tied=True, jitter=0.05, heads=True, scale=None, **kw):
+def make_oracle(cfg, seed=1234, tied=True, jitter=0.05, heads=True, scale=None, kv_bf16=None, **kw):
     """(weights dict of torch tensors, oracle Model) with heads registered at cfg.exit_layers."""
     import oracle
     w = synth.make_weights(cfg, seed=seed, tied=tied, norm_gain_jitter=jitter)
-    m = oracle.model_from_torch(cfg, w)
+    m = oracle.model_from_torch(cfg, w, kv_bf16=kv_bf16)
     if heads:
         for l in cfg.exit_layers:
             m.set_head(l, None, cfg.logit_scale if scale is None else scale)

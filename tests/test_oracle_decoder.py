@@ -10,18 +10,23 @@ from paper_2506_03700_b200 import synth
 from helpers import make_oracle, np_decoder_logits, widen
 
 
-@pytest.mark.parametrize("dtype,tied,kv", [("fp32", True, 2), ("bf16", False, 6), ("fp32", False, 1)])
-def test_logits_match_numpy_restatement(dtype, tied, kv):
-    cfg = synth.small_config(dtype=dtype, n_kv_heads=kv, resid_scale=1.0)
-    w, m = make_oracle(cfg, tied=tied, heads=False)
+@pytest.mark.parametrize("dtype,tied,kv,kv_bf16", [("fp32", True, 2, False), ("bf16", False, 6, False),
+                                                    ("fp32", False, 1, False), ("bf16", True, 2, True)])
+def test_logits_match_numpy_restatement(dtype, tied, kv, kv_bf16):
+    """kv_bf16: the bf16 configurations keep K/V in a bf16 cache; the restatement rounds them with
+    torch's conversion, the oracle with its own bit arithmetic."""
+    cfg = synth.small_config(dtype=dtype, n_kv_heads=kv, resid_scale=1.0, sigma=0.1)
+    w, m = make_oracle(cfg, tied=tied, heads=False, kv_bf16=kv_bf16)
     W = {k: widen(v) for k, v in w.items()}
     toks = synth.make_prompt(cfg, n=13).numpy()
-    ref = np_decoder_logits(cfg, W, toks)
+    ref = np_decoder_logits(cfg, W, toks, kv_bf16=kv_bf16)
+    if kv_bf16:   # the rounding is not a no-op on this model
+        assert np.abs(ref - np_decoder_logits(cfg, W, toks)).max() > 1e-6
     got = m.full_logits(toks)
     assert np.abs(got - ref).max() < 1e-10 * max(1.0, np.abs(ref).max())
     # hidden state after an intermediate layer
     h = m.hidden_after(toks, 2)
-    href = np_decoder_logits(cfg, W, toks, upto_layer=2, return_hidden=True)[-1]
+    href = np_decoder_logits(cfg, W, toks, upto_layer=2, return_hidden=True, kv_bf16=kv_bf16)[-1]
     assert np.abs(h - href).max() < 1e-11
 
 
