@@ -69,6 +69,7 @@ typedef struct {
     int64_t row_layers;      /* sum over processed layers of the rows processed there */
     int64_t truncated;       /* verified tokens dropped to end a call on the requested count */
     int64_t exits_at_layer[ADA_MAX_LAYERS]; /* indexed by 1-based exit layer */
+    int64_t layer_passes;    /* decoder-layer passes launched (each streams one layer's weights once) */
     int64_t host_syncs;      /* stream synchronisations the decode loop needed */
     int64_t kernel_launches; /* kernels of this library launched by the decode calls */
     double decode_ms;        /* device time of the decode calls (CUDA events on the session stream) */
@@ -152,6 +153,14 @@ int ada_debug_get_state(ada_session *s, int32_t seq, int32_t *len_out, int32_t *
 /* Copy K (which=0) or V (which=1) of one cached position of one layer into host_out
  * [n_kv_heads*head_dim] as fp32. */
 int ada_debug_read_kv(ada_session *s, int32_t seq, int32_t which, int32_t layer0, int32_t pos, float *host_out);
+/* Per-kernel-class device timing (CUDA events around every launch; slows the run, for analysis
+ * only).  Classes: 0 step set-up and control, 1 RMSNorm, 2 QKV GEMM, 3 RoPE + KV write, 4 attention,
+ * 5 O-proj GEMM, 6 gate/up GEMM, 7 SwiGLU, 8 down GEMM, 9 LM-head stream, 10 head transformation T,
+ * 11 other.  ada_debug_profile_read returns, accumulated since profiling was switched on, the device
+ * milliseconds, launch counts and algorithmic HBM bytes (weights or KV the launch must read) per class. */
+#define ADA_PROF_CLASSES 12
+int ada_debug_profile(ada_session *s, int32_t on);
+int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out, double *bytes_out);
 /* Select the GEMM path: 0 = CUDA-core kernels (any dtype), 1 = tensor-core kernels (bf16 only). */
 int ada_debug_set_path(ada_session *s, int32_t path);
 

@@ -27,6 +27,7 @@ EXPORTS = [
     "ada_session_create", "ada_session_destroy", "ada_session_reset", "ada_prefill", "ada_plain_decode",
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
+    "ada_debug_profile", "ada_debug_profile_read",
 ]
 
 
@@ -55,7 +56,7 @@ class Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in
                 ("steps", "head_evals", "early_exits", "verify_steps", "accepted", "rejected", "discarded",
                  "row_layers", "truncated")] + \
-               [("exits_at_layer", C.c_int64 * ADA_MAX_LAYERS), ("host_syncs", C.c_int64),
+               [("exits_at_layer", C.c_int64 * ADA_MAX_LAYERS), ("layer_passes", C.c_int64), ("host_syncs", C.c_int64),
                 ("kernel_launches", C.c_int64), ("decode_ms", C.c_double)]
 
     def as_dict(self) -> dict:
@@ -101,6 +102,8 @@ def load() -> C.CDLL:
         L.ada_debug_get_state.argtypes = [vp, i32, C.POINTER(i32), vp]
         L.ada_debug_read_kv.argtypes = [vp, i32, i32, i32, i32, vp]
         L.ada_debug_set_path.argtypes = [vp, i32]
+        L.ada_debug_profile.argtypes = [vp, i32]
+        L.ada_debug_profile_read.argtypes = [vp, vp, vp, vp]
         _LIB = L
     return _LIB
 
@@ -240,6 +243,21 @@ class Session:
         out = np.zeros(c.n_kv_heads * c.head_dim, dtype=np.float32)
         _ck(load().ada_debug_read_kv(self.h, seq, which, layer0, pos, out.ctypes.data), "ada_debug_read_kv")
         return out
+
+    PROF_CLASSES = ("control", "rmsnorm", "qkv_gemm", "rope_kv", "attention", "o_gemm", "gate_up_gemm", "swiglu",
+                    "down_gemm", "lm_head", "head_T", "other")
+
+    def profile(self, on: bool):
+        _ck(load().ada_debug_profile(self.h, 1 if on else 0), "ada_debug_profile")
+
+    def profile_read(self) -> dict:
+        """class -> dict(ms, launches, bytes) accumulated since profiling was switched on."""
+        n = len(self.PROF_CLASSES)
+        ms = np.zeros(n, dtype=np.float64)
+        la = np.zeros(n, dtype=np.int64)
+        by = np.zeros(n, dtype=np.float64)
+        _ck(load().ada_debug_profile_read(self.h, ms.ctypes.data, la.ctypes.data, by.ctypes.data), "ada_debug_profile_read")
+        return {c: dict(ms=float(ms[i]), launches=int(la[i]), bytes=float(by[i])) for i, c in enumerate(self.PROF_CLASSES)}
 
     def set_path(self, path: int):
         _ck(load().ada_debug_set_path(self.h, path), "ada_debug_set_path")

@@ -59,7 +59,13 @@ struct ada_session {
     int32_t *pinned = nullptr; // small read-back area
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     int path = 0;
-    int64_t launches = 0, syncs = 0;
+    int64_t launches = 0, syncs = 0, layer_passes = 0;
+    // per-class profiling
+    bool prof = false;
+    std::vector<cudaEvent_t> prof_ev;
+    std::vector<std::pair<int, double>> prof_rec;  // (class, bytes) per recorded launch
+    double prof_ms[ADA_PROF_CLASSES] = {0}, prof_bytes[ADA_PROF_CLASSES] = {0};
+    int64_t prof_launches[ADA_PROF_CLASSES] = {0};
     // debug
     float *capture_dev = nullptr;
     int capture_cap = 0;
@@ -121,10 +127,47 @@ int check_cfg(const ada_config &g) {
     return ADA_OK;
 }
 
+// ---- profiling: events around every launch when switched on ------------------------------------
+
+constexpr size_t kProfMaxRec = 1 << 17;
+
+struct Prof {
+    ada_session *S;
+    bool on;
+    Prof(ada_session *S_, int cls, double bytes) : S(S_), on(S_->prof && S_->prof_rec.size() < kProfMaxRec) {
+        if (!on) return;
+        size_t i = S->prof_rec.size();
+        while (S->prof_ev.size() < 2 * (i + 1)) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+            S->prof_ev.push_back(e);
+        }
+        S->prof_rec.push_back({cls, bytes});
+        cudaEventRecord(S->prof_ev[2 * i], S->stream);
+    }
+    ~Prof() {
+        if (on) cudaEventRecord(S->prof_ev[2 * (S->prof_rec.size() - 1) + 1], S->stream);
+    }
+};
+
+// Fold the recorded events into the per-class sums (stream must be idle).
+void prof_collect(ada_session *S) {
+    for (size_t i = 0; i < S->prof_rec.size(); ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, S->prof_ev[2 * i], S->prof_ev[2 * i + 1]) != cudaSuccess) continue;
+        int cls = S->prof_rec[i].first;
+        S->prof_ms[cls] += ms;
+        S->prof_bytes[cls] += S->prof_rec[i].second;
+        S->prof_launches[cls] += 1;
+    }
+    S->prof_rec.clear();
+}
+
 // ---- typed launch helpers --------------------------------------------------------------------
 
 template <typename T>
-int launch_gemv(ada_session *S, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy, int sel) {
+int launch_gemv(ada_session *S, int cls, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy, int sel) {
+    Prof pf(S, cls, (double)N * K * sizeof(T));
     int blocks = std::min((N + 7) / 8, 148 * 4);
     if (epi == 0)
         k_gemv<T, 0><<<blocks, 256, 0, S->stream>>>(S->c, (const T *)W, N, K, X, ldx, Y, ldy, sel);
@@ -138,6 +181,7 @@ int launch_gemv(ada_session *S, int epi, const void *W, int N, int K, const floa
 template <typename T>
 int launch_attn(ada_session *S, int layer, int rows) {
     const ada_config &g = S->m->cfg;
+    Prof pf(S, 4, 0.0);
     dim3 grid(S->n_chunks, g.n_q_heads, rows);
     switch (g.head_dim / 32) {
         case 1: k_attn_partial<T, 1><<<grid, 32, 0, S->stream>>>(S->c, layer); break;
@@ -165,23 +209,36 @@ int run_layer_t(ada_session *S, int layer, int rows) {
     const int d = g.d_model, qd = g.n_q_heads * g.head_dim, qkv_rows = S->c.qkv_rows;
     const int ldx = d;
     int rc;
-    k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)w.attn_norm, layer, S->c.xn, ldx);
+    S->layer_passes++;
+    {
+        Prof pf(S, 1, 0.0);
+        k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)w.attn_norm, layer, S->c.xn, ldx);
+    }
     CK(cudaGetLastError());
     S->launches++;
-    if ((rc = launch_gemv<T>(S, 0, w.wqkv, qkv_rows, d, S->c.xn, ldx, S->c.qkv, qkv_rows, layer))) return rc;
-    k_rope_kv<T><<<rows, 128, 0, S->stream>>>(S->c, layer);
+    if ((rc = launch_gemv<T>(S, 2, 0, w.wqkv, qkv_rows, d, S->c.xn, ldx, S->c.qkv, qkv_rows, layer))) return rc;
+    {
+        Prof pf(S, 3, 0.0);
+        k_rope_kv<T><<<rows, 128, 0, S->stream>>>(S->c, layer);
+    }
     CK(cudaGetLastError());
     S->launches++;
     if ((rc = launch_attn<T>(S, layer, rows))) return rc;
-    if ((rc = launch_gemv<T>(S, 1, w.wo, d, qd, S->c.attn_out, qd, S->c.resid, d, layer))) return rc;
-    k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)w.ffn_norm, layer, S->c.xn, ldx);
+    if ((rc = launch_gemv<T>(S, 5, 1, w.wo, d, qd, S->c.attn_out, qd, S->c.resid, d, layer))) return rc;
+    {
+        Prof pf(S, 1, 0.0);
+        k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)w.ffn_norm, layer, S->c.xn, ldx);
+    }
     CK(cudaGetLastError());
     S->launches++;
-    if ((rc = launch_gemv<T>(S, 0, w.w_gate_up, 2 * g.d_ff, d, S->c.xn, ldx, S->c.gu, 2 * g.d_ff, layer))) return rc;
-    k_swiglu<<<dim3((g.d_ff + 255) / 256, rows), 256, 0, S->stream>>>(S->c, layer);
+    if ((rc = launch_gemv<T>(S, 6, 0, w.w_gate_up, 2 * g.d_ff, d, S->c.xn, ldx, S->c.gu, 2 * g.d_ff, layer))) return rc;
+    {
+        Prof pf(S, 7, 0.0);
+        k_swiglu<<<dim3((g.d_ff + 255) / 256, rows), 256, 0, S->stream>>>(S->c, layer);
+    }
     CK(cudaGetLastError());
     S->launches++;
-    if ((rc = launch_gemv<T>(S, 1, w.w_down, d, g.d_ff, S->c.hact, g.d_ff, S->c.resid, d, layer))) return rc;
+    if ((rc = launch_gemv<T>(S, 8, 1, w.w_down, d, g.d_ff, S->c.hact, g.d_ff, S->c.resid, d, layer))) return rc;
     return ADA_OK;
 }
 
@@ -193,7 +250,10 @@ int run_head_t(ada_session *S, int layer1, int sel, int rows) {
     const ada_config &g = m->cfg;
     const int d = g.d_model;
     int rc;
-    k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)m->final_norm, sel, S->c.xn, d);
+    {
+        Prof pf(S, 1, 0.0);
+        k_rmsnorm<T><<<rows, 256, 0, S->stream>>>(S->c, (const T *)m->final_norm, sel, S->c.xn, d);
+    }
     CK(cudaGetLastError());
     S->launches++;
     const float *x = S->c.xn;
@@ -201,14 +261,17 @@ int run_head_t(ada_session *S, int layer1, int sel, int rows) {
     if (layer1 > 0) {
         scale = m->head_scale[layer1];
         if (m->head_T[layer1]) {
-            if ((rc = launch_gemv<T>(S, 0, m->head_T[layer1], d, d, S->c.xn, d, S->t_out, d, sel))) return rc;
+            if ((rc = launch_gemv<T>(S, 10, 0, m->head_T[layer1], d, d, S->c.xn, d, S->t_out, d, sel))) return rc;
             x = S->t_out;
         }
     }
     const int store = (layer1 == 0 && S->capture_dev) ? 1 : 0;
-    k_head_partial<T><<<S->head_blocks, 256, 0, S->stream>>>(S->c, (const T *)m->lm_head, x, d, scale, sel, store);
-    CK(cudaGetLastError());
-    k_head_final<<<rows, 32, 0, S->stream>>>(S->c, S->head_blocks, sel);
+    {
+        Prof pf(S, 9, (double)g.vocab * d * sizeof(T));
+        k_head_partial<T><<<S->head_blocks, 256, 0, S->stream>>>(S->c, (const T *)m->lm_head, x, d, scale, sel, store);
+        CK(cudaGetLastError());
+        k_head_final<<<rows, 32, 0, S->stream>>>(S->c, S->head_blocks, sel);
+    }
     CK(cudaGetLastError());
     S->launches += 2;
     return ADA_OK;
@@ -223,6 +286,7 @@ int run_head(ada_session *S, int layer1, int sel, int rows) {
 
 int step_begin(ada_session *S) {
     const ada_model *m = S->m;
+    Prof pf(S, 0, 0.0);
     if (m->cfg.dtype == ADA_DTYPE_BF16)
         k_step_begin<__nv_bfloat16><<<1, 256, 0, S->stream>>>(S->c, (const __nv_bfloat16 *)m->tok_embed, m->cfg.rope_base);
     else
@@ -234,6 +298,7 @@ int step_begin(ada_session *S) {
 
 int capture_rows(ada_session *S, int row0) {
     if (!S->capture_dev) return ADA_OK;
+    Prof pf(S, 11, 0.0);
     k_capture<<<64, 256, 0, S->stream>>>(S->c, row0);
     CK(cudaGetLastError());
     k_capture_advance<<<1, 32, 0, S->stream>>>(S->c);
@@ -266,12 +331,13 @@ int ensure_pages(ada_session *S, int seq, int positions) {
     return ADA_OK;
 }
 
-void add_stats(ada_session *S, const DevStats &d, ada_stats *out, float ms, int64_t l0, int64_t s0) {
+void add_stats(ada_session *S, const DevStats &d, ada_stats *out, float ms, int64_t l0, int64_t s0, int64_t p0) {
     if (!out) return;
     out->steps += d.steps; out->head_evals += d.head_evals; out->early_exits += d.early_exits;
     out->verify_steps += d.verify_steps; out->accepted += d.accepted; out->rejected += d.rejected;
     out->discarded += d.discarded; out->row_layers += d.row_layers; out->truncated += d.truncated;
     for (int i = 0; i < ADA_MAX_LAYERS; ++i) out->exits_at_layer[i] += d.exits_at_layer[i];
+    out->layer_passes += S->layer_passes - p0;
     out->host_syncs += S->syncs - s0;
     out->kernel_launches += S->launches - l0;
     out->decode_ms += ms;
@@ -300,7 +366,7 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
         tg.target_len[s] = target;
         max_steps_plain = std::max(max_steps_plain, target - S->h_len[s]);
     }
-    const int64_t l0 = S->launches, s0 = S->syncs;
+    const int64_t l0 = S->launches, s0 = S->syncs, p0 = S->layer_passes;
     const int rows = S->batch * S->slots;
     int rc;
     // zero the device counters, set targets
@@ -319,7 +385,10 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
             if ((rc = step_begin(S))) return rc;
             for (int l = 0; l < L; ++l) if ((rc = run_layer(S, l, rows))) return rc;
             if ((rc = run_head(S, 0, SEL_FINAL, rows))) return rc;
-            k_verify<<<1, 32, 0, S->stream>>>(S->c);
+            {
+                Prof pf(S, 0, 0.0);
+                k_verify<<<1, 32, 0, S->stream>>>(S->c);
+            }
             CK(cudaGetLastError());
             S->launches++;
             if ((rc = capture_rows(S, 0))) return rc;
@@ -338,7 +407,10 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
                 if ((rc = run_layer(S, l, rows))) return rc;
                 if (e_i < n_exit && exit_layers[e_i] == l + 1) {
                     if ((rc = run_head(S, l + 1, SEL_HEAD, rows))) return rc;
-                    k_exit_control<<<1, 32, 0, S->stream>>>(S->c, l + 1);
+                    {
+                        Prof pf(S, 0, 0.0);
+                        k_exit_control<<<1, 32, 0, S->stream>>>(S->c, l + 1);
+                    }
                     CK(cudaGetLastError());
                     S->launches++;
                     ++e_i;
@@ -348,7 +420,10 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
             }
             if (reached_top) {
                 if ((rc = run_head(S, 0, SEL_FINAL, rows))) return rc;
-                k_verify<<<1, 32, 0, S->stream>>>(S->c);
+                {
+                    Prof pf(S, 0, 0.0);
+                    k_verify<<<1, 32, 0, S->stream>>>(S->c);
+                }
                 CK(cudaGetLastError());
                 S->launches++;
                 if ((rc = capture_rows(S, 0))) return rc;
@@ -383,7 +458,8 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
         S->h_len[s] = tg.target_len[s];
     }
     S->tape.clear();
-    add_stats(S, ds, stats, ms, l0, s0);
+    if (S->prof) prof_collect(S);
+    add_stats(S, ds, stats, ms, l0, s0, p0);
     return ADA_OK;
 }
 
@@ -580,6 +656,7 @@ void ada_session_destroy(ada_session *S) {
     if (S->pinned) cudaFreeHost(S->pinned);
     if (S->ev0) cudaEventDestroy(S->ev0);
     if (S->ev1) cudaEventDestroy(S->ev1);
+    for (cudaEvent_t e : S->prof_ev) cudaEventDestroy(e);
     delete S;
 }
 
@@ -705,6 +782,28 @@ int ada_debug_read_kv(ada_session *S, int32_t seq, int32_t which, int32_t layer0
             else { uint32_t b = ((uint32_t)tmp[2 * i] | ((uint32_t)tmp[2 * i + 1] << 8)) << 16; memcpy(&f, &b, 4); }
             host_out[h * g.head_dim + i] = f;
         }
+    }
+    return ADA_OK;
+}
+
+int ada_debug_profile(ada_session *S, int32_t on) {
+    if (!S) return ADA_EINVAL;
+    CK(cudaStreamSynchronize(S->stream));
+    if (on && !S->prof) {
+        for (int i = 0; i < ADA_PROF_CLASSES; ++i) { S->prof_ms[i] = 0; S->prof_bytes[i] = 0; S->prof_launches[i] = 0; }
+        S->prof_rec.clear();
+    }
+    if (!on && S->prof) prof_collect(S);
+    S->prof = on != 0;
+    return ADA_OK;
+}
+
+int ada_debug_profile_read(ada_session *S, double *ms_out, int64_t *launches_out, double *bytes_out) {
+    if (!S || !ms_out || !launches_out || !bytes_out) return ADA_EINVAL;
+    CK(cudaStreamSynchronize(S->stream));
+    prof_collect(S);
+    for (int i = 0; i < ADA_PROF_CLASSES; ++i) {
+        ms_out[i] = S->prof_ms[i]; launches_out[i] = S->prof_launches[i]; bytes_out[i] = S->prof_bytes[i];
     }
     return ADA_OK;
 }
