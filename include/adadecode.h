@@ -164,6 +164,22 @@ int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out
 /* Select the GEMM path: 0 = CUDA-core kernels (any dtype), 1 = tensor-core kernels (bf16 only). */
 int ada_debug_set_path(ada_session *s, int32_t path);
 
+/* Run the weight-streaming skinny GEMM of the decode kernel by itself (the kernel behind the QKV,
+ * O, gate/up, down and LM-head products of a layer pass, Algorithm 1 "process all tokens in P[l]
+ * in parallel"): bf16 weights W_dev [N, K] row-major, fp32 activations X_dev [cols, K], 1 <= cols
+ * <= 8, fp32 result Y_dev [cols, ldy].
+ *   mode 0: Y[c][n] = sum_k W[n][k] X[c][k], n < N.
+ *   mode 1: W stacks a gate matrix over an up matrix (N/2 rows each, N/2 a multiple of 16):
+ *           Y[c][n] = silu(gate_n . X[c]) * (up_n . X[c]), n < N/2.
+ * K must be a multiple of 64.  work_dev is device scratch of at least ada_debug_gemm_work_bytes(K)
+ * bytes, 256-byte aligned.  The product is launched `repeat` >= 1 times back to back inside one
+ * kernel; *ms_out (nullable) receives the device time of that kernel.  All pointers except ms_out
+ * are device pointers.  Returns ADA_ETIMEOUT if a bounded device-side wait expired. */
+size_t ada_debug_gemm_work_bytes(int32_t K);
+int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols,
+                   void *work_dev, size_t work_bytes, float *Y_dev, int32_t ldy, int32_t repeat, void *cuda_stream,
+                   float *ms_out);
+
 #ifdef __cplusplus
 }
 #endif

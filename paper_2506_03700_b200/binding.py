@@ -27,7 +27,7 @@ EXPORTS = [
     "ada_session_create", "ada_session_destroy", "ada_session_reset", "ada_prefill", "ada_plain_decode",
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
-    "ada_debug_profile", "ada_debug_profile_read",
+    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_work_bytes",
 ]
 
 
@@ -104,6 +104,9 @@ def load() -> C.CDLL:
         L.ada_debug_set_path.argtypes = [vp, i32]
         L.ada_debug_profile.argtypes = [vp, i32]
         L.ada_debug_profile_read.argtypes = [vp, vp, vp, vp]
+        L.ada_debug_gemm_work_bytes.restype = sz
+        L.ada_debug_gemm_work_bytes.argtypes = [i32]
+        L.ada_debug_gemm.argtypes = [vp, i32, i32, i32, vp, i32, vp, sz, vp, i32, i32, vp, C.POINTER(C.c_float)]
         _LIB = L
     return _LIB
 
@@ -111,6 +114,26 @@ def load() -> C.CDLL:
 def _ck(rc: int, where: str):
     if rc != 0:
         raise AdaError(rc, where)
+
+
+def debug_gemm(W, X, mode: int = 0, repeat: int = 1):
+    """The weight-streaming GEMM by itself: W bf16 [N, K] (cuda), X fp32 [cols, K] (cuda).
+    Returns (Y fp32 [cols, N or N/2], device milliseconds of the kernel)."""
+    import torch
+    lib = load()
+    N, K = W.shape
+    cols = X.shape[0]
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.is_contiguous()
+    assert X.is_cuda and X.dtype == torch.float32 and X.is_contiguous() and X.shape[1] == K
+    n_out = N // 2 if mode == 1 else N
+    wb = lib.ada_debug_gemm_work_bytes(K)
+    work = torch.empty(wb + 256, dtype=torch.uint8, device="cuda")
+    off = (-work.data_ptr()) % 256
+    Y = torch.zeros(cols, n_out, dtype=torch.float32, device="cuda")
+    ms = C.c_float(0.0)
+    _ck(lib.ada_debug_gemm(W.data_ptr(), N, K, mode, X.data_ptr(), cols, work.data_ptr() + off, wb, Y.data_ptr(), n_out,
+                           repeat, torch.cuda.current_stream().cuda_stream, C.byref(ms)), "ada_debug_gemm")
+    return Y, ms.value
 
 
 class Model:

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "kernels.cuh"
+#include "gemm_probe.cuh"
 
 using namespace ada;
 
@@ -30,6 +31,39 @@ struct LayerW {
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Tensor map of a row-major bf16 weight matrix [N][K] for the streaming GEMM: dimensions (64
+// elements, N rows, K/64 groups), box (64, 16, 8), 128-byte swizzle, zero fill outside.  The
+// driver entry point is looked up at run time, so the library loads without libcuda.
+int make_weight_map(CUtensorMap *out, const void *W, int N, int K) {
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        cudaError_t e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qr);
+        if (e != cudaSuccess || qr != cudaDriverEntryPointSuccess || !fn) {
+            g_cuda_err = std::string("cuTensorMapEncodeTiled is not available: ") + cudaGetErrorString(e);
+            return ADA_ECUDA;
+        }
+        encode = (EncodeFn)fn;
+    }
+    if (K % 64 || N < 1 || (uintptr_t)W % 16) return ADA_EUNSUPPORTED;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)N, (cuuint64_t)(K / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)st::TILE_N, (cuuint32_t)st::KG};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(W), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_cuda_err = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string((int)r);
+        return ADA_ECUDA;
+    }
+    return ADA_OK;
+}
 
 }  // namespace
 
@@ -813,6 +847,52 @@ int ada_debug_set_path(ada_session *S, int32_t path) {
     if (path == 1) return ADA_EUNSUPPORTED;
     S->path = path;
     return ADA_OK;
+}
+
+size_t ada_debug_gemm_work_bytes(int32_t K) {
+    if (K < 64) return 0;
+    return st::xfrag_bytes(K) + 512;
+}
+
+int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols, void *work_dev,
+                   size_t work_bytes, float *Y_dev, int32_t ldy, int32_t repeat, void *cuda_stream, float *ms_out) {
+    if (!W_dev || !X_dev || !work_dev || !Y_dev || N < 1 || K < 64 || K % 64 || cols < 1 || cols > st::MAX_COLS) return ADA_EINVAL;
+    if (mode < 0 || mode > 1 || repeat < 1) return ADA_EINVAL;
+    if (mode == 1 && (N % 2 || (N / 2) % 16)) return ADA_EINVAL;
+    if ((uintptr_t)W_dev % 16 || (uintptr_t)work_dev % 256 || ldy < (mode == 1 ? N / 2 : N)) return ADA_EINVAL;
+    if (work_bytes < ada_debug_gemm_work_bytes(K)) return ADA_ECAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int dev = 0, sms = 0;
+    CK(cudaGetDevice(&dev));
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CK(cudaFuncSetAttribute(k_gemm_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st::SMEM_BYTES));
+    int *err = (int *)((char *)work_dev + st::xfrag_bytes(K));
+    CUtensorMap *dmap = (CUtensorMap *)((char *)work_dev + st::xfrag_bytes(K) + 256);
+    CUtensorMap hmap;
+    int rc = make_weight_map(&hmap, W_dev, N, K);
+    if (rc) return rc;
+    CK(cudaMemsetAsync(err, 0, sizeof(int), stream));
+    CK(cudaMemcpyAsync(dmap, &hmap, sizeof(hmap), cudaMemcpyHostToDevice, stream));
+    CK(cudaStreamSynchronize(stream));   // hmap lives on this stack frame
+    k_xfrag_pack<<<(K + 255) / 256, 256, 0, stream>>>(X_dev, K, cols, (__nv_bfloat16 *)work_dev);
+    CK(cudaGetLastError());
+    cudaEvent_t e0, e1;
+    CK(cudaEventCreate(&e0));
+    CK(cudaEventCreate(&e1));
+    cudaEventRecord(e0, stream);
+    k_gemm_probe<<<sms, st::THREADS, st::SMEM_BYTES, stream>>>(dmap, N, K, mode, (const uint4 *)work_dev, Y_dev, ldy, cols, repeat, err);
+    cudaError_t le = cudaGetLastError();
+    cudaEventRecord(e1, stream);
+    int herr = 0;
+    cudaError_t ce = le == cudaSuccess ? cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, stream) : le;
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+    float ms = 0.f;
+    if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    CK(ce);
+    if (ms_out) *ms_out = ms;
+    return herr ? ADA_ETIMEOUT : ADA_OK;
 }
 
 }  // extern "C"

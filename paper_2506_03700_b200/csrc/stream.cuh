@@ -1,0 +1,402 @@
+// Weight-streaming primitives of the persistent decode kernel (sm_100a).
+//
+// The decode step is bound by HBM bandwidth: every weight byte is read once per pass and used
+// for at most eight tokens.  The pieces here keep the memory pipe full:
+//   * weights reach shared memory through TMA tensor copies (cp.async.bulk.tensor, one 16 KB box
+//     of 16 rows x 512 k per instruction, 128-byte swizzled) issued by a dedicated producer warp
+//     into a ring of stages guarded by mbarriers; the producer runs ahead of the consumers across
+//     phase boundaries, because the weight sequence of a CTA does not depend on activations.
+//     (Sixteen 1 KB untiled bulk copies per stage reached only 3.6 TB/s on B200: the copy engine
+//     spends about 40 ns per request whatever its size, so requests have to be large.)
+//   * activations arrive through a second, small ring in the register layout the tensor-core
+//     instruction wants, already split into a bf16 high part and a bf16 low part, so that
+//     fp32 activations lose nothing: W.x = W.hi(x) + W.lo(x) with fp32 accumulation;
+//   * eight consumer warps multiply with mma.sync m16n8k16 (weights are the 16-row operand, the
+//     up-to-eight tokens are the 8 columns).  The tensor cores are used as a cheap way to issue
+//     the multiply-adds; the bound stays the memory system.
+//   * all CTAs of the persistent grid meet at a counter-based grid barrier between phases.
+// Every wait is bounded: on expiry an error word is set and all later waits fall through.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ada {
+namespace st {
+
+constexpr int KC = 512;                          // k elements per stage
+constexpr int KSTEPS = KC / 16;                  // mma k-steps per stage
+constexpr int TILE_N = 16;                       // weight rows per stage (mma M)
+constexpr int KG = KC / 64;                      // 64-element (128-byte) k groups per stage
+constexpr int W_STAGE = TILE_N * KC * 2;         // 16384: [k group][row][128 B, 16-byte chunks xor-swizzled by row%8]
+constexpr int X_STAGE = KSTEPS * 32 * 16;        // 16384: [k-step][lane][b0.hi b1.hi b0.lo b1.lo]
+constexpr int NW = 10;                           // weight stages in flight per CTA
+constexpr int NX = 3;                            // activation stages
+constexpr int CONS_WARPS = 8;
+constexpr int CONS_THREADS = CONS_WARPS * 32;
+constexpr int THREADS = CONS_THREADS + 64;       // + weight producer warp + activation producer warp
+constexpr int MAX_COLS = 8;                      // tokens per pass (mma N)
+constexpr int RED_BYTES = CONS_WARPS * 2 * 128 * 4;  // cross-warp reduction scratch (two tiles per warp)
+
+constexpr int ERR_TIMEOUT_MBAR = 1, ERR_TIMEOUT_GRID = 2;
+constexpr unsigned long long WAIT_NS = 2000000000ull;   // a single wait gives up after two seconds
+
+struct Smem {                                    // must start on a 1024-byte boundary (swizzle pattern)
+    alignas(1024) unsigned char w[NW][W_STAGE];
+    alignas(128) unsigned char x[NX][X_STAGE];
+    alignas(16) float red[RED_BYTES / 4];
+    alignas(16) float vec[64];                    // per-column scalars (rstd, ...)
+    alignas(8) unsigned long long w_full[NW], w_empty[NW], x_full[NX], x_empty[NX];
+    int abort;
+    int bcast[8];
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t s32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(unsigned long long *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(s32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+// Bulk copy global -> shared of `bytes` (multiple of 16; both addresses 16-byte aligned), completing
+// on `bar` with the byte count.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, unsigned long long *bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(s32(dst)),
+        "l"(src), "r"(bytes), "r"(s32(bar)), "l"(pol)
+        : "memory");
+}
+// TMA tensor copy of one box of a rank-3 map (coordinates innermost first) into shared memory.
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, unsigned long long *bar,
+                                            uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(
+            s32(dst)),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(s32(bar)), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                 : "r"(s32(p)));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&a)[4], const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                 : "r"(s32(p)));
+}
+// d += a (16x16, row) * b (16x8, col), bf16 inputs, fp32 accumulation.
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, %0;" ::"n"(CONS_THREADS) : "memory"); }
+
+__device__ __forceinline__ uint32_t ld_acquire(const unsigned *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// ---------------------------------------------------------------- bounded waits
+
+struct Shared {            // what every role needs to wait safely
+    Smem *sm;
+    int *err;              // global error word (0 = fine)
+};
+
+__device__ __forceinline__ bool aborted(const Shared &S) { return *(volatile int *)&S.sm->abort != 0; }
+
+__device__ __noinline__ void raise_error(const Shared &S, int code) {
+    atomicCAS(S.err, 0, code);
+    *(volatile int *)&S.sm->abort = 1;
+}
+
+// Wait for an mbarrier phase.  Once an error is raised (here or anywhere in the grid) every wait
+// falls through at once: the roles then run to the end of their loops on whatever data is there,
+// so that no warp is left behind at a block-level barrier, and the kernel ends.
+__device__ __forceinline__ void mbar_wait(const Shared &S, unsigned long long *bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return;
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try(bar, parity)) return;
+        if ((it & 127u) == 0) {
+            if (aborted(S)) return;
+            if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
+            unsigned long long t = gtime();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > WAIT_NS) { raise_error(S, ERR_TIMEOUT_MBAR); return; }
+        }
+    }
+}
+
+// Grid barrier on a monotonically increasing counter: arrive once per CTA, wait for `target`.
+__device__ __forceinline__ void grid_arrive(unsigned *ctr) {
+    __threadfence();
+    fence_proxy_async();
+    red_release_add(ctr, 1u);
+}
+__device__ __forceinline__ void grid_wait(const Shared &S, const unsigned *ctr, unsigned target) {
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (ld_acquire(ctr) >= target) return;
+        if ((it & 63u) == 0) {
+            if (aborted(S)) return;
+            if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
+            unsigned long long t = gtime();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > WAIT_NS) { raise_error(S, ERR_TIMEOUT_GRID); return; }
+        }
+        __nanosleep(32);
+    }
+}
+
+// ---------------------------------------------------------------- activation layout
+
+// Activations for a GEMM of depth K live in global memory as ceil(K/KC) blocks of X_STAGE bytes;
+// block c, k-step s, lane l holds 16 bytes: the mma B fragment (b0, b1) of the bf16 high parts,
+// then of the bf16 low parts, for token column l/4 and k = 16 s + 2 (l%4) + {0,1} (+8 for b1).
+__device__ __forceinline__ size_t xfrag_index(int k, int col) {   // index in 2-byte units of the high part
+    const int chunk = k / KC, ks = (k % KC) >> 4, kk = k & 15;
+    const int lane = col * 4 + ((kk & 7) >> 1);
+    return ((((size_t)chunk * KSTEPS + ks) * 32 + lane) << 3) + ((kk >> 3) << 1) + (kk & 1);
+}
+__device__ __forceinline__ void xfrag_store(__nv_bfloat16 *X, int k, int col, float v) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+    const size_t i = xfrag_index(k, col);
+    X[i] = hi;
+    X[i + 4] = lo;
+}
+__host__ __device__ inline size_t xfrag_bytes(int K) { return (size_t)((K + KC - 1) / KC) * X_STAGE; }
+
+// ---------------------------------------------------------------- GEMM phase
+
+// One GEMM as seen by the whole grid: Y[n][col] = sum_k W[n][k] X[k][col].
+//   pair == 1: N rows, tiles of 16 rows (the last may be ragged).
+//   pair == 2: W holds two stacked matrices of `half` rows each (gate over up); a tile is rows
+//              [16 t, 16 t + 16) of both, and the epilogue sees both accumulators.
+// The weights are described by a rank-3 tensor map over the row-major [N][K] matrix, dimensions
+// (64 elements, N rows, K/64 groups) with strides (2 B, 2K B, 128 B) and box (64, 16, 8): one box
+// is a stage.  Rows past N and k groups past K read as zeros.  K must be a multiple of 64.
+struct Gemm {
+    const CUtensorMap *W;
+    const uint4 *X;
+    int N, K, pair, half;
+    __device__ __forceinline__ int tiles() const { return pair == 2 ? half / TILE_N : (N + TILE_N - 1) / TILE_N; }
+};
+
+struct Rings { uint32_t wi, xi; };   // stage counters of one role (slot = i % N, parity = (i / N) & 1)
+
+__device__ __forceinline__ void cta_tile_range(int T, int cta, int G, int &t0, int &t1) {
+    t0 = (int)((long long)T * cta / G);
+    t1 = (int)((long long)T * (cta + 1) / G);
+}
+
+// Weight producer warp: streams this CTA's tiles of the GEMM through the weight ring.
+__device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol) {
+    Smem *sm = S.sm;
+    const int lane = threadIdx.x & 31;
+    int t0, t1;
+    cta_tile_range(g.tiles(), cta, G, t0, t1);
+    const int nch = (g.K + KC - 1) / KC;
+    for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
+        const int ng = min(CONS_WARPS, t1 - g0);
+        for (int kc = 0; kc < nch; ++kc) {
+            for (int s = 0; s < ng; ++s) {
+                for (int p = 0; p < g.pair; ++p) {
+                    const int slot = r.wi % NW;
+                    mbar_wait(S, &sm->w_empty[slot], ((r.wi / NW) & 1) ^ 1);
+                    if (lane == 0 && !aborted(S)) {
+                        mbar_expect_tx(&sm->w_full[slot], (uint32_t)W_STAGE);
+                        tma_load_3d(sm->w[slot], g.W, 0, (g0 + s) * TILE_N + p * g.half, kc * KG, &sm->w_full[slot], pol);
+                    }
+                    ++r.wi;
+                }
+            }
+        }
+    }
+}
+
+// Activation producer warp: one stage per (tile group, k chunk).
+__device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol) {
+    Smem *sm = S.sm;
+    const int lane = threadIdx.x & 31;
+    int t0, t1;
+    cta_tile_range(g.tiles(), cta, G, t0, t1);
+    const int nch = (g.K + KC - 1) / KC;
+    for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
+        for (int kc = 0; kc < nch; ++kc) {
+            const int klen = min(KC, g.K - kc * KC);
+            const int slot = r.xi % NX;
+            mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
+            if (lane == 0 && !aborted(S)) {
+                const uint32_t bytes = (uint32_t)(klen / 16) * 512u;
+                mbar_expect_tx(&sm->x_full[slot], bytes);
+                bulk_g2s(sm->x[slot], reinterpret_cast<const unsigned char *>(g.X) + (size_t)kc * X_STAGE, bytes, &sm->x_full[slot], pol);
+            }
+            ++r.xi;
+        }
+    }
+}
+
+// Consumer warps.  Within a group of up to eight tiles the warps are arranged as TS tile slots x
+// KS k-splits (TS * KS = 8, TS the smallest power of two holding the group); a warp multiplies
+// the k-steps s = ks_id (mod KS) of its slot's stages.  The k-splits of a tile are summed in a
+// fixed order through shared memory, then `epi(tile, acc)` runs in the slot's first warp with
+//   acc[p][i]: fragment element i of matrix p: rows lane/4 (i<2) or lane/4+8, columns 2(lane%4)+(i&1).
+// The arrangement depends only on the tile partition, never on which token columns are in use.
+template <int PAIR, class Epi>
+__device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int cta, int G, Rings &r, Epi &&epi) {
+    Smem *sm = S.sm;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int t0, t1;
+    cta_tile_range(g.tiles(), cta, G, t0, t1);
+    const int nch = (g.K + KC - 1) / KC;
+    // ldmatrix source of this lane inside a stage: row (lane%8) + 8 ((lane/8)%2), 16-byte chunk lane/16 of the k-step
+    const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+    const int a_off = a_row * 128, a_hi = lane >> 4, a_sw = a_row & 7;
+    for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
+        const int ng = min(CONS_WARPS, t1 - g0);
+        int TS = 1;
+        while (TS < ng) TS <<= 1;
+        const int KS = CONS_WARPS / TS;
+        const int slot_id = warp % TS, ks_id = warp / TS;
+        float acc[PAIR][4][4];   // [matrix][even/odd step x hi/lo][fragment]
+#pragma unroll
+        for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[p][q][i] = 0.f;
+        for (int kc = 0; kc < nch; ++kc) {
+            const int ksteps = min(KC, g.K - kc * KC) >> 4;
+            const int xslot = r.xi % NX;
+            mbar_wait(S, &sm->x_full[xslot], (r.xi / NX) & 1);
+            const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + lane;
+            for (int s = 0; s < ng; ++s) {
+#pragma unroll
+                for (int p = 0; p < PAIR; ++p) {
+                    const int wslot = r.wi % NW;
+                    mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
+                    if (s == slot_id) {
+                        const unsigned char *ws = sm->w[wslot] + a_off;
+                        int par = 0;
+#pragma unroll 4
+                        for (int ks = ks_id; ks < ksteps; ks += KS) {
+                            uint32_t a[4];
+                            ldmatrix_x4(a, ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
+                            const uint4 b = xs[ks * 32];
+                            mma16816(acc[p][par], a, b.x, b.y);
+                            mma16816(acc[p][par + 2], a, b.z, b.w);
+                            par ^= 1;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->w_empty[wslot]);
+                    ++r.wi;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm->x_empty[xslot]);
+            ++r.xi;
+        }
+        // fold the four partial accumulators in a fixed order: (even.hi + odd.hi) + (even.lo + odd.lo)
+        float d[PAIR][4];
+#pragma unroll
+        for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) d[p][i] = (acc[p][0][i] + acc[p][1][i]) + (acc[p][2][i] + acc[p][3][i]);
+        if (KS > 1) {
+            float *red = sm->red + (size_t)warp * (PAIR * 128);
+#pragma unroll
+            for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) red[(p * 4 + i) * 32 + lane] = d[p][i];
+            bar_consumers();
+            if (ks_id == 0) {
+                for (int q = 1; q < KS; ++q) {
+                    const float *o = sm->red + (size_t)(q * TS + slot_id) * (PAIR * 128);
+#pragma unroll
+                    for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) d[p][i] += o[(p * 4 + i) * 32 + lane];
+                }
+            }
+        }
+        if (ks_id == 0 && slot_id < ng) epi(g0 + slot_id, d);
+        if (KS > 1) bar_consumers();
+    }
+}
+
+// The dynamic shared memory is requested SMEM_BYTES long; the structure starts at its first
+// 1024-byte boundary.
+constexpr size_t SMEM_BYTES = sizeof(Smem) + 1024;
+__device__ __forceinline__ Smem *smem_base(unsigned char *raw) {
+    const uint32_t a = s32(raw);
+    return reinterpret_cast<Smem *>(raw + ((1024u - (a & 1023u)) & 1023u));
+}
+
+// Shared-memory set-up by the whole block (call once, followed by __syncthreads()).
+__device__ __forceinline__ void smem_init(Smem *sm) {
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NW; ++i) { mbar_init(&sm->w_full[i], 1); mbar_init(&sm->w_empty[i], CONS_WARPS); }
+        for (int i = 0; i < NX; ++i) { mbar_init(&sm->x_full[i], 1); mbar_init(&sm->x_empty[i], CONS_WARPS); }
+        sm->abort = 0;
+        fence_mbar_init();
+        fence_proxy_async();
+    }
+}
+
+// After an error the producers stop issuing copies; give the ones already in flight time to land
+// before the block's shared memory is released.
+__device__ __forceinline__ void settle_on_abort(const Shared &S) {
+    __syncthreads();
+    if (!aborted(S)) return;
+    const unsigned long long t0 = gtime();
+    while (gtime() - t0 < 200000ull) __nanosleep(1000);
+}
+
+}  // namespace st
+}  // namespace ada
