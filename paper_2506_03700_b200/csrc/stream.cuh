@@ -32,13 +32,14 @@ constexpr int TILE_N = 16;                       // weight rows per stage (mma M
 constexpr int KG = KC / 64;                      // 64-element (128-byte) k groups per stage
 constexpr int W_STAGE = TILE_N * KC * 2;         // 16384: [k group][row][128 B, 16-byte chunks xor-swizzled by row%8]
 constexpr int X_STAGE = KSTEPS * 32 * 16;        // 16384: [k-step][lane][b0.hi b1.hi b0.lo b1.lo]
-constexpr int NW = 10;                           // weight stages in flight per CTA
+constexpr int NW = 9;                            // weight stages in flight per CTA
 constexpr int NX = 3;                            // activation stages
 constexpr int CONS_WARPS = 8;
 constexpr int CONS_THREADS = CONS_WARPS * 32;
 constexpr int THREADS = CONS_THREADS + 64;       // + weight producer warp + activation producer warp
 constexpr int MAX_COLS = 8;                      // tokens per pass (mma N)
 constexpr int RED_BYTES = CONS_WARPS * 2 * 128 * 4;  // cross-warp reduction scratch (two tiles per warp)
+constexpr int SCRATCH_BYTES = 33 * 1024;         // consumers' scratch: GEMM reduction, or the attention phase's buffers
 
 constexpr int ERR_TIMEOUT_MBAR = 1, ERR_TIMEOUT_GRID = 2;
 constexpr unsigned long long WAIT_NS = 2000000000ull;   // a single wait gives up after two seconds
@@ -46,7 +47,7 @@ constexpr unsigned long long WAIT_NS = 2000000000ull;   // a single wait gives u
 struct Smem {                                    // must start on a 1024-byte boundary (swizzle pattern)
     alignas(1024) unsigned char w[NW][W_STAGE];
     alignas(128) unsigned char x[NX][X_STAGE];
-    alignas(16) float red[RED_BYTES / 4];
+    alignas(16) unsigned char scratch[SCRATCH_BYTES];
     alignas(16) float vec[64];                    // per-column scalars (rstd, ...)
     alignas(8) unsigned long long w_full[NW], w_empty[NW], x_full[NX], x_empty[NX];
     int abort;
@@ -124,7 +125,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&a)[4], const void *
 }
 // d += a (16x16, row) * b (16x8, col), bf16 inputs, fp32 accumulation.
 __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -141,10 +142,32 @@ __device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
 
 // ---------------------------------------------------------------- bounded waits
 
+// Optional event trace (test hook): records (globaltimer ns, code) pairs while `tr_on` is set.
+struct Trace {
+    unsigned long long *buf;   // [cap][2], or nullptr
+    unsigned *count;
+    unsigned cap;
+};
+
 struct Shared {            // what every role needs to wait safely
     Smem *sm;
     int *err;              // global error word (0 = fine)
+    Trace tr;
+    int tr_on;             // this block is currently tracing
 };
+
+constexpr int EV_PHASE_BEGIN = 1, EV_X0 = 2, EV_W0 = 3, EV_MAIN_END = 4, EV_EPI_END = 5, EV_WP_BEGIN = 6, EV_WP_END = 7,
+              EV_ITEM = 8, EV_COMBINE = 9, EV_ARRIVE = 10;
+
+__device__ __forceinline__ void trace(const Shared &S, int ev, int arg) {
+    if (S.tr_on && S.tr.buf) {
+        const unsigned i = atomicAdd(S.tr.count, 1u);
+        if (i < S.tr.cap) {
+            S.tr.buf[2 * (size_t)i] = gtime();
+            S.tr.buf[2 * (size_t)i + 1] = ((unsigned long long)blockIdx.x << 32) | ((unsigned long long)(arg & 0xffff) << 8) | (unsigned)ev;
+        }
+    }
+}
 
 __device__ __forceinline__ bool aborted(const Shared &S) { return *(volatile int *)&S.sm->abort != 0; }
 
@@ -241,6 +264,7 @@ __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, i
     int t0, t1;
     cta_tile_range(g.tiles(), cta, G, t0, t1);
     const int nch = (g.K + KC - 1) / KC;
+    if (lane == 0) trace(S, EV_WP_BEGIN, 0);
     for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
         const int ng = min(CONS_WARPS, t1 - g0);
         for (int kc = 0; kc < nch; ++kc) {
@@ -257,6 +281,7 @@ __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, i
             }
         }
     }
+    if (lane == 0) trace(S, EV_WP_END, 0);
 }
 
 // Activation producer warp: one stage per (tile group, k chunk).
@@ -277,6 +302,34 @@ __device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, i
                 bulk_g2s(sm->x[slot], reinterpret_cast<const unsigned char *>(g.X) + (size_t)kc * X_STAGE, bytes, &sm->x_full[slot], pol);
             }
             ++r.xi;
+        }
+    }
+}
+
+// The k-steps ks_id + KS_ j (j < 32 / KS_) of one full weight stage: fragment loads run PF steps
+// ahead of the multiply-adds that use them.  Even j accumulate into acc[0] (high parts) and acc[2]
+// (low parts), odd j into acc[1] and acc[3]: four independent accumulation chains.
+template <int KS_>
+__device__ __forceinline__ void stage_full(float (&acc)[4][4], const unsigned char *ws, const uint4 *xs, int ks_id, int a_hi, int a_sw) {
+    constexpr int NJ = KSTEPS / KS_;
+    constexpr int PF = NJ < 4 ? NJ : 4;
+    uint32_t a[PF][4];
+    uint4 b[PF];
+#pragma unroll
+    for (int j = 0; j < PF; ++j) {
+        const int ks = ks_id + KS_ * j;
+        ldmatrix_x4(a[j], ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
+        b[j] = xs[ks * 32];
+    }
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+        const int cur = j % PF;
+        mma16816(acc[j & 1], a[cur], b[cur].x, b[cur].y);
+        mma16816(acc[(j & 1) + 2], a[cur], b[cur].z, b[cur].w);
+        if (j + PF < NJ) {
+            const int ks = ks_id + KS_ * (j + PF);
+            ldmatrix_x4(a[cur], ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
+            b[cur] = xs[ks * 32];
         }
     }
 }
@@ -314,23 +367,33 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
             const int ksteps = min(KC, g.K - kc * KC) >> 4;
             const int xslot = r.xi % NX;
             mbar_wait(S, &sm->x_full[xslot], (r.xi / NX) & 1);
+            if (threadIdx.x == 0 && kc == 0 && g0 == t0) trace(S, EV_X0, 0);
             const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + lane;
             for (int s = 0; s < ng; ++s) {
 #pragma unroll
                 for (int p = 0; p < PAIR; ++p) {
                     const int wslot = r.wi % NW;
                     mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
+                    if (threadIdx.x == 0 && kc == 0 && g0 == t0 && s == 0 && p == 0) trace(S, EV_W0, 0);
                     if (s == slot_id) {
                         const unsigned char *ws = sm->w[wslot] + a_off;
-                        int par = 0;
-#pragma unroll 4
-                        for (int ks = ks_id; ks < ksteps; ks += KS) {
-                            uint32_t a[4];
-                            ldmatrix_x4(a, ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
-                            const uint4 b = xs[ks * 32];
-                            mma16816(acc[p][par], a, b.x, b.y);
-                            mma16816(acc[p][par + 2], a, b.z, b.w);
-                            par ^= 1;
+                        if (ksteps == KSTEPS) {   // full chunk: software-pipelined, fully unrolled per k-split
+                            switch (KS) {
+                                case 1: stage_full<1>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
+                                case 2: stage_full<2>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
+                                case 4: stage_full<4>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
+                                default: stage_full<8>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
+                            }
+                        } else {                  // short last chunk of K
+                            int par = 0;
+                            for (int ks = ks_id; ks < ksteps; ks += KS) {
+                                uint32_t a[4];
+                                ldmatrix_x4(a, ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
+                                const uint4 b = xs[ks * 32];
+                                if (par == 0) { mma16816(acc[p][0], a, b.x, b.y); mma16816(acc[p][2], a, b.z, b.w); }
+                                else { mma16816(acc[p][1], a, b.x, b.y); mma16816(acc[p][3], a, b.z, b.w); }
+                                par ^= 1;
+                            }
                         }
                     }
                     __syncwarp();
@@ -342,6 +405,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
             if (lane == 0) mbar_arrive(&sm->x_empty[xslot]);
             ++r.xi;
         }
+        if (threadIdx.x == 0 && g0 + CONS_WARPS >= t1) trace(S, EV_MAIN_END, 0);
         // fold the four partial accumulators in a fixed order: (even.hi + odd.hi) + (even.lo + odd.lo)
         float d[PAIR][4];
 #pragma unroll
@@ -349,7 +413,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
 #pragma unroll
             for (int i = 0; i < 4; ++i) d[p][i] = (acc[p][0][i] + acc[p][1][i]) + (acc[p][2][i] + acc[p][3][i]);
         if (KS > 1) {
-            float *red = sm->red + (size_t)warp * (PAIR * 128);
+            float *red = reinterpret_cast<float *>(sm->scratch) + (size_t)warp * (PAIR * 128);
 #pragma unroll
             for (int p = 0; p < PAIR; ++p)
 #pragma unroll
@@ -357,7 +421,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
             bar_consumers();
             if (ks_id == 0) {
                 for (int q = 1; q < KS; ++q) {
-                    const float *o = sm->red + (size_t)(q * TS + slot_id) * (PAIR * 128);
+                    const float *o = reinterpret_cast<const float *>(sm->scratch) + (size_t)(q * TS + slot_id) * (PAIR * 128);
 #pragma unroll
                     for (int p = 0; p < PAIR; ++p)
 #pragma unroll
@@ -373,6 +437,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
 // The dynamic shared memory is requested SMEM_BYTES long; the structure starts at its first
 // 1024-byte boundary.
 constexpr size_t SMEM_BYTES = sizeof(Smem) + 1024;
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a block may use");
 __device__ __forceinline__ Smem *smem_base(unsigned char *raw) {
     const uint32_t a = s32(raw);
     return reinterpret_cast<Smem *>(raw + ((1024u - (a & 1023u)) & 1023u));
