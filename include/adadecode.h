@@ -46,6 +46,7 @@ extern "C" {
 
 #define ADA_MAX_BATCH 16
 #define ADA_MAX_LAYERS 256
+#define ADA_PROF_CLASSES 12
 
 typedef struct ada_model ada_model;     /* opaque */
 typedef struct ada_session ada_session; /* opaque: sequences, paged KV metadata, in-flight state */
@@ -158,7 +159,6 @@ int ada_debug_read_kv(ada_session *s, int32_t seq, int32_t which, int32_t layer0
  * 5 O-proj GEMM, 6 gate/up GEMM, 7 SwiGLU, 8 down GEMM, 9 LM-head stream, 10 head transformation T,
  * 11 other.  ada_debug_profile_read returns, accumulated since profiling was switched on, the device
  * milliseconds, launch counts and algorithmic HBM bytes (weights or KV the launch must read) per class. */
-#define ADA_PROF_CLASSES 12
 int ada_debug_profile(ada_session *s, int32_t on);
 int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out, double *bytes_out);
 /* Select the GEMM path: 0 = CUDA-core kernels (any dtype), 1 = tensor-core kernels (bf16 only). */

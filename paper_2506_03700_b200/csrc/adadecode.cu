@@ -638,6 +638,8 @@ int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, i
     c.page_tokens = page_tokens;
     c.page_shift = 0;
     while ((1 << c.page_shift) < page_tokens) c.page_shift++;
+    c.kv_swz = 0;
+    if (g.dtype == ADA_DTYPE_BF16) c.kv_swz = (g.head_dim / 8) % 8 == 0 ? 7 : (g.head_dim / 8) % 4 == 0 ? 3 : (g.head_dim / 8) % 2 == 0 ? 1 : 0;
     c.max_pages = S->max_pages; c.max_seq = max_seq_len; c.slots = S->slots; c.n_chunks = S->n_chunks;
     c.st = (DevState *)(b + lay.st); c.rt = (RowTable *)(b + lay.rt); c.fill = (int32_t *)(b + lay.fill);
     c.tokens = (int32_t *)(b + lay.tokens); c.page_table = (int32_t *)(b + lay.page_table);
@@ -813,7 +815,11 @@ int ada_debug_read_kv(ada_session *S, int32_t seq, int32_t which, int32_t layer0
         for (int i = 0; i < g.head_dim; ++i) {
             float f;
             if (esz == 4) memcpy(&f, tmp.data() + 4 * i, 4);
-            else { uint32_t b = ((uint32_t)tmp[2 * i] | ((uint32_t)tmp[2 * i + 1] << 8)) << 16; memcpy(&f, &b, 4); }
+            else {   // bf16 rows are stored with their 16-byte chunks xor-swizzled by the position
+                const int j = (((i >> 3) ^ (pos & S->c.kv_swz)) << 3) | (i & 7);
+                uint32_t b = ((uint32_t)tmp[2 * j] | ((uint32_t)tmp[2 * j + 1] << 8)) << 16;
+                memcpy(&f, &b, 4);
+            }
             host_out[h * g.head_dim + i] = f;
         }
     }

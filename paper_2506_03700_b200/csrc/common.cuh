@@ -26,6 +26,9 @@ struct RowTable {
 struct DevStats {
     long long steps, head_evals, early_exits, verify_steps, accepted, rejected, discarded, row_layers, truncated;
     long long exits_at_layer[ADA_MAX_LAYERS];
+    long long layer_passes;              // counted on the device by the persistent kernel
+    long long phase_ns[ADA_PROF_CLASSES];    // device time per phase class (persistent kernel, measured in CTA 0)
+    long long phase_count[ADA_PROF_CLASSES];
 };
 
 // Device-resident decoding state of a session.

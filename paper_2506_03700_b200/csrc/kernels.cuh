@@ -21,7 +21,7 @@ constexpr int SEL_LAST = -3;   // the single row rt->n_rows-1 (prefill: last pro
 struct Ctx {
     int d, nq, nkv, hd, dff, vocab, L, qkv_rows, group;
     float eps;
-    int page_tokens, page_shift, max_pages, max_seq, slots, n_chunks;
+    int page_tokens, page_shift, max_pages, max_seq, slots, n_chunks, kv_swz;
     DevState *st;
     RowTable *rt;
     int32_t *fill;        // [batch][L]
@@ -122,10 +122,20 @@ __device__ __forceinline__ int build_row_list(const Ctx &c, int sel, int *rows_s
     return *n_sh;
 }
 
+// Element index of the first element of one cached row (K or V of one position, one kv head).
+// Pool layout: [page][layer][K|V][kv head][position in page][head_dim].
 __device__ __forceinline__ size_t kv_index(const Ctx &c, int seq, int layer, int which, int head, int pos) {
     int page = c.page_table[seq * c.max_pages + (pos >> c.page_shift)];
     int t = pos & (c.page_tokens - 1);
     return ((((size_t)page * c.L + layer) * 2 + which) * c.nkv + head) * ((size_t)c.page_tokens * c.hd) + (size_t)t * c.hd;
+}
+// Inside a bf16 row the 16-byte chunks (8 elements) are stored xor-swizzled by the position:
+// element j sits at chunk (j/8) ^ (pos & swz), swz = 7 when head_dim is a multiple of 64 (else the
+// largest of 3, 1, 0 whose block size divides head_dim/8).  A page of rows copied verbatim into
+// shared memory can then be read with ldmatrix (8 rows x 16 bytes) without bank conflicts.  fp32
+// rows are stored plainly (swz = 0).
+__device__ __forceinline__ int kv_swz(const Ctx &c, int j, int pos) {
+    return (((j >> 3) ^ (pos & c.kv_swz)) << 3) | (j & 7);
 }
 
 // ------------------------------------------------------------------ step set-up
@@ -327,12 +337,12 @@ __global__ void k_rope_kv(Ctx c, int layer) {
         float x0 = kin[h * c.hd + j], x1 = kin[h * c.hd + j + half];
         float co = cs[2 * j], si = cs[2 * j + 1];
         size_t o = kv_index(c, seq, layer, 0, h, pos);
-        pool[o + j] = from_f<T>(x0 * co - x1 * si);
-        pool[o + j + half] = from_f<T>(x1 * co + x0 * si);
+        pool[o + kv_swz(c, j, pos)] = from_f<T>(x0 * co - x1 * si);
+        pool[o + kv_swz(c, j + half, pos)] = from_f<T>(x1 * co + x0 * si);
     }
     for (int i = threadIdx.x; i < c.nkv * c.hd; i += blockDim.x) {
         int h = i / c.hd, j = i - h * c.hd;
-        pool[kv_index(c, seq, layer, 1, h, pos) + j] = from_f<T>(vin[i]);
+        pool[kv_index(c, seq, layer, 1, h, pos) + kv_swz(c, j, pos)] = from_f<T>(vin[i]);
     }
 }
 
@@ -357,11 +367,15 @@ __global__ void __launch_bounds__(32) k_attn_partial(Ctx c, int layer) {
     for (int e = 0; e < EPL; ++e) { qv[e] = c.q[((size_t)r * c.nq + h) * c.hd + lane * EPL + e]; acc[e] = 0.f; }
     float m = -INFINITY, l = 0.f;
     for (int t = t0; t <= t1; ++t) {
-        const T *kp = pool + kv_index(c, seq, layer, 0, kvh, t) + lane * EPL;
-        const T *vp = pool + kv_index(c, seq, layer, 1, kvh, t) + lane * EPL;
+        const T *kp = pool + kv_index(c, seq, layer, 0, kvh, t);
+        const T *vp = pool + kv_index(c, seq, layer, 1, kvh, t);
         float dot = 0.f, vv[EPL];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) { dot = fmaf(qv[e], to_f<T>(kp[e]), dot); vv[e] = to_f<T>(vp[e]); }
+        for (int e = 0; e < EPL; ++e) {
+            const int j = kv_swz(c, lane * EPL + e, t);
+            dot = fmaf(qv[e], to_f<T>(kp[j]), dot);
+            vv[e] = to_f<T>(vp[j]);
+        }
         float sc = warp_sum(dot) * scale;
         float mn = fmaxf(m, sc);
         float corr = expf(m - mn), p = expf(sc - mn);

@@ -1,0 +1,1052 @@
+// The persistent decode kernel: Algorithm 1 of the paper, one cooperative launch for many steps.
+//
+// One CTA per SM, ten warps: a weight producer, an activation / KV producer and eight consumers.
+// Every CTA walks the same program
+//     control | for each layer: QKV | attention | O | gate-up | down | [head, control] ... | final head | control
+// with a grid barrier between phases.  The weight producer is not held by those barriers: it
+// keeps the TMA ring full with the tiles of the coming phases, so HBM keeps streaming while the
+// consumers meet.  All decoding state (sequence, per-layer fill levels, in-flight tokens, row
+// residuals, counters) lives in device memory; the control points run in CTA 0, which publishes
+// each decision (continue the climb, start the next token, stop) to the other CTAs through a
+// sequence-numbered record.  The host launches, waits, and launches again until the call is done.
+//
+// Token columns: the up-to-eight tokens of a pass (the newest token and the early-predicted
+// tokens still in flight, Algorithm 1's P[l] (+) t_i) are the eight columns of the tensor-core
+// tile; column = position - base, fixed for the life of a token.  Per-column buffers therefore
+// persist across steps: a token that left the climb at layer e finds its residual, its
+// normalisation partial sums and its layer-(e+1) GEMM input where its last pass left them.
+// Each column's numbers depend only on that column's own inputs (never on which other columns
+// ride along), which is what makes the adaptive output bit-identical to plain greedy decoding.
+#pragma once
+
+#include "kernels.cuh"
+#include "stream.cuh"
+
+namespace ada {
+namespace mg {
+
+using namespace st;
+
+constexpr int ACT_CONTINUE = 1, ACT_NEWSTEP = 2, ACT_STOP = 3;
+constexpr int CTRL_START = 0, CTRL_HEAD = 1, CTRL_TOP = 2;
+constexpr int ATT_PAGE = 64;          // cache positions per attention sub-block (= KV page size on this path)
+constexpr int ATT_CHUNK = kAttnChunk; // positions per attention work item (fixed: anchored at position 0)
+constexpr int ERR_BAD_STATE = 3;
+
+struct StepDesc {
+    int n_cols;                // columns with a token (in flight + newest)
+    int newest;                // column of the newest token
+    int head_ok;               // the newest token may consult intermediate heads in this step
+    int pmax;                  // position of the newest token
+    int first_layer[MAX_COLS]; // 0-based layer at which the column resumes (INT_MAX: no token)
+    int pos[MAX_COLS];
+};
+
+struct Pub {                   // what CTA 0 publishes at a control point
+    unsigned seq;
+    int action;
+    StepDesc d;
+    int pad[10];
+};
+
+struct MegaLayer {
+    const CUtensorMap *wqkv, *wo, *wgu, *wdown, *wT;
+    const __nv_bfloat16 *attn_norm, *ffn_norm;
+    float head_scale;
+    int has_head;
+};
+
+struct MegaModel {
+    const CUtensorMap *lm_head;
+    const __nv_bfloat16 *tok_embed, *final_norm;
+    float rope_base;
+    int pad;
+    MegaLayer layer[ADA_MAX_LAYERS + 1];   // [l] for 0-based layer l; head fields of 1-based layer e live in layer[e]
+};
+
+struct MegaArgs {
+    Ctx c;
+    const MegaModel *mm;
+    const int *exit_at;        // [L + 1]: 1 if this call consults the head after 1-based layer e
+    __nv_bfloat16 *XA, *XB, *XO, *XH, *XF, *XT;   // GEMM inputs in fragment layout (see stream.cuh)
+    float *ssq_a, *ssq_b;      // [d/16][8] partial sums of squares of the residual (per 16-feature tile, per column)
+    float *qkvraw;             // [8][qkv_rows]
+    float *attn_part;          // [8 * nq][n_chunks][hd + 4]
+    float *head_part;          // [grid][8][4]
+    unsigned *attn_cnt;        // [nkv]
+    unsigned *grid_ctr;
+    Pub *pub;                  // [2]
+    int *err;
+    int step_budget;           // steps this launch may start
+    int store_logits;
+    Trace trace;               // test hook: event trace of the steps [trace_step0, trace_step1) of this launch
+    int trace_step0, trace_step1;
+};
+
+// ---------------------------------------------------------------- small helpers
+
+__device__ __forceinline__ float ldcg(const float *p) { return __ldcg(p); }
+
+__device__ __forceinline__ unsigned active_mask(const StepDesc &d, int layer) {
+    unsigned m = 0;
+#pragma unroll
+    for (int c = 0; c < MAX_COLS; ++c) m |= (d.first_layer[c] <= layer ? 1u : 0u) << c;
+    return m;
+}
+
+// rstd[c] = 1 / sqrt(sum_tiles ssq[tile][c] / d + eps), one warp per column, fixed summation order.
+__device__ __forceinline__ void compute_rstd(Smem *sm, const float *ssq, int ntiles, int d, float eps) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float s = 0.f;
+    for (int t = lane; t < ntiles; t += 32) s += ldcg(ssq + (size_t)t * MAX_COLS + warp);
+    s = warp_sum(s);
+    if (lane == 0) sm->vec[warp] = 1.0f / sqrtf(s / (float)d + eps);
+    bar_consumers();
+}
+
+// Grid barrier as seen by the consumers of a CTA.
+__device__ __forceinline__ void barrier_consumers(const Shared &S, unsigned *ctr, unsigned &bar_no, int G, int cls) {
+    if (threadIdx.x == 0) trace(S, EV_EPI_END, cls);
+    bar_consumers();
+    ++bar_no;
+    if (threadIdx.x == 0) {
+        grid_arrive(ctr);
+        trace(S, EV_ARRIVE, cls);
+        grid_wait(S, ctr, bar_no * (unsigned)G);
+        trace(S, EV_PHASE_BEGIN, cls);
+    }
+    bar_consumers();
+}
+
+// Merge the per-CTA (max, sum exp, argmax) partials of one column, by one whole warp: lane i folds
+// CTAs i, i+32, ... in ascending order, then the lanes are folded by a butterfly (the merge is
+// symmetric, so every lane ends with the same value).
+__device__ __forceinline__ HeadResult merge_head(const float *head_part, int G, int col) {
+    const int lane = threadIdx.x & 31;
+    Msa a; a.m = -INFINITY; a.s = 0.f; a.i = INT_MAX;
+    for (int b = lane; b < G; b += 32) {
+        const float *o = head_part + ((size_t)b * MAX_COLS + col) * 4;
+        Msa x; x.m = ldcg(o); x.s = ldcg(o + 1); x.i = __float_as_int(ldcg(o + 2));
+        a = msa_merge(a, x);
+    }
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        Msa o;
+        o.m = __shfl_xor_sync(0xffffffffu, a.m, off);
+        o.s = __shfl_xor_sync(0xffffffffu, a.s, off);
+        o.i = __shfl_xor_sync(0xffffffffu, a.i, off);
+        a = msa_merge(a, o);
+    }
+    HeadResult hr; hr.token = a.i; hr.zmax = a.m; hr.sumexp = a.s; hr.p = 1.0f / a.s;
+    return hr;
+}
+
+// ---------------------------------------------------------------- control point (CTA 0, consumer warps)
+
+// Applies the outcome of the step that just ended (Eq. 1 after a head; verification and rollback,
+// Eq. 2 at temperature zero, after the final head), then sets up the next step: its columns, the
+// embedding of its newest token, that token's rotary table; finally publishes the action.
+__device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind, int e, unsigned pub_no, const StepDesc &dprev,
+                                          int &steps_started) {
+    const Ctx &c = A.c;
+    DevState *st = c.st;
+    const MegaModel &M = *A.mm;
+    const int tid = threadIdx.x, G = gridDim.x;
+    Pub *pub = A.pub + (pub_no & 1);
+    // (a) head results of the columns that matter: warp w merges column w
+    if (kind != CTRL_START) {
+        const int w = tid >> 5;
+        const bool want = kind == CTRL_HEAD ? w == dprev.newest : w < dprev.n_cols;
+        if (want) {
+            const HeadResult hr = merge_head(A.head_part, G, w);
+            if ((tid & 31) == 0) c.head_res[w] = hr;
+        }
+    }
+    __threadfence_block();
+    bar_consumers();
+    // (b) bookkeeping, one thread
+    if (tid == 0) {
+        int action = ACT_NEWSTEP, verified = 0;
+        int32_t *tok = c.tokens;
+        if (*(volatile int *)A.err != 0) action = ACT_STOP;
+        if (action != ACT_STOP && kind == CTRL_HEAD) {
+            const int len = st->len[0];
+            const HeadResult hr = c.head_res[dprev.newest];
+            bool decide = hr.p > st->gamma;
+            if (st->tape_i < st->tape_n) {
+                const uint8_t t = st->tape[st->tape_i++];
+                if (t == 0) decide = false;
+                if (t == 1) decide = true;
+            }
+            st->st.head_evals++;
+            if (c.head_log && st->head_log_n < kHeadLogCap) {
+                float *hl = c.head_log + 4 * (size_t)st->head_log_n;
+                hl[0] = (float)st->st.steps; hl[1] = (float)e; hl[2] = (float)hr.token; hl[3] = hr.p;
+                st->head_log_n++;
+            }
+            if (!decide) action = ACT_CONTINUE;
+            else {
+                for (int l = 0; l < e; ++l) {
+                    st->st.row_layers += len - c.fill[l];
+                    c.fill[l] = len;
+                }
+                tok[len] = min(max(hr.token, 0), c.vocab - 1);
+                st->len[0] = len + 1;
+                st->st.early_exits++;
+                st->st.exits_at_layer[e]++;
+                st->st.steps++;
+                st->st.layer_passes += e;
+            }
+        }
+        if (action != ACT_STOP && kind == CTRL_TOP) {
+            const int len = st->len[0], base = st->base[0], nrow = len - base;
+            for (int l = 0; l < c.L; ++l) st->st.row_layers += len - c.fill[l];
+            int bad = -1;
+            for (int j = 0; j + 1 < nrow; ++j)
+                if (c.head_res[j].token != tok[base + j + 1]) { bad = j; break; }
+            int new_base, keep;
+            if (bad < 0) {
+                st->st.accepted += nrow - 1;
+                tok[len] = min(max(c.head_res[nrow - 1].token, 0), c.vocab - 1);
+                new_base = len;
+                keep = nrow;
+            } else {
+                st->st.accepted += bad;
+                st->st.rejected += 1;
+                st->st.discarded += nrow - 2 - bad;
+                new_base = base + bad + 1;
+                tok[new_base] = min(max(c.head_res[bad].token, 0), c.vocab - 1);
+                keep = bad + 1;
+            }
+            int new_len = new_base + 1;
+            if (new_len > st->target_len[0]) {
+                st->st.truncated += new_len - st->target_len[0];
+                new_len = st->target_len[0];
+                new_base = new_len - 1;
+            }
+            for (int l = 0; l < c.L; ++l) c.fill[l] = new_base;
+            st->len[0] = new_len;
+            st->base[0] = new_base;
+            st->st.verify_steps++;
+            st->st.steps++;
+            st->st.layer_passes += c.L;
+            if (new_len >= st->target_len[0]) st->done[0] = 1;
+            st->keep_rows = keep;
+            verified = 1;
+        }
+        if (action == ACT_NEWSTEP) {
+            if (st->done[0]) { action = ACT_STOP; st->n_done = 1; }
+            else if (steps_started >= A.step_budget) action = ACT_STOP;
+        }
+        if (action == ACT_NEWSTEP) {
+            ++steps_started;
+            const int len = st->len[0], base = st->base[0];
+            StepDesc nd;
+            nd.n_cols = len - base;
+            nd.newest = len - 1 - base;
+            nd.pmax = len - 1;
+            nd.head_ok = (len - 1 - base) < st->max_early && len < st->target_len[0];
+            if (nd.n_cols < 1 || nd.n_cols > c.slots || nd.n_cols > MAX_COLS || len > c.max_seq || base < 0) {
+                atomicCAS(A.err, 0, ERR_BAD_STATE);
+                action = ACT_STOP;
+            }
+            for (int j = 0; j < MAX_COLS; ++j) {
+                int fl = INT_MAX;
+                const int pos = base + j;
+                if (j < nd.n_cols) {
+                    fl = 0;
+                    for (int l = 0; l < c.L; ++l) fl += c.fill[l] > pos;
+                }
+                nd.first_layer[j] = fl;
+                nd.pos[j] = pos;
+            }
+            pub->d = nd;
+        }
+        pub->action = action;
+        sm->bcast[0] = action;
+        sm->bcast[3] = verified;
+    }
+    bar_consumers();
+    const int action = sm->bcast[0];
+    // (c) logits of the verified rows (test hook), then the embedding of the next newest token
+    if (kind == CTRL_TOP && c.capture && sm->bcast[3]) {
+        const int keep = st->keep_rows, at = st->capture_n;
+        for (int j = 0; j < keep && at + j < st->capture_cap; ++j) {
+            const float *src = c.logit_stage + (size_t)j * c.vocab;
+            float *dst = c.capture + (size_t)(at + j) * c.vocab;
+            for (int i = tid; i < c.vocab; i += CONS_THREADS) dst[i] = __ldcg(src + i);
+        }
+        bar_consumers();
+        if (tid == 0) st->capture_n = min(st->capture_cap, at + keep);
+    }
+    if (action == ACT_NEWSTEP) {
+        const StepDesc &nd = pub->d;
+        const int col = nd.newest, pos = nd.pmax;
+        const int tokid = min(max(c.tokens[pos], 0), c.vocab - 1);
+        const __nv_bfloat16 *erow = M.tok_embed + (size_t)tokid * c.d;
+        const __nv_bfloat16 *g0 = M.layer[0].attn_norm;
+        for (int n0 = 0; n0 < c.d; n0 += CONS_THREADS) {
+            const int n = n0 + tid;
+            float v = 0.f;
+            if (n < c.d) {
+                v = __bfloat162float(erow[n]);
+                c.resid[(size_t)col * c.d + n] = v;
+                xfrag_store(A.XA, n, col, v * __bfloat162float(g0[n]));
+            }
+            float q = v * v;
+            q += __shfl_xor_sync(0xffffffffu, q, 1);
+            q += __shfl_xor_sync(0xffffffffu, q, 2);
+            q += __shfl_xor_sync(0xffffffffu, q, 4);
+            q += __shfl_xor_sync(0xffffffffu, q, 8);
+            if ((tid & 15) == 0 && n < c.d) A.ssq_a[(size_t)(n >> 4) * MAX_COLS + col] = q;
+        }
+        const int half = c.hd / 2;
+        for (int i = tid; i < half; i += CONS_THREADS) {
+            const double freq = pow((double)M.rope_base, -2.0 * i / c.hd);
+            double sn, cs;
+            sincos((double)pos * freq, &sn, &cs);
+            c.rope_cs[((size_t)col * half + i) * 2 + 0] = (float)cs;
+            c.rope_cs[((size_t)col * half + i) * 2 + 1] = (float)sn;
+        }
+    }
+    __threadfence();
+    fence_proxy_async();
+    bar_consumers();
+    if (tid == 0) {
+        __threadfence();
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&pub->seq), "r"(pub_no) : "memory");
+    }
+}
+
+// Every role of every CTA passes here; returns the action and (for a new step) the descriptor.
+template <int ROLE>
+__device__ __forceinline__ int control_point(const MegaArgs &A, const Shared &S, int kind, int e, unsigned &pub_no, StepDesc &d,
+                                             int &steps_started) {
+    Smem *sm = S.sm;
+    ++pub_no;
+    const Pub *pub = A.pub + (pub_no & 1);
+    int action;
+    if (ROLE == 2) {
+        if (blockIdx.x == 0) control_cta0(A, sm, kind, e, pub_no, d, steps_started);
+        if (threadIdx.x == 0) {
+            grid_wait(S, &pub->seq, pub_no);
+            sm->bcast[1] = aborted(S) ? ACT_STOP : *(volatile const int *)&pub->action;
+        }
+        bar_consumers();
+        action = sm->bcast[1];
+    } else {
+        grid_wait(S, &pub->seq, pub_no);
+        action = aborted(S) ? ACT_STOP : *(volatile const int *)&pub->action;
+    }
+    if (action == ACT_NEWSTEP) {
+        const volatile int *src = reinterpret_cast<const volatile int *>(&pub->d);
+        int *dst = reinterpret_cast<int *>(&d);
+#pragma unroll
+        for (int i = 0; i < (int)(sizeof(StepDesc) / 4); ++i) dst[i] = src[i];
+        if (d.n_cols < 1 || d.n_cols > MAX_COLS || d.newest < 0 || d.newest >= MAX_COLS || d.pmax < 0 || d.pmax >= A.c.max_seq)
+            action = ACT_STOP;   // cannot happen unless memory was corrupted; never index with it
+    }
+    return action;
+}
+
+// ---------------------------------------------------------------- attention phase
+
+// Shared memory of the attention phase, carved from the consumers' scratch.  The query fragments
+// are dead once the last score tile of an item is computed; the merge buffers reuse their space.
+template <int HD> struct AttnSmem {
+    union {
+        uint32_t qfrag[2][HD / 16][32][8];   // A fragments of the rotated, scaled queries: hi a0..a3, lo a0..a3
+        float o[2][2][16][HD];               // merge buffers [query tile][source]
+    };
+    float ml[2][2][2][16];                   // [query tile][source][max | sum][row]
+};
+static_assert(sizeof(AttnSmem<128>) <= SCRATCH_BYTES, "attention buffers exceed the consumers' scratch");
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// K/V producer: for every work item of this CTA, the K and V page blocks of its sub-blocks.
+__device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, Rings &r, uint64_t pol) {
+    const Ctx &c = A.c;
+    Smem *sm = S.sm;
+    const int lane = threadIdx.x & 31, cta = blockIdx.x, G = gridDim.x;
+    const int nchunk = d.pmax / ATT_CHUNK + 1, n_items = c.nkv * nchunk;
+    const uint32_t bytes = (uint32_t)(ATT_PAGE * c.hd * 2);
+    const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
+    for (int item = cta; item < n_items; item += G) {
+        const int kvh = item / nchunk, j = item - kvh * nchunk;
+        const int p_base = j * ATT_CHUNK;
+        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.pmax - p_base) / ATT_PAGE + 1);
+        for (int sb = 0; sb < nsb; ++sb) {
+            const int page = c.page_table[(p_base + sb * ATT_PAGE) >> c.page_shift];
+            for (int which = 0; which < 2; ++which) {
+                const int slot = r.xi % NX;
+                mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
+                if (lane == 0 && !aborted(S)) {
+                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + which) * c.nkv + kvh) * ((size_t)ATT_PAGE * c.hd);
+                    mbar_expect_tx(&sm->x_full[slot], bytes);
+                    bulk_g2s(sm->x[slot], pool + blk, bytes, &sm->x_full[slot], pol);
+                }
+                ++r.xi;
+            }
+        }
+    }
+}
+
+// Merge (max, sum, unnormalised output) of another warp, read from shared memory, into this warp's.
+template <int NT, int HD>
+__device__ __forceinline__ void attn_merge_from(float (&o)[NT][4], float (&m_run)[2], float (&l_run)[2], const float (*so)[HD],
+                                                const float (*sml)[16], int lane) {
+#pragma unroll
+    for (int rh = 0; rh < 2; ++rh) {
+        const int row = (lane >> 2) + 8 * rh;
+        const float ms = sml[0][row], ls = sml[1][row];
+        const float mn = fmaxf(m_run[rh], ms);
+        float a = 1.f, b = 0.f;
+        if (mn != -INFINITY) { a = __expf(m_run[rh] - mn); b = __expf(ms - mn); }
+        m_run[rh] = mn;
+        l_run[rh] = l_run[rh] * a + ls * b;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i2 = 0; i2 < 2; ++i2) o[nt][2 * rh + i2] = o[nt][2 * rh + i2] * a + so[row][nt * 8 + 2 * (lane & 3) + i2] * b;
+    }
+}
+template <int NT, int HD>
+__device__ __forceinline__ void attn_merge_to(const float (&o)[NT][4], const float (&m_run)[2], const float (&l_run)[2], float (*so)[HD],
+                                              float (*sml)[16], int lane) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) so[(lane >> 2) + 8 * (i >> 1)][nt * 8 + 2 * (lane & 3) + (i & 1)] = o[nt][i];
+    if ((lane & 3) == 0) {
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+            sml[0][(lane >> 2) + 8 * rh] = m_run[rh];
+            sml[1][(lane >> 2) + 8 * rh] = l_run[rh];
+        }
+    }
+}
+
+// Consumers: causal attention of every active column over the cache plus the in-flight rows.
+// Work item = (kv head, 256-position chunk).  Within a 64-position sub-block warp (mt, qr) handles
+// query tile mt (16 of the up to 32 (column, q head) pairs of the kv head) and positions
+// [16 qr, 16 qr + 16).  K and V rows of the columns processed in this pass are not in the cache
+// yet: they are rotated / rounded here from the QKV output, patched into the shared-memory copy
+// and written to the cache by the item that owns their position.
+template <int HD>
+__device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, unsigned mask, Rings &r) {
+    const Ctx &c = A.c;
+    Smem *sm = S.sm;
+    AttnSmem<HD> *as = reinterpret_cast<AttnSmem<HD> *>(sm->scratch);
+    constexpr int KSQ = HD / 16, NT = HD / 8, HALF = HD / 2;
+    constexpr int ATT_STRIDE = HD + 4;                     // floats per chunk partial: output, max, sum, padding (16-byte rows)
+    constexpr int QPT = 32 * HALF / CONS_THREADS;          // (query, rotation pair) items per thread
+    constexpr int KPT = MAX_COLS * HALF / CONS_THREADS;    // new-row K rotation pairs per thread
+    constexpr int VPT = MAX_COLS * HD / CONS_THREADS;      // new-row V elements per thread
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x, G = gridDim.x;
+    const int group = c.group, qd = c.nq * HD;
+    const int nchunk = d.pmax / ATT_CHUNK + 1, n_items = c.nkv * nchunk;
+    const int mt = warp >> 2, qr = warp & 3;
+    const float scale = rsqrtf((float)HD);
+    __nv_bfloat16 *pool = reinterpret_cast<__nv_bfloat16 *>(c.kv_pool);
+    for (int item = cta; item < n_items; item += G) {
+        const int kvh = item / nchunk, j = item - kvh * nchunk;
+        const int p_base = j * ATT_CHUNK;
+        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.pmax - p_base) / ATT_PAGE + 1);
+        // columns of this pass whose (new) K/V row lies in this chunk
+        unsigned item_new = 0;
+#pragma unroll
+        for (int cc = 0; cc < MAX_COLS; ++cc)
+            if (((mask >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK) item_new |= 1u << cc;
+        // ---- all global reads of the item are issued up front: queries, and the new rows' k / v
+        float qx0[QPT], qx1[QPT], qco[QPT], qsi[QPT];
+#pragma unroll
+        for (int u = 0; u < QPT; ++u) {
+            const int idx = tid + u * CONS_THREADS;
+            const int qcol = idx / HALF, jj = idx - qcol * HALF;
+            const int cc = qcol / group, g = qcol - cc * group;
+            qx0[u] = 0.f; qx1[u] = 0.f; qco[u] = 1.f; qsi[u] = 0.f;
+            if (cc < MAX_COLS && ((mask >> cc) & 1u)) {
+                const float *q = A.qkvraw + (size_t)cc * c.qkv_rows + (size_t)(kvh * group + g) * HD;
+                const float *cs = c.rope_cs + (size_t)cc * HALF * 2;
+                qx0[u] = __ldcg(q + jj); qx1[u] = __ldcg(q + jj + HALF); qco[u] = __ldcg(cs + 2 * jj); qsi[u] = __ldcg(cs + 2 * jj + 1);
+            }
+        }
+        __nv_bfloat16 nk0[KPT], nk1[KPT], nv[VPT];
+        if (item_new) {
+            float kx0[KPT], kx1[KPT], kco[KPT], ksi[KPT], vx[VPT];
+#pragma unroll
+            for (int u = 0; u < KPT; ++u) {
+                const int idx = tid + u * CONS_THREADS, cc = idx / HALF, jj = idx - cc * HALF;
+                kx0[u] = 0.f; kx1[u] = 0.f; kco[u] = 1.f; ksi[u] = 0.f;
+                if ((item_new >> cc) & 1u) {
+                    const float *k = A.qkvraw + (size_t)cc * c.qkv_rows + qd + (size_t)kvh * HD;
+                    const float *cs = c.rope_cs + (size_t)cc * HALF * 2;
+                    kx0[u] = __ldcg(k + jj); kx1[u] = __ldcg(k + jj + HALF); kco[u] = __ldcg(cs + 2 * jj); ksi[u] = __ldcg(cs + 2 * jj + 1);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < VPT; ++u) {
+                const int idx = tid + u * CONS_THREADS, cc = idx / HD, jj = idx - cc * HD;
+                vx[u] = ((item_new >> cc) & 1u) ? __ldcg(A.qkvraw + (size_t)cc * c.qkv_rows + qd + (size_t)(c.nkv + kvh) * HD + jj) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < KPT; ++u) {
+                nk0[u] = __float2bfloat16_rn(kx0[u] * kco[u] - kx1[u] * ksi[u]);
+                nk1[u] = __float2bfloat16_rn(kx1[u] * kco[u] + kx0[u] * ksi[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < VPT; ++u) nv[u] = __float2bfloat16_rn(vx[u]);
+        }
+        bar_consumers();   // the previous item is done with the shared buffers
+        // ---- rotated, scaled queries -> A fragments (hi / lo)
+#pragma unroll
+        for (int u = 0; u < QPT; ++u) {
+            const int idx = tid + u * CONS_THREADS;
+            const int qcol = idx / HALF, jj = idx - qcol * HALF;
+            const float y0 = (qx0[u] * qco[u] - qx1[u] * qsi[u]) * scale, y1 = (qx1[u] * qco[u] + qx0[u] * qsi[u]) * scale;
+            const int row = qcol & 15, m = qcol >> 4;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int dim = jj + h * HALF;
+                const float y = h ? y1 : y0;
+                const int ks = dim >> 4, kk = dim & 15;
+                const int ln = (row & 7) * 4 + ((kk & 7) >> 1), reg = (row >> 3) + 2 * (kk >> 3);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(y);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(y - __bfloat162float(hi));
+                __nv_bfloat16 *f = reinterpret_cast<__nv_bfloat16 *>(&as->qfrag[m][ks][ln][0]);
+                f[reg * 2 + (kk & 1)] = hi;
+                f[8 + reg * 2 + (kk & 1)] = lo;
+            }
+        }
+        bar_consumers();
+        // ---- per-warp online softmax state: rows (lane/4) and (lane/4)+8 of query tile mt
+        int lim[2];
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+            const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = qcol / group;
+            lim[rh] = (cc < MAX_COLS && ((mask >> cc) & 1u)) ? d.pos[cc] : -1;
+        }
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float o[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[nt][i] = 0.f;
+        for (int sb = 0; sb < nsb; ++sb) {
+            const int p0 = p_base + sb * ATT_PAGE;
+            unsigned newm = 0;   // new rows inside this sub-block (uniform over the block)
+#pragma unroll
+            for (int cc = 0; cc < MAX_COLS; ++cc)
+                if (((item_new >> cc) & 1u) && d.pos[cc] >= p0 && d.pos[cc] < p0 + ATT_PAGE) newm |= 1u << cc;
+            const int page = c.page_table[p0 >> c.page_shift];
+            float s[2][4];
+            {   // ---- K block
+                const int slot = r.xi % NX;
+                mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                unsigned char *kb = sm->x[slot];
+                if (newm) {
+                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + 0) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
+#pragma unroll
+                    for (int u = 0; u < KPT; ++u) {
+                        const int idx = tid + u * CONS_THREADS, cc = idx / HALF, jj = idx - cc * HALF;
+                        if ((newm >> cc) & 1u) {
+                            const int pos = d.pos[cc], t = pos - p0;
+                            const int e0 = t * HD + ((((jj >> 3) ^ (pos & 7)) << 3) | (jj & 7));
+                            const int e1 = t * HD + (((((jj + HALF) >> 3) ^ (pos & 7)) << 3) | (jj & 7));
+                            reinterpret_cast<__nv_bfloat16 *>(kb)[e0] = nk0[u];
+                            reinterpret_cast<__nv_bfloat16 *>(kb)[e1] = nk1[u];
+                            pool[blk + e0] = nk0[u];
+                            pool[blk + e1] = nk1[u];
+                        }
+                    }
+                    bar_consumers();
+                }
+                float sh[2][4], sl[2][4];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { sh[nt][i] = 0.f; sl[nt][i] = 0.f; }
+                const int id = lane >> 3;
+                const int pl = 16 * qr + (lane & 7) + 8 * (id >> 1);
+                const unsigned char *krow = kb + pl * (HD * 2);
+                uint4 qh[KSQ], ql[KSQ];
+                uint32_t kf[KSQ][4];
+#pragma unroll
+                for (int ks = 0; ks < KSQ; ++ks) {
+                    qh[ks] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][0]);
+                    ql[ks] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][4]);
+                    ldmatrix_x4(kf[ks], krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
+                }
+#pragma unroll
+                for (int ks = 0; ks < KSQ; ++ks) {
+                    const uint32_t ah[4] = {qh[ks].x, qh[ks].y, qh[ks].z, qh[ks].w}, al[4] = {ql[ks].x, ql[ks].y, ql[ks].z, ql[ks].w};
+                    mma16816(sh[0], ah, kf[ks][0], kf[ks][1]);
+                    mma16816(sh[1], ah, kf[ks][2], kf[ks][3]);
+                    mma16816(sl[0], al, kf[ks][0], kf[ks][1]);
+                    mma16816(sl[1], al, kf[ks][2], kf[ks][3]);
+                }
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int pos = p0 + 16 * qr + 8 * nt + 2 * (lane & 3) + (i & 1);
+                        s[nt][i] = pos <= lim[i >> 1] ? sh[nt][i] + sl[nt][i] : -INFINITY;
+                    }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->x_empty[slot]);
+                ++r.xi;
+            }
+            // ---- online softmax over this warp's 16 positions
+            uint32_t ph[4], plo[4];
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                float mx = fmaxf(fmaxf(s[0][2 * rh], s[0][2 * rh + 1]), fmaxf(s[1][2 * rh], s[1][2 * rh + 1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float mn = fmaxf(m_run[rh], mx);
+                float corr = 1.f, p[4] = {0.f, 0.f, 0.f, 0.f};
+                if (mn != -INFINITY) {
+                    corr = __expf(m_run[rh] - mn);
+                    p[0] = __expf(s[0][2 * rh] - mn); p[1] = __expf(s[0][2 * rh + 1] - mn);
+                    p[2] = __expf(s[1][2 * rh] - mn); p[3] = __expf(s[1][2 * rh + 1] - mn);
+                }
+                m_run[rh] = mn;
+                l_run[rh] = l_run[rh] * corr + ((p[0] + p[1]) + (p[2] + p[3]));
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) { o[nt][2 * rh] *= corr; o[nt][2 * rh + 1] *= corr; }
+                // A fragment of P: a0/a1 = n-tile 0 (rows r / r+8), a2/a3 = n-tile 1
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
+                ph[rh] = *reinterpret_cast<const uint32_t *>(&h0);
+                ph[2 + rh] = *reinterpret_cast<const uint32_t *>(&h1);
+                plo[rh] = pack_bf16(p[0] - __low2float(h0), p[1] - __high2float(h0));
+                plo[2 + rh] = pack_bf16(p[2] - __low2float(h1), p[3] - __high2float(h1));
+            }
+            {   // ---- V block
+                const int slot = r.xi % NX;
+                mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                unsigned char *vb = sm->x[slot];
+                if (newm) {
+                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + 1) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
+#pragma unroll
+                    for (int u = 0; u < VPT; ++u) {
+                        const int idx = tid + u * CONS_THREADS, cc = idx / HD, jj = idx - cc * HD;
+                        if ((newm >> cc) & 1u) {
+                            const int pos = d.pos[cc], t = pos - p0;
+                            const int e0 = t * HD + ((((jj >> 3) ^ (pos & 7)) << 3) | (jj & 7));
+                            reinterpret_cast<__nv_bfloat16 *>(vb)[e0] = nv[u];
+                            pool[blk + e0] = nv[u];
+                        }
+                    }
+                    bar_consumers();
+                }
+                const int id = lane >> 3;
+                const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
+                const unsigned char *vrow = vb + pl * (HD * 2);
+                uint32_t vf[NT / 2][4];
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) ldmatrix_x4_trans(vf[np], vrow + ((((2 * np) | (id >> 1)) ^ (pl & 7)) << 4));
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) {
+                    mma16816(o[2 * np], ph, vf[np][0], vf[np][1]);
+                    mma16816(o[2 * np + 1], ph, vf[np][2], vf[np][3]);
+                    mma16816(o[2 * np], plo, vf[np][0], vf[np][1]);
+                    mma16816(o[2 * np + 1], plo, vf[np][2], vf[np][3]);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->x_empty[slot]);
+                ++r.xi;
+            }
+        }
+        // ---- row sums over the quad, then merge the four position quarters of each query tile:
+        //      (q0 + q1) and (q2 + q3), then the two halves
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+            l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 1);
+            l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 2);
+        }
+        bar_consumers();   // every warp is done with the query fragments, whose space the merge reuses
+        if (qr & 1) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        bar_consumers();
+        if (!(qr & 1)) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        bar_consumers();
+        if (qr == 2) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+        bar_consumers();
+        if (qr == 0) {
+            attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+            // ---- chunk partial (unnormalised output, max, sum) of every valid (column, q head)
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const int qcol = mt * 16 + (lane >> 2) + 8 * rh, cc = qcol / group, g = qcol - cc * group;
+                if (cc < MAX_COLS && ((mask >> cc) & 1u) && d.pos[cc] >= p_base) {
+                    float *out = A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + j) * ATT_STRIDE;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        *reinterpret_cast<float2 *>(out + nt * 8 + 2 * (lane & 3)) = make_float2(o[nt][2 * rh], o[nt][2 * rh + 1]);
+                    if ((lane & 3) == 0) *reinterpret_cast<float2 *>(out + HD) = make_float2(m_run[rh], l_run[rh]);
+                }
+            }
+        }
+        // ---- the CTA that finishes a kv head's last item merges the chunks of that head
+        if (tid == 0) trace(S, EV_ITEM, item);
+        __threadfence();
+        bar_consumers();
+        if (tid == 0) sm->bcast[2] = (int)atomicAdd(A.attn_cnt + kvh, 1u);
+        bar_consumers();
+        if (sm->bcast[2] == nchunk - 1) {
+            __threadfence();
+            // (1) every (max, sum) pair of the head's chunks -> shared memory, all loads in flight at once
+            float *sm_m = &as->o[0][0][0][0];                       // [32][nchunk]
+            float *sm_e = sm_m + 32 * nchunk;                        // [32][nchunk]: sum, then exp(max_k - max)
+            float *sm_den = &as->ml[0][0][0][0];                     // [32]
+            const int nqc = MAX_COLS * group;
+            for (int idx = tid; idx < nqc * nchunk; idx += CONS_THREADS) {
+                const int qcol = idx / nchunk, k = idx - qcol * nchunk, cc = qcol / group, g = qcol - cc * group;
+                float2 v = make_float2(-INFINITY, 0.f);
+                if (((mask >> cc) & 1u) && k <= d.pos[cc] / ATT_CHUNK)
+                    v = __ldcg(reinterpret_cast<const float2 *>(A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + k) * ATT_STRIDE + HD));
+                sm_m[idx] = v.x;
+                sm_e[idx] = v.y;
+            }
+            bar_consumers();
+            // (2) per (column, q head): weights exp(m_k - max) and the denominator, chunks in ascending order
+            if (tid < nqc) {
+                float Mx = -INFINITY;
+                for (int k = 0; k < nchunk; ++k) Mx = fmaxf(Mx, sm_m[tid * nchunk + k]);
+                float den = 0.f;
+                for (int k = 0; k < nchunk; ++k) {
+                    const float mk = sm_m[tid * nchunk + k];
+                    const float w = mk == -INFINITY ? 0.f : __expf(mk - Mx);
+                    den += sm_e[tid * nchunk + k] * w;
+                    sm_e[tid * nchunk + k] = w;
+                }
+                sm_den[tid] = den;
+            }
+            bar_consumers();
+            // (3) outputs, four features per thread and pass, eight chunk loads in flight
+            for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
+                const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = qcol / group, g = qcol - cc * group;
+                if (!((mask >> cc) & 1u)) continue;
+                const int h = kvh * group + g;
+                const int nch = d.pos[cc] / ATT_CHUNK + 1;
+                const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE + dim;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k0 = 0; k0 < nch; k0 += 8) {
+                    float4 ov[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        ov[u] = k0 + u < nch ? __ldcg(reinterpret_cast<const float4 *>(part + (size_t)(k0 + u) * ATT_STRIDE)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (k0 + u < nch) {
+                            const float w = sm_e[qcol * nchunk + k0 + u];
+                            acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
+                        }
+                    }
+                }
+                const float den = sm_den[qcol];
+                xfrag_store(A.XO, h * HD + dim, cc, acc.x / den);
+                xfrag_store(A.XO, h * HD + dim + 1, cc, acc.y / den);
+                xfrag_store(A.XO, h * HD + dim + 2, cc, acc.z / den);
+                xfrag_store(A.XO, h * HD + dim + 3, cc, acc.w / den);
+            }
+            if (tid == 0) { A.attn_cnt[kvh] = 0u; trace(S, EV_COMBINE, kvh); }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- the walker
+
+template <int ROLE, int PAIR, class Epi>
+__device__ __forceinline__ void gemm_phase(const Shared &S, const Gemm &g, Rings &r, uint64_t pol, Epi &&epi) {
+    const int cta = blockIdx.x, G = gridDim.x;
+    if (ROLE == 0) gemm_produce_w(S, g, cta, G, r, pol);
+    else if (ROLE == 1) gemm_produce_x(S, g, cta, G, r, pol);
+    else gemm_consume<PAIR>(S, g, cta, G, r, epi);
+}
+
+struct NoEpi {
+    template <class T> __device__ __forceinline__ void operator()(int, T &) const {}
+};
+
+// ROLE 0: weight producer warp, 1: activation / KV producer warp, 2: consumer warps.
+template <int ROLE, int HD>
+__device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
+    const Ctx &c = A.c;
+    const MegaModel &M = *A.mm;
+    Smem *sm = S.sm;
+    const int G = gridDim.x, lane = threadIdx.x & 31;
+    const int L = c.L, d_model = c.d, qd = c.nq * c.hd, ntd = d_model / 16;
+    const uint64_t pol = ROLE == 0 ? policy_evict_first() : policy_evict_last();
+    Rings r{0, 0};
+    unsigned bar_no = 0, pub_no = 0;
+    int steps_started = 0;
+    StepDesc d;
+    d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0;
+#pragma unroll
+    for (int i = 0; i < MAX_COLS; ++i) { d.first_layer[i] = INT_MAX; d.pos[i] = 0; }
+
+    // barrier between phases, per role; CTA 0 books the time since the previous one to the phase's class
+    unsigned long long t_last = gtime();
+    auto phase_barrier = [&](int cls) {
+        if (ROLE == 2) {
+            barrier_consumers(S, A.grid_ctr, bar_no, G, cls);
+            if (blockIdx.x == 0 && threadIdx.x == 0) {
+                const unsigned long long t = gtime();
+                c.st->st.phase_ns[cls] += (long long)(t - t_last);
+                c.st->st.phase_count[cls] += 1;
+                t_last = t;
+            }
+        } else ++bar_no;
+    };
+    auto book_control = [&]() {
+        if (ROLE == 2 && blockIdx.x == 0 && threadIdx.x == 0) {
+            const unsigned long long t = gtime();
+            c.st->st.phase_ns[0] += (long long)(t - t_last);
+            c.st->st.phase_count[0] += 1;
+            t_last = t;
+        }
+    };
+    // the activation producer must not fetch a phase's input before the phase that wrote it is complete
+    auto x_ready = [&]() {
+        if (ROLE == 1) {
+            grid_wait(S, A.grid_ctr, bar_no * (unsigned)G);
+            fence_proxy_async();
+        }
+    };
+    // head over E* with the fused (max, sum exp, argmax) reduction; X = final-normed residual (or T output)
+    auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols) {
+        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0;
+        x_ready();
+        if (ROLE == 2) {
+            if (ssq) compute_rstd(sm, ssq, ntd, d_model, c.eps);
+            Msa run[2];
+            run[0].m = run[1].m = -INFINITY; run[0].s = run[1].s = 0.f; run[0].i = run[1].i = INT_MAX;
+            const int c0 = 2 * (lane & 3);
+            const float r0 = ssq ? sm->vec[c0] * scale : scale, r1 = ssq ? sm->vec[c0 + 1] * scale : scale;
+            gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8;
+                    if (n < c.vocab) {
+                        const float z = acc[0][i] * ((i & 1) ? r1 : r0);
+                        if (A.store_logits && ((cols >> (c0 + (i & 1))) & 1u)) c.logit_stage[(size_t)(c0 + (i & 1)) * c.vocab + n] = z;
+                        Msa one; one.m = z; one.s = 1.f; one.i = n;
+                        run[i & 1] = msa_merge(run[i & 1], one);
+                    }
+                }
+            });
+            // lanes sharing lane%4 hold the same columns: fold them, then the warps, in a fixed order
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    Msa o;
+                    o.m = __shfl_xor_sync(0xffffffffu, run[q].m, off);
+                    o.s = __shfl_xor_sync(0xffffffffu, run[q].s, off);
+                    o.i = __shfl_xor_sync(0xffffffffu, run[q].i, off);
+                    run[q] = msa_merge(run[q], o);
+                }
+            }
+            const int warp = threadIdx.x >> 5;
+            float *wp = reinterpret_cast<float *>(sm->scratch);   // [warp][col][4]
+            bar_consumers();
+            if (lane < 4) {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    float *o = wp + ((size_t)warp * MAX_COLS + c0 + q) * 4;
+                    o[0] = run[q].m; o[1] = run[q].s; o[2] = __int_as_float(run[q].i);
+                }
+            }
+            bar_consumers();
+            if (threadIdx.x < MAX_COLS) {
+                Msa a; a.m = -INFINITY; a.s = 0.f; a.i = INT_MAX;
+                for (int w = 0; w < CONS_WARPS; ++w) {
+                    const float *o = wp + ((size_t)w * MAX_COLS + threadIdx.x) * 4;
+                    Msa x; x.m = o[0]; x.s = o[1]; x.i = __float_as_int(o[2]);
+                    a = msa_merge(a, x);
+                }
+                float *o = A.head_part + ((size_t)blockIdx.x * MAX_COLS + threadIdx.x) * 4;
+                o[0] = a.m; o[1] = a.s; o[2] = __int_as_float(a.i);
+            }
+        } else {
+            gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+        }
+        phase_barrier(9);
+    };
+
+    int action = control_point<ROLE>(A, S, CTRL_START, 0, pub_no, d, steps_started);
+    book_control();
+    int step_i = 0;
+    while (action == ACT_NEWSTEP) {
+        bool restart = false;
+        S.tr_on = step_i >= A.trace_step0 && step_i < A.trace_step1;
+        ++step_i;
+        for (int l = 0; l < L; ++l) {
+            const MegaLayer &ly = M.layer[l];
+            const unsigned mask = active_mask(d, l);
+            // ---- QKV
+            {
+                Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0;
+                x_ready();
+                if (ROLE == 2) {
+                    compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);
+                    const int c0 = 2 * (lane & 3);
+                    const float r0 = sm->vec[c0], r1 = sm->vec[c0 + 1];
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
+                            if (n < c.qkv_rows && ((mask >> cc) & 1u)) A.qkvraw[(size_t)cc * c.qkv_rows + n] = acc[0][i] * ((i & 1) ? r1 : r0);
+                        }
+                    });
+                } else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+                phase_barrier(2);
+            }
+            // ---- attention (the KV producer may run ahead: rows of this pass are patched in by the consumers)
+            if (ROLE == 1) attn_produce(A, S, d, l, r, pol);
+            if (ROLE == 2) attn_consume<HD>(A, S, d, l, mask, r);
+            phase_barrier(4);
+            // ---- O projection + residual; prepares the FFN input
+            {
+                Gemm g; g.W = ly.wo; g.X = reinterpret_cast<const uint4 *>(A.XO); g.N = d_model; g.K = qd; g.pair = 1; g.half = 0;
+                x_ready();
+                if (ROLE == 2) {
+                    const __nv_bfloat16 *gain = ly.ffn_norm;
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                        const int c0 = 2 * (lane & 3);
+                        float sq[2] = {0.f, 0.f};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
+                            if ((mask >> cc) & 1u) {
+                                float *rp = c.resid + (size_t)cc * d_model + n;
+                                const float v = *rp + acc[0][i];
+                                *rp = v;
+                                xfrag_store(A.XB, n, cc, v * __bfloat162float(gain[n]));
+                                sq[i & 1] += v * v;
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            sq[q] += __shfl_xor_sync(0xffffffffu, sq[q], 4);
+                            sq[q] += __shfl_xor_sync(0xffffffffu, sq[q], 8);
+                            sq[q] += __shfl_xor_sync(0xffffffffu, sq[q], 16);
+                            if (lane < 4 && ((mask >> (c0 + q)) & 1u)) A.ssq_b[(size_t)tile * MAX_COLS + c0 + q] = sq[q];
+                        }
+                    });
+                } else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+                phase_barrier(5);
+            }
+            // ---- gate / up + SwiGLU
+            {
+                Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff;
+                x_ready();
+                if (ROLE == 2) {
+                    compute_rstd(sm, A.ssq_b, ntd, d_model, c.eps);
+                    const int c0 = 2 * (lane & 3);
+                    const float r0 = sm->vec[c0], r1 = sm->vec[c0 + 1];
+                    gemm_consume<2>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[2][4]) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
+                            if ((mask >> cc) & 1u) {
+                                const float rs = (i & 1) ? r1 : r0;
+                                const float gv = acc[0][i] * rs, u = acc[1][i] * rs;
+                                xfrag_store(A.XH, n, cc, gv / (1.0f + expf(-gv)) * u);
+                            }
+                        }
+                    });
+                } else gemm_phase<ROLE, 2>(S, g, r, pol, NoEpi());
+                phase_barrier(6);
+            }
+            // ---- down projection + residual; prepares the next layer's (and the head's) input
+            {
+                Gemm g; g.W = ly.wdown; g.X = reinterpret_cast<const uint4 *>(A.XH); g.N = d_model; g.K = c.dff; g.pair = 1; g.half = 0;
+                x_ready();
+                if (ROLE == 2) {
+                    const __nv_bfloat16 *gain_next = l + 1 < L ? M.layer[l + 1].attn_norm : nullptr;
+                    const bool want_f = l + 1 == L || A.exit_at[l + 1] != 0;
+                    const __nv_bfloat16 *gain_f = M.final_norm;
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                        const int c0 = 2 * (lane & 3);
+                        float sq[2] = {0.f, 0.f};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
+                            if ((mask >> cc) & 1u) {
+                                float *rp = c.resid + (size_t)cc * d_model + n;
+                                const float v = *rp + acc[0][i];
+                                *rp = v;
+                                if (gain_next) xfrag_store(A.XA, n, cc, v * __bfloat162float(gain_next[n]));
+                                if (want_f) xfrag_store(A.XF, n, cc, v * __bfloat162float(gain_f[n]));
+                                sq[i & 1] += v * v;
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            sq[q] += __shfl_xor_sync(0xffffffffu, sq[q], 4);
+                            sq[q] += __shfl_xor_sync(0xffffffffu, sq[q], 8);
+                            sq[q] += __shfl_xor_sync(0xffffffffu, sq[q], 16);
+                            if (lane < 4 && ((mask >> (c0 + q)) & 1u)) A.ssq_a[(size_t)tile * MAX_COLS + c0 + q] = sq[q];
+                        }
+                    });
+                } else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+                phase_barrier(8);
+            }
+            // ---- intermediate head (Section 2.1) and the early-prediction rule (Eq. 1)
+            if (l + 1 < L && A.exit_at[l + 1] != 0 && d.head_ok) {
+                const MegaLayer &hl = M.layer[l + 1];
+                if (hl.wT) {
+                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0;
+                    x_ready();
+                    if (ROLE == 2) {
+                        compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);
+                        const int c0 = 2 * (lane & 3);
+                        const float r0 = sm->vec[c0], r1 = sm->vec[c0 + 1];
+                        gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
+                                xfrag_store(A.XT, n, cc, acc[0][i] * ((i & 1) ? r1 : r0));
+                            }
+                        });
+                    } else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+                    phase_barrier(10);
+                    head_phase(A.XT, nullptr, hl.head_scale, 0u);
+                } else {
+                    head_phase(A.XF, A.ssq_a, hl.head_scale, 0u);
+                }
+                action = control_point<ROLE>(A, S, CTRL_HEAD, l + 1, pub_no, d, steps_started);
+                book_control();
+                if (action != ACT_CONTINUE) { restart = true; break; }
+            }
+        }
+        if (!restart) {
+            // ---- final head for every column, then verification (Eq. 2 at temperature zero) in the control point
+            head_phase(A.XF, A.ssq_a, 1.0f, active_mask(d, L - 1));
+            action = control_point<ROLE>(A, S, CTRL_TOP, 0, pub_no, d, steps_started);
+            book_control();
+        }
+    }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(THREADS, 1) k_decode_persistent(const __grid_constant__ MegaArgs A) {
+    extern __shared__ unsigned char smem_raw[];
+    Smem *sm = smem_base(smem_raw);
+    smem_init(sm);
+    __syncthreads();
+    Shared S{sm, A.err, A.trace, 0};
+    const int warp = threadIdx.x >> 5;
+    if (warp == CONS_WARPS) run<0, HD>(A, S);
+    else if (warp == CONS_WARPS + 1) run<1, HD>(A, S);
+    else run<2, HD>(A, S);
+    settle_on_abort(S);
+}
+
+}  // namespace mg
+}  // namespace ada
