@@ -154,15 +154,31 @@ int ada_debug_get_state(ada_session *s, int32_t seq, int32_t *len_out, int32_t *
 /* Copy K (which=0) or V (which=1) of one cached position of one layer into host_out
  * [n_kv_heads*head_dim] as fp32. */
 int ada_debug_read_kv(ada_session *s, int32_t seq, int32_t which, int32_t layer0, int32_t pos, float *host_out);
-/* Per-kernel-class device timing (CUDA events around every launch; slows the run, for analysis
- * only).  Classes: 0 step set-up and control, 1 RMSNorm, 2 QKV GEMM, 3 RoPE + KV write, 4 attention,
+/* Per-kernel-class device timing (path 0: CUDA events around every launch, which slows the run;
+ * path 1: the persistent kernel's own per-phase timers, read in CTA 0, always running).  Classes: 0 step set-up and control, 1 RMSNorm, 2 QKV GEMM, 3 RoPE + KV write, 4 attention,
  * 5 O-proj GEMM, 6 gate/up GEMM, 7 SwiGLU, 8 down GEMM, 9 LM-head stream, 10 head transformation T,
  * 11 other.  ada_debug_profile_read returns, accumulated since profiling was switched on, the device
  * milliseconds, launch counts and algorithmic HBM bytes (weights or KV the launch must read) per class. */
 int ada_debug_profile(ada_session *s, int32_t on);
 int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out, double *bytes_out);
-/* Select the GEMM path: 0 = CUDA-core kernels (any dtype), 1 = tensor-core kernels (bf16 only). */
+/* Select the decode path: 1 = the persistent kernel (one cooperative launch runs many steps of
+ * Algorithm 1; bf16 models, one sequence, at most 8 tokens per pass, 64-token KV pages, head_dim 64
+ * or 128, at most 4 q heads per kv head, d_model / n_q_heads*head_dim / d_ff multiples of 64,
+ * max_seq_len at most 256 * head_dim); it is the default wherever a session qualifies.  0 = one
+ * kernel per operation on CUDA cores (any dtype, any batch; also what prefill uses).
+ * ADA_EUNSUPPORTED if path 1 is asked of a session that does not qualify. */
 int ada_debug_set_path(ada_session *s, int32_t path);
+int ada_debug_get_path(ada_session *s, int32_t *path_out);
+/* Steps of Algorithm 1 one launch of the persistent kernel may start before it returns to the host
+ * (default 256; the host relaunches until the call is complete). */
+int ada_debug_set_launch_steps(ada_session *s, int32_t steps);
+/* Event trace of the persistent kernel: while the kernel runs the steps [step0, step1) of a launch
+ * (counted from 0 in every launch), every CTA appends (nanosecond timestamp, code) pairs of
+ * uint64 to dev_buf [cap_events][2]; code = CTA << 32 | argument << 8 | event (1 phase begin, 2
+ * first activation stage landed, 3 first weight stage landed, 4 last tile group multiplied, 5
+ * epilogue done, 6 / 7 weight producer starts / ends a phase, 8 attention item done, 9 attention
+ * chunks merged, 10 barrier arrival).  count_dev receives the number of events.  NULL stops. */
+int ada_debug_trace(ada_session *s, uint64_t *dev_buf, uint32_t *count_dev, uint32_t cap_events, int32_t step0, int32_t step1);
 
 /* Run the weight-streaming skinny GEMM of the decode kernel by itself (the kernel behind the QKV,
  * O, gate/up, down and LM-head products of a layer pass, Algorithm 1 "process all tokens in P[l]

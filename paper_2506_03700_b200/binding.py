@@ -27,7 +27,7 @@ EXPORTS = [
     "ada_session_create", "ada_session_destroy", "ada_session_reset", "ada_prefill", "ada_plain_decode",
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
-    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_work_bytes",
+    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace",
 ]
 
 
@@ -102,6 +102,9 @@ def load() -> C.CDLL:
         L.ada_debug_get_state.argtypes = [vp, i32, C.POINTER(i32), vp]
         L.ada_debug_read_kv.argtypes = [vp, i32, i32, i32, i32, vp]
         L.ada_debug_set_path.argtypes = [vp, i32]
+        L.ada_debug_get_path.argtypes = [vp, C.POINTER(i32)]
+        L.ada_debug_set_launch_steps.argtypes = [vp, i32]
+        L.ada_debug_trace.argtypes = [vp, vp, vp, C.c_uint32, i32, i32]
         L.ada_debug_profile.argtypes = [vp, i32]
         L.ada_debug_profile_read.argtypes = [vp, vp, vp, vp]
         L.ada_debug_gemm_work_bytes.restype = sz
@@ -284,6 +287,30 @@ class Session:
 
     def set_path(self, path: int):
         _ck(load().ada_debug_set_path(self.h, path), "ada_debug_set_path")
+
+    def get_path(self) -> int:
+        p = C.c_int32(-1)
+        _ck(load().ada_debug_get_path(self.h, C.byref(p)), "ada_debug_get_path")
+        return p.value
+
+    def set_launch_steps(self, steps: int):
+        _ck(load().ada_debug_set_launch_steps(self.h, steps), "ada_debug_set_launch_steps")
+
+    def trace(self, cap_events: int, step0: int, step1: int):
+        """Record the persistent kernel's events of steps [step0, step1) of every following launch."""
+        import torch
+        self._trace = torch.zeros(cap_events, 2, dtype=torch.int64, device="cuda")
+        self._trace_n = torch.zeros(1, dtype=torch.int32, device="cuda")
+        _ck(load().ada_debug_trace(self.h, self._trace.data_ptr(), self._trace_n.data_ptr(), cap_events, step0, step1),
+            "ada_debug_trace")
+
+    def traced(self) -> np.ndarray:
+        """Rows (ns, cta, arg, event) of the recorded events, in time order."""
+        n = min(int(self._trace_n.item()), self._trace.shape[0])
+        t = self._trace[:n].cpu().numpy()
+        code = t[:, 1]
+        out = np.stack([t[:, 0], code >> 32, (code >> 8) & 0xffff, code & 0xff], axis=1)
+        return out[np.argsort(out[:, 0], kind="stable")]
 
     def __del__(self):
         try:

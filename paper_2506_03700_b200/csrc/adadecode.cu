@@ -4,11 +4,13 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <memory>
 #include <string>
 #include <vector>
 
 #include "kernels.cuh"
 #include "gemm_probe.cuh"
+#include "mega.cuh"
 
 using namespace ada;
 
@@ -93,6 +95,14 @@ struct ada_session {
     int32_t *pinned = nullptr; // small read-back area
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     int path = 0;
+    // persistent-kernel path (bf16, one sequence, up to eight token columns)
+    bool mega = false;
+    int grid = 0;
+    mg::MegaArgs margs;
+    CUtensorMap *maps_dev = nullptr;      // [5 L + 2]: wqkv, wo, wgu, wdown per layer, lm_head, then T per 1-based layer
+    mg::MegaModel *mm_dev = nullptr;
+    int *exit_at_dev = nullptr;
+    int steps_per_launch = 256;
     int64_t launches = 0, syncs = 0, layer_passes = 0;
     // per-class profiling
     bool prof = false;
@@ -107,6 +117,8 @@ struct ada_session {
     int head_log_cap = 0;
     int32_t *head_log_n_out = nullptr;
     std::vector<uint8_t> tape;
+    std::vector<CUtensorMap> maps_host;
+    std::unique_ptr<mg::MegaModel> mm_host;
 };
 
 namespace {
@@ -114,13 +126,14 @@ namespace {
 // Scratch layout (all offsets 256-byte aligned).
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
-        head_part, logit_stage, head_log, t_out, total;
+        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qkvraw, attn_cnt,
+        grid_ctr, pub, err, total;
 };
 
 int rows_alloc_for(int batch, int max_early) { return std::max(batch * (max_early + 1), 32); }
 
 Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, int head_blocks) {
-    Layout L;
+    Layout L{};
     const int R = rows_alloc_for(batch, max_early);
     const int qd = g.n_q_heads * g.head_dim, qkv_rows = (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim;
     const int n_chunks = (max_seq + kAttnChunk - 1) / kAttnChunk;
@@ -146,6 +159,25 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
     L.logit_stage = take(sizeof(float) * (size_t)R * g.vocab);
     L.head_log = take(sizeof(float) * 4 * kHeadLogCap);
     L.t_out = take(sizeof(float) * (size_t)R * g.d_model);
+    // persistent-kernel buffers (bf16 models)
+    if (g.dtype == ADA_DTYPE_BF16) {
+        L.maps = take(sizeof(CUtensorMap) * (5 * (size_t)g.n_layers + 2));
+        L.mm = take(sizeof(mg::MegaModel));
+        L.exit_at = take(sizeof(int) * (g.n_layers + 1));
+        L.xa = take(st::xfrag_bytes(g.d_model));
+        L.xb = take(st::xfrag_bytes(g.d_model));
+        L.xf = take(st::xfrag_bytes(g.d_model));
+        L.xt = take(st::xfrag_bytes(g.d_model));
+        L.xo = take(st::xfrag_bytes(qd));
+        L.xh = take(st::xfrag_bytes(g.d_ff));
+        L.ssq_a = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
+        L.ssq_b = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
+        L.qkvraw = take(sizeof(float) * (size_t)st::MAX_COLS * qkv_rows);
+        L.attn_cnt = take(sizeof(unsigned) * g.n_kv_heads);
+        L.grid_ctr = take(256);
+        L.pub = take(sizeof(mg::Pub) * 2);
+        L.err = take(256);
+    }
     L.total = o;
     return L;
 }
@@ -371,10 +403,145 @@ void add_stats(ada_session *S, const DevStats &d, ada_stats *out, float ms, int6
     out->verify_steps += d.verify_steps; out->accepted += d.accepted; out->rejected += d.rejected;
     out->discarded += d.discarded; out->row_layers += d.row_layers; out->truncated += d.truncated;
     for (int i = 0; i < ADA_MAX_LAYERS; ++i) out->exits_at_layer[i] += d.exits_at_layer[i];
-    out->layer_passes += S->layer_passes - p0;
+    out->layer_passes += S->layer_passes - p0 + d.layer_passes;
     out->host_syncs += S->syncs - s0;
     out->kernel_launches += S->launches - l0;
     out->decode_ms += ms;
+}
+
+// ---- persistent-kernel path --------------------------------------------------------------------
+
+template <int HD> const void *persistent_kernel() { return (const void *)mg::k_decode_persistent<HD>; }
+const void *persistent_kernel_for(int hd) { return hd == 64 ? persistent_kernel<64>() : persistent_kernel<128>(); }
+
+// Decide whether this session can run the persistent kernel and build what it needs: tensor maps
+// of every weight matrix, the device-side model description, the argument block.
+int setup_persistent(ada_session *S, const Layout &lay) {
+    const ada_model *m = S->m;
+    const ada_config &g = m->cfg;
+    S->mega = false;
+    S->path = 0;
+    const int qd = g.n_q_heads * g.head_dim, group = g.n_q_heads / g.n_kv_heads;
+    if (g.dtype != ADA_DTYPE_BF16 || S->batch != 1 || S->slots > st::MAX_COLS || S->page_tokens != mg::ATT_PAGE) return ADA_OK;
+    if ((g.head_dim != 64 && g.head_dim != 128) || group > 4) return ADA_OK;
+    if (g.d_model % 64 || qd % 64 || g.d_ff % 64) return ADA_OK;
+    if (S->n_chunks > g.head_dim) return ADA_OK;   // the chunk merge stages 2 x 32 x n_chunks floats in shared memory
+    int dev = 0, sms = 0, coop = 0, nb = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return ADA_OK; }
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    const void *kern = persistent_kernel_for(g.head_dim);
+    if (!coop || sms < 1 ||
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st::SMEM_BYTES) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, st::THREADS, st::SMEM_BYTES) != cudaSuccess || nb < 1) {
+        cudaGetLastError();
+        return ADA_OK;
+    }
+    S->grid = std::min(sms, S->head_blocks);
+    const int L = g.n_layers;
+    char *b = (char *)S->scratch;
+    S->maps_dev = (CUtensorMap *)(b + lay.maps);
+    S->mm_dev = (mg::MegaModel *)(b + lay.mm);
+    S->exit_at_dev = (int *)(b + lay.exit_at);
+    S->maps_host.assign(5 * (size_t)L + 2, CUtensorMap());
+    S->mm_host.reset(new mg::MegaModel());
+    mg::MegaModel &M = *S->mm_host;
+    memset(&M, 0, sizeof(M));
+    for (int l = 0; l < L; ++l) {
+        const LayerW &w = m->layers[l];
+        if (make_weight_map(&S->maps_host[4 * l + 0], w.wqkv, S->c.qkv_rows, g.d_model) ||
+            make_weight_map(&S->maps_host[4 * l + 1], w.wo, g.d_model, qd) ||
+            make_weight_map(&S->maps_host[4 * l + 2], w.w_gate_up, 2 * g.d_ff, g.d_model) ||
+            make_weight_map(&S->maps_host[4 * l + 3], w.w_down, g.d_model, g.d_ff))
+            return ADA_OK;
+        M.layer[l].wqkv = S->maps_dev + 4 * l + 0;
+        M.layer[l].wo = S->maps_dev + 4 * l + 1;
+        M.layer[l].wgu = S->maps_dev + 4 * l + 2;
+        M.layer[l].wdown = S->maps_dev + 4 * l + 3;
+        M.layer[l].attn_norm = (const __nv_bfloat16 *)w.attn_norm;
+        M.layer[l].ffn_norm = (const __nv_bfloat16 *)w.ffn_norm;
+    }
+    if (make_weight_map(&S->maps_host[4 * L], m->lm_head, g.vocab, g.d_model)) return ADA_OK;
+    M.lm_head = S->maps_dev + 4 * L;
+    M.tok_embed = (const __nv_bfloat16 *)m->tok_embed;
+    M.final_norm = (const __nv_bfloat16 *)m->final_norm;
+    M.rope_base = g.rope_base;
+    CK(cudaMemcpyAsync(S->maps_dev, S->maps_host.data(), sizeof(CUtensorMap) * S->maps_host.size(), cudaMemcpyHostToDevice, S->stream));
+    CK(cudaMemcpyAsync(S->mm_dev, &M, sizeof(M), cudaMemcpyHostToDevice, S->stream));
+    CK(cudaStreamSynchronize(S->stream));
+    mg::MegaArgs &a = S->margs;
+    a.c = S->c;
+    a.mm = S->mm_dev;
+    a.exit_at = S->exit_at_dev;
+    a.XA = (__nv_bfloat16 *)(b + lay.xa); a.XB = (__nv_bfloat16 *)(b + lay.xb); a.XO = (__nv_bfloat16 *)(b + lay.xo);
+    a.XH = (__nv_bfloat16 *)(b + lay.xh); a.XF = (__nv_bfloat16 *)(b + lay.xf); a.XT = (__nv_bfloat16 *)(b + lay.xt);
+    a.ssq_a = (float *)(b + lay.ssq_a); a.ssq_b = (float *)(b + lay.ssq_b);
+    a.qkvraw = (float *)(b + lay.qkvraw);
+    a.attn_part = S->c.attn_part;
+    a.head_part = S->c.head_part;
+    a.attn_cnt = (unsigned *)(b + lay.attn_cnt);
+    a.grid_ctr = (unsigned *)(b + lay.grid_ctr);
+    a.pub = (mg::Pub *)(b + lay.pub);
+    a.err = (int *)(b + lay.err);
+    a.step_budget = S->steps_per_launch;
+    a.store_logits = 0;
+    a.trace = st::Trace{nullptr, nullptr, 0};
+    a.trace_step0 = a.trace_step1 = 0;
+    S->mega = true;
+    S->path = 1;
+    return ADA_OK;
+}
+
+// Run the persistent kernel until the call's token targets are met.
+int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool plain) {
+    const ada_model *m = S->m;
+    const ada_config &g = m->cfg;
+    const int L = g.n_layers;
+    std::vector<int> ex(L + 1, 0);
+    mg::MegaModel &M = *S->mm_host;
+    if (!plain) {
+        for (int i = 0; i < n_exit; ++i) {
+            const int e = exit_layers[i];
+            ex[e] = 1;
+            M.layer[e].has_head = 1;
+            M.layer[e].head_scale = m->head_scale[e];
+            M.layer[e].wT = nullptr;
+            if (m->head_T[e]) {
+                CUtensorMap &tm = S->maps_host[4 * (size_t)L + 1 + e];
+                int rc = make_weight_map(&tm, m->head_T[e], g.d_model, g.d_model);
+                if (rc) return rc;
+                CK(cudaMemcpyAsync(S->maps_dev + 4 * L + 1 + e, &tm, sizeof(tm), cudaMemcpyHostToDevice, S->stream));
+                M.layer[e].wT = S->maps_dev + 4 * L + 1 + e;
+            }
+            CK(cudaMemcpyAsync(&S->mm_dev->layer[e], &M.layer[e], sizeof(mg::MegaLayer), cudaMemcpyHostToDevice, S->stream));
+        }
+    }
+    CK(cudaMemcpyAsync(S->exit_at_dev, ex.data(), sizeof(int) * (L + 1), cudaMemcpyHostToDevice, S->stream));
+    CK(cudaStreamSynchronize(S->stream));   // ex and the maps live on the host until copied
+    S->syncs++;
+    mg::MegaArgs a = S->margs;
+    a.c = S->c;   // capture pointers may have changed
+    a.step_budget = S->steps_per_launch;
+    a.store_logits = S->capture_dev ? 1 : 0;
+    const void *kern = persistent_kernel_for(g.head_dim);
+    for (long long guard = 0;; ++guard) {
+        if (guard > (1ll << 24)) return ADA_ETIMEOUT;
+        CK(cudaMemsetAsync(a.grid_ctr, 0, sizeof(unsigned), S->stream));
+        CK(cudaMemsetAsync(a.pub, 0, sizeof(mg::Pub) * 2, S->stream));
+        void *params[] = {(void *)&a};
+        CK(cudaLaunchCooperativeKernel(kern, dim3(S->grid), dim3(st::THREADS), params, st::SMEM_BYTES, S->stream));
+        S->launches++;
+        CK(cudaMemcpyAsync(S->pinned, &S->c.st->n_climbing, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+        CK(cudaMemcpyAsync(S->pinned + 2, a.err, sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+        CK(cudaStreamSynchronize(S->stream));
+        S->syncs++;
+        if (S->pinned[2] != 0) {
+            g_cuda_err = "persistent decode kernel: device-side error " + std::to_string(S->pinned[2]);
+            return S->pinned[2] == mg::ERR_BAD_STATE ? ADA_ESTATE : ADA_ETIMEOUT;
+        }
+        if (S->pinned[1] >= S->batch) break;
+    }
+    return ADA_OK;
 }
 
 // Shared body of both decode calls.
@@ -413,7 +580,9 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
     S->launches++;
 
     const bool plain = (n_exit == 0 || max_early == 0);
-    if (plain) {
+    if (S->mega && S->path == 1) {
+        if ((rc = run_persistent(S, exit_layers, n_exit, plain))) return rc;
+    } else if (plain) {
         // every step is one token through all layers; the step count is known, no read-back needed
         for (int it = 0; it < max_steps_plain; ++it) {
             if ((rc = step_begin(S))) return rc;
@@ -492,7 +661,18 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
         S->h_len[s] = tg.target_len[s];
     }
     S->tape.clear();
-    if (S->prof) prof_collect(S);
+    if (S->prof) {
+        prof_collect(S);
+        const ada_config &g = m->cfg;
+        const double esz = (double)m->esz, d = g.d_model, qdm = (double)g.n_q_heads * g.head_dim;
+        const double wbytes[ADA_PROF_CLASSES] = {0, 0, (double)S->c.qkv_rows * d * esz, 0, 0, d * qdm * esz, 2.0 * g.d_ff * d * esz, 0,
+                                                 d * g.d_ff * esz, (double)g.vocab * d * esz, d * d * esz, 0};
+        for (int i = 0; i < ADA_PROF_CLASSES; ++i) {   // phases of the persistent kernel, timed on the device
+            S->prof_ms[i] += (double)ds.phase_ns[i] * 1e-6;
+            S->prof_launches[i] += ds.phase_count[i];
+            S->prof_bytes[i] += wbytes[i] * (double)ds.phase_count[i];
+        }
+    }
     add_stats(S, ds, stats, ms, l0, s0, p0);
     return ADA_OK;
 }
@@ -668,8 +848,13 @@ int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, i
     memset(&hs, 0, sizeof(hs));
     hs.batch = batch; hs.slots = S->slots; hs.n_layers = g.n_layers; hs.max_seq = max_seq_len;
     CKS(cudaMemcpyAsync(c.st, &hs, offsetof(DevState, len), cudaMemcpyHostToDevice, S->stream));
+    CKS(cudaMemsetAsync(kv_pool_dev, 0, (size_t)n_pages * page_bytes, S->stream));   // masked cache rows must hold finite numbers
     CKS(cudaStreamSynchronize(S->stream));
 #undef CKS
+    {
+        int rc = setup_persistent(S, lay);
+        if (rc) return fail(rc);
+    }
     // free list: pages are handed out from the back, in a scrambled order so that the page-table
     // indirection is always exercised
     S->free_pages.resize(n_pages);
@@ -850,8 +1035,29 @@ int ada_debug_profile_read(ada_session *S, double *ms_out, int64_t *launches_out
 
 int ada_debug_set_path(ada_session *S, int32_t path) {
     if (!S || path < 0 || path > 1) return ADA_EINVAL;
-    if (path == 1) return ADA_EUNSUPPORTED;
+    if (path == 1 && !S->mega) return ADA_EUNSUPPORTED;
     S->path = path;
+    return ADA_OK;
+}
+
+int ada_debug_get_path(ada_session *S, int32_t *path_out) {
+    if (!S || !path_out) return ADA_EINVAL;
+    *path_out = S->path;
+    return ADA_OK;
+}
+
+int ada_debug_set_launch_steps(ada_session *S, int32_t steps) {
+    if (!S || steps < 1) return ADA_EINVAL;
+    S->steps_per_launch = steps;
+    return ADA_OK;
+}
+
+int ada_debug_trace(ada_session *S, uint64_t *dev_buf, uint32_t *count_dev, uint32_t cap_events, int32_t step0, int32_t step1) {
+    if (!S || !S->mega) return ADA_EUNSUPPORTED;
+    if (dev_buf && (!count_dev || cap_events < 1 || step0 < 0 || step1 < step0)) return ADA_EINVAL;
+    S->margs.trace = st::Trace{(unsigned long long *)dev_buf, count_dev, dev_buf ? cap_events : 0};
+    S->margs.trace_step0 = dev_buf ? step0 : 0;
+    S->margs.trace_step1 = dev_buf ? step1 : 0;
     return ADA_OK;
 }
 
