@@ -77,6 +77,21 @@ def check_against_oracle(pair, prompt, gpu_tokens, gpu_logits):
     return worst
 
 
+def clear_gamma(pair, prompt, n, exits, cap, gamma0, tol, max_seq=256):
+    """A threshold near gamma0 that no head probability of the oracle's own run comes within `tol` of
+    (so that the GPU, whose probabilities differ by rounding, takes the same decisions).  The set of
+    probabilities depends on the threshold, so every candidate is checked by an oracle run."""
+    for k in range(40):
+        gamma = gamma0 + 0.0173 * ((k + 1) // 2) * (1 if k % 2 else -1)
+        O = oracle.Session(pair.om, max_seq)
+        O.record_heads()
+        O.prefill(prompt)
+        O.adaptive_decode(n, gamma, exits, cap)
+        if len(O.heads) and np.abs(O.heads[:, 3] - gamma).min() > tol:
+            return gamma
+    return None
+
+
 @pytest.mark.parametrize("mk,dtype,n_prompt,n_gen", [(small, "fp32", 7, 40), (small, "bf16", 7, 40),
                                                      (medium, "fp32", 33, 24), (medium, "bf16", 70, 24)])
 def test_plain_decode_matches_oracle(mk, dtype, n_prompt, n_gen):
@@ -144,7 +159,10 @@ def test_adaptive_schedule_and_heads_match_oracle(dtype, T_noise):
     cfg = medium(dtype)
     pair = Pair(cfg, T_noise=T_noise)
     prompt = synth.make_prompt(cfg, n=17).numpy()
-    n, gamma = 40, 0.45
+    n = 40
+    ptol = 1e-4 if dtype == "fp32" else 3e-3
+    gamma = clear_gamma(pair, prompt, n, cfg.exit_layers, 5, 0.45, 2 * ptol)
+    assert gamma is not None
     S = pair.gpu()
     S.capture_heads()
     S.prefill(prompt)
@@ -156,8 +174,7 @@ def test_adaptive_schedule_and_heads_match_oracle(dtype, T_noise):
     ost = oracle.Stats()
     ref = O.adaptive_decode(n, gamma, cfg.exit_layers, 5, stats=ost)
     gh, oh = S.captured_heads(), O.heads
-    ptol = 1e-4 if dtype == "fp32" else 2e-2
-    if np.array_equal(ref, out) and np.abs(oh[:, 3] - gamma).min() > ptol:
+    if np.array_equal(ref, out):
         assert len(gh) == len(oh)
         assert np.array_equal(gh[:, :3].astype(np.int64), oh[:, :3].astype(np.int64))
         assert np.abs(gh[:, 3] - oh[:, 3]).max() <= ptol
@@ -165,8 +182,14 @@ def test_adaptive_schedule_and_heads_match_oracle(dtype, T_noise):
                   "row_layers", "truncated"):
             assert getattr(st, k) == getattr(ost, k), k
         assert st.early_exits > 0
-    else:
-        pytest.skip("near-tie between the GPU and the oracle on this seed")
+    else:   # the two greedy runs part at a near-tie of the final logits: nothing to compare beyond it
+        O2 = pair.cpu()
+        O2.record_logits(n + 4)
+        O2.prefill(prompt)
+        r2 = O2.plain_decode(n)
+        k = int(np.argmax(r2 != out))
+        z = np.sort(O2.logits[k])
+        assert z[-1] - z[-2] <= tol(cfg, O2.logits[k].std())
 
 
 def test_forced_tapes_never_change_the_output():
