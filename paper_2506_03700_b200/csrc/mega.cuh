@@ -501,6 +501,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
 #pragma unroll
             for (int u = 0; u < VPT; ++u) nv[u] = __float2bfloat16_rn(vx[u]);
         }
+        if (tid == 0) trace(S, 15, 0);
         bar_consumers();   // the previous item is done with the shared buffers
         // ---- rotated, scaled queries -> A fragments (hi / lo)
 #pragma unroll
@@ -546,7 +547,9 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             float s[2][4];
             {   // ---- K block
                 const int slot = r.xi % NX;
+                if (tid == 0) trace(S, 11, sb);
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                if (tid == 0) trace(S, 12, sb);
                 unsigned char *kb = sm->x[slot];
                 if (newm) {
                     const size_t blk = ((((size_t)page * c.L + layer) * 2 + 0) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
@@ -627,7 +630,9 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             }
             {   // ---- V block
                 const int slot = r.xi % NX;
+                if (tid == 0) trace(S, 13, sb);
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                if (tid == 0) trace(S, 14, sb);
                 unsigned char *vb = sm->x[slot];
                 if (newm) {
                     const size_t blk = ((((size_t)page * c.L + layer) * 2 + 1) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
@@ -661,6 +666,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 ++r.xi;
             }
         }
+        if (tid == 0) trace(S, 16, 0);
         // ---- row sums over the quad, then merge the four position quarters of each query tile:
         //      (q0 + q1) and (q2 + q3), then the two halves
 #pragma unroll
