@@ -98,7 +98,16 @@ __device__ __forceinline__ unsigned active_mask(const StepDesc &d, int layer) {
 __device__ __forceinline__ void compute_rstd(Smem *sm, const float *ssq, int ntiles, int d, float eps) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float s = 0.f;
-    for (int t = lane; t < ntiles; t += 32) s += ldcg(ssq + (size_t)t * MAX_COLS + warp);
+    for (int t0 = 0; t0 < ntiles; t0 += 256) {   // eight loads in flight per lane; the order of the sum is fixed
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int t = t0 + lane + 32 * u;
+            v[u] = t < ntiles ? ldcg(ssq + (size_t)t * MAX_COLS + warp) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
+    }
     s = warp_sum(s);
     if (lane == 0) sm->vec[warp] = 1.0f / sqrtf(s / (float)d + eps);
     bar_consumers();
@@ -409,9 +418,11 @@ __device__ __forceinline__ void attn_merge_from(float (&o)[NT][4], float (&m_run
         m_run[rh] = mn;
         l_run[rh] = l_run[rh] * a + ls * b;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int i2 = 0; i2 < 2; ++i2) o[nt][2 * rh + i2] = o[nt][2 * rh + i2] * a + so[row][nt * 8 + 2 * (lane & 3) + i2] * b;
+        for (int nt = 0; nt < NT; ++nt) {   // columns rotated by 8 (row % 8): conflict-free 8-byte accesses
+            const float2 v = *reinterpret_cast<const float2 *>(&so[row][(nt * 8 + 2 * (lane & 3) + 8 * (row & 7)) & (HD - 1)]);
+            o[nt][2 * rh] = o[nt][2 * rh] * a + v.x * b;
+            o[nt][2 * rh + 1] = o[nt][2 * rh + 1] * a + v.y * b;
+        }
     }
 }
 template <int NT, int HD>
@@ -420,7 +431,10 @@ __device__ __forceinline__ void attn_merge_to(const float (&o)[NT][4], const flo
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) so[(lane >> 2) + 8 * (i >> 1)][nt * 8 + 2 * (lane & 3) + (i & 1)] = o[nt][i];
+        for (int rh = 0; rh < 2; ++rh) {
+            const int row = (lane >> 2) + 8 * rh;
+            *reinterpret_cast<float2 *>(&so[row][(nt * 8 + 2 * (lane & 3) + 8 * (row & 7)) & (HD - 1)]) = make_float2(o[nt][2 * rh], o[nt][2 * rh + 1]);
+        }
     if ((lane & 3) == 0) {
 #pragma unroll
         for (int rh = 0; rh < 2; ++rh) {
@@ -790,6 +804,9 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     Rings r{0, 0};
     unsigned bar_no = 0, pub_no = 0;
     int steps_started = 0;
+    // CTAs that share the tiles of each kind of GEMM (the rest idle through that phase)
+    const int n_qkv = balanced_ctas((c.qkv_rows + 15) / 16, G), n_d = balanced_ctas(ntd, G), n_gu = balanced_ctas(c.dff / 16, G),
+              n_head = balanced_ctas((c.vocab + 15) / 16, G);
     StepDesc d;
     d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0;
 #pragma unroll
@@ -825,7 +842,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     };
     // head over E* with the fused (max, sum exp, argmax) reduction; X = final-normed residual (or T output)
     auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols) {
-        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0;
+        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head;
         x_ready();
         if (ROLE == 2) {
             if (ssq) compute_rstd(sm, ssq, ntd, d_model, c.eps);
@@ -896,7 +913,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             const unsigned mask = active_mask(d, l);
             // ---- QKV
             {
-                Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0;
+                Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_qkv;
                 x_ready();
                 if (ROLE == 2) {
                     compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);
@@ -918,11 +935,18 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             phase_barrier(4);
             // ---- O projection + residual; prepares the FFN input
             {
-                Gemm g; g.W = ly.wo; g.X = reinterpret_cast<const uint4 *>(A.XO); g.N = d_model; g.K = qd; g.pair = 1; g.half = 0;
+                Gemm g; g.W = ly.wo; g.X = reinterpret_cast<const uint4 *>(A.XO); g.N = d_model; g.K = qd; g.pair = 1; g.half = 0; g.ctas = n_d;
                 x_ready();
                 if (ROLE == 2) {
                     const __nv_bfloat16 *gain = ly.ffn_norm;
-                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                    float rv[4] = {0.f, 0.f, 0.f, 0.f};
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile) {   // the residual is fetched while the weights stream
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = 2 * (lane & 3) + (i & 1);
+                            rv[i] = ((mask >> cc) & 1u) ? c.resid[(size_t)cc * d_model + n] : 0.f;
+                        }
+                    }, [&](int tile, float (&acc)[1][4]) {
                         const int c0 = 2 * (lane & 3);
                         float sq[2] = {0.f, 0.f};
 #pragma unroll
@@ -930,7 +954,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
                             if ((mask >> cc) & 1u) {
                                 float *rp = c.resid + (size_t)cc * d_model + n;
-                                const float v = *rp + acc[0][i];
+                                const float v = rv[i] + acc[0][i];
                                 *rp = v;
                                 xfrag_store(A.XB, n, cc, v * __bfloat162float(gain[n]));
                                 sq[i & 1] += v * v;
@@ -949,7 +973,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             }
             // ---- gate / up + SwiGLU
             {
-                Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff;
+                Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff; g.ctas = n_gu;
                 x_ready();
                 if (ROLE == 2) {
                     compute_rstd(sm, A.ssq_b, ntd, d_model, c.eps);
@@ -971,13 +995,20 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             }
             // ---- down projection + residual; prepares the next layer's (and the head's) input
             {
-                Gemm g; g.W = ly.wdown; g.X = reinterpret_cast<const uint4 *>(A.XH); g.N = d_model; g.K = c.dff; g.pair = 1; g.half = 0;
+                Gemm g; g.W = ly.wdown; g.X = reinterpret_cast<const uint4 *>(A.XH); g.N = d_model; g.K = c.dff; g.pair = 1; g.half = 0; g.ctas = n_d;
                 x_ready();
                 if (ROLE == 2) {
                     const __nv_bfloat16 *gain_next = l + 1 < L ? M.layer[l + 1].attn_norm : nullptr;
                     const bool want_f = l + 1 == L || A.exit_at[l + 1] != 0;
                     const __nv_bfloat16 *gain_f = M.final_norm;
-                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                    float rv[4] = {0.f, 0.f, 0.f, 0.f};
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = 2 * (lane & 3) + (i & 1);
+                            rv[i] = ((mask >> cc) & 1u) ? c.resid[(size_t)cc * d_model + n] : 0.f;
+                        }
+                    }, [&](int tile, float (&acc)[1][4]) {
                         const int c0 = 2 * (lane & 3);
                         float sq[2] = {0.f, 0.f};
 #pragma unroll
@@ -985,7 +1016,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
                             if ((mask >> cc) & 1u) {
                                 float *rp = c.resid + (size_t)cc * d_model + n;
-                                const float v = *rp + acc[0][i];
+                                const float v = rv[i] + acc[0][i];
                                 *rp = v;
                                 if (gain_next) xfrag_store(A.XA, n, cc, v * __bfloat162float(gain_next[n]));
                                 if (want_f) xfrag_store(A.XF, n, cc, v * __bfloat162float(gain_f[n]));
@@ -1007,7 +1038,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             if (l + 1 < L && A.exit_at[l + 1] != 0 && d.head_ok) {
                 const MegaLayer &hl = M.layer[l + 1];
                 if (hl.wT) {
-                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0;
+                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_d;
                     x_ready();
                     if (ROLE == 2) {
                         compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);

@@ -247,14 +247,30 @@ struct Gemm {
     const CUtensorMap *W;
     const uint4 *X;
     int N, K, pair, half;
+    int ctas;   // CTAs 0 .. ctas-1 share the tiles (see balanced_ctas); 0 = the whole grid
     __device__ __forceinline__ int tiles() const { return pair == 2 ? half / TILE_N : (N + TILE_N - 1) / TILE_N; }
 };
 
 struct Rings { uint32_t wi, xi; };   // stage counters of one role (slot = i % N, parity = (i / N) & 1)
 
 __device__ __forceinline__ void cta_tile_range(int T, int cta, int G, int &t0, int &t1) {
+    if (cta >= G) { t0 = t1 = 0; return; }
     t0 = (int)((long long)T * cta / G);
     t1 = (int)((long long)T * (cta + 1) / G);
+}
+// How many CTAs should share T equal tiles.  One SM's TMA unit moves at most about 58 GB/s of
+// 16 KB boxes, 1.3 times its fair share of HBM, so a CTA holding one tile more than the others
+// cannot catch up and everybody waits for it at the phase barrier.  About three quarters of the
+// SMs already saturate HBM, so the count in [0.76 G, G] that wastes the fewest tile slots
+// (ceil(T / g) g - T) is used; the idle CTAs prefetch the next phase meanwhile.
+__host__ __device__ inline int balanced_ctas(int T, int G) {
+    int lo = (G * 76 + 99) / 100, best = G;
+    long long best_waste = -1;
+    for (int g = G; g >= lo && g >= 1; --g) {
+        const long long waste = (long long)((T + g - 1) / g) * g - T;
+        if (best_waste < 0 || waste < best_waste) { best_waste = waste; best = g; }
+    }
+    return best;
 }
 
 // Weight producer warp: streams this CTA's tiles of the GEMM through the weight ring.
@@ -262,7 +278,7 @@ __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, i
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31;
     int t0, t1;
-    cta_tile_range(g.tiles(), cta, G, t0, t1);
+    cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
     const int nch = (g.K + KC - 1) / KC;
     if (lane == 0) trace(S, EV_WP_BEGIN, 0);
     for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
@@ -289,7 +305,7 @@ __device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, i
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31;
     int t0, t1;
-    cta_tile_range(g.tiles(), cta, G, t0, t1);
+    cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
     const int nch = (g.K + KC - 1) / KC;
     for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
         for (int kc = 0; kc < nch; ++kc) {
@@ -340,12 +356,13 @@ __device__ __forceinline__ void stage_full(float (&acc)[4][4], const unsigned ch
 // fixed order through shared memory, then `epi(tile, acc)` runs in the slot's first warp with
 //   acc[p][i]: fragment element i of matrix p: rows lane/4 (i<2) or lane/4+8, columns 2(lane%4)+(i&1).
 // The arrangement depends only on the tile partition, never on which token columns are in use.
-template <int PAIR, class Epi>
-__device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int cta, int G, Rings &r, Epi &&epi) {
+// `pre(tile)` runs in the same warp before the group's first stage (a place to start loads the epilogue will need).
+template <int PAIR, class Pre, class Epi>
+__device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int cta, int G, Rings &r, Pre &&pre, Epi &&epi) {
     Smem *sm = S.sm;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int t0, t1;
-    cta_tile_range(g.tiles(), cta, G, t0, t1);
+    cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
     const int nch = (g.K + KC - 1) / KC;
     // ldmatrix source of this lane inside a stage: row (lane%8) + 8 ((lane/8)%2), 16-byte chunk lane/16 of the k-step
     const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
@@ -356,6 +373,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
         while (TS < ng) TS <<= 1;
         const int KS = CONS_WARPS / TS;
         const int slot_id = warp % TS, ks_id = warp / TS;
+        if (ks_id == 0 && slot_id < ng) pre(g0 + slot_id);
         float acc[PAIR][4][4];   // [matrix][even/odd step x hi/lo][fragment]
 #pragma unroll
         for (int p = 0; p < PAIR; ++p)
@@ -441,6 +459,14 @@ static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a block
 __device__ __forceinline__ Smem *smem_base(unsigned char *raw) {
     const uint32_t a = s32(raw);
     return reinterpret_cast<Smem *>(raw + ((1024u - (a & 1023u)) & 1023u));
+}
+
+struct NoPre {
+    __device__ __forceinline__ void operator()(int) const {}
+};
+template <int PAIR, class Epi>
+__device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int cta, int G, Rings &r, Epi &&epi) {
+    gemm_consume<PAIR>(S, g, cta, G, r, NoPre(), epi);
 }
 
 // Shared-memory set-up by the whole block (call once, followed by __syncthreads()).
