@@ -119,7 +119,7 @@ def run_ours(args):
     build.build()
     cfg = synth.CONFIGS[args.workload]
     K, Wm = args.steps, args.warmup
-    gen_len = cfg.gen_len
+    gen_len = args.gen_len if args.gen_len > 0 else cfg.gen_len
     per_step = max(1, gen_len // K)
     gen_len = per_step * K
     max_seq = cfg.prompt_len + gen_len + 16
@@ -130,6 +130,8 @@ def run_ours(args):
         model.set_exit_head(l, None, cfg.logit_scale)
     prompt = synth.make_prompt(cfg, seed=5678).numpy()
     sess = binding.Session(model, 1, max_seq, 64, 5)
+    if args.launch_steps > 0:
+        sess.set_launch_steps(args.launch_steps)
     out = np.empty((1, per_step), dtype=np.int32)
     try:
         pinned = torch.empty((1, per_step), dtype=torch.int32).pin_memory()
@@ -296,6 +298,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=12)
     ap.add_argument("--ref-tokens", type=int, default=2)
+    ap.add_argument("--gen-len", type=int, default=0, help="generate this many tokens instead of the workload's (profiling runs)")
+    ap.add_argument("--launch-steps", type=int, default=0, help="decode steps per launch of the persistent kernel (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -174,10 +174,11 @@ int ada_debug_get_path(ada_session *s, int32_t *path_out);
 int ada_debug_set_launch_steps(ada_session *s, int32_t steps);
 /* Event trace of the persistent kernel: while the kernel runs the steps [step0, step1) of a launch
  * (counted from 0 in every launch), every CTA appends (nanosecond timestamp, code) pairs of
- * uint64 to dev_buf [cap_events][2]; code = CTA << 32 | argument << 8 | event (1 phase begin, 2
+ * uint64 to its own region of dev_buf [SMs][cap_events][2]; code = CTA << 32 | argument << 8 | event (1 phase begin, 2
  * first activation stage landed, 3 first weight stage landed, 4 last tile group multiplied, 5
  * epilogue done, 6 / 7 weight producer starts / ends a phase, 8 attention item done, 9 attention
- * chunks merged, 10 barrier arrival).  count_dev receives the number of events.  NULL stops. */
+ * chunks merged, 10 barrier arrival, 11.. attention sub-steps).  count_dev [SMs] receives the number of
+ * events of each CTA in the last traced launch.  NULL stops. */
 int ada_debug_trace(ada_session *s, uint64_t *dev_buf, uint32_t *count_dev, uint32_t cap_events, int32_t step0, int32_t step1);
 
 /* Run the weight-streaming skinny GEMM of the decode kernel by itself (the kernel behind the QKV,

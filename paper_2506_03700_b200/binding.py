@@ -297,17 +297,20 @@ class Session:
         _ck(load().ada_debug_set_launch_steps(self.h, steps), "ada_debug_set_launch_steps")
 
     def trace(self, cap_events: int, step0: int, step1: int):
-        """Record the persistent kernel's events of steps [step0, step1) of every following launch."""
+        """Record the persistent kernel's events of steps [step0, step1) of every following launch
+        (`cap_events` per CTA)."""
         import torch
-        self._trace = torch.zeros(cap_events, 2, dtype=torch.int64, device="cuda")
-        self._trace_n = torch.zeros(1, dtype=torch.int32, device="cuda")
+        sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+        self._trace = torch.zeros(sms, cap_events, 2, dtype=torch.int64, device="cuda")
+        self._trace_n = torch.zeros(sms, dtype=torch.int32, device="cuda")
         _ck(load().ada_debug_trace(self.h, self._trace.data_ptr(), self._trace_n.data_ptr(), cap_events, step0, step1),
             "ada_debug_trace")
 
     def traced(self) -> np.ndarray:
         """Rows (ns, cta, arg, event) of the recorded events, in time order."""
-        n = min(int(self._trace_n.item()), self._trace.shape[0])
-        t = self._trace[:n].cpu().numpy()
+        n = self._trace_n.cpu().numpy()
+        t = self._trace.cpu().numpy()
+        t = np.concatenate([t[i, :min(int(n[i]), t.shape[1])] for i in range(t.shape[0])], axis=0)
         code = t[:, 1]
         out = np.stack([t[:, 0], code >> 32, (code >> 8) & 0xffff, code & 0xff], axis=1)
         return out[np.argsort(out[:, 0], kind="stable")]

@@ -26,6 +26,7 @@ k_gemm_probe(const CUtensorMap *__restrict__ W, int N, int K, int mode, const ui
     st::Gemm g;
     g.W = W; g.X = X; g.N = N; g.K = K; g.pair = mode == 1 ? 2 : 1; g.half = mode == 1 ? N / 2 : 0;
     g.ctas = st::balanced_ctas(g.tiles(), gridDim.x);
+    g.cp0 = 0; g.ncp = (cols + 1) / 2;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x, G = gridDim.x;
     st::Rings r{0, 0};

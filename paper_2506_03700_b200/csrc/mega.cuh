@@ -590,21 +590,25 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 const int id = lane >> 3;
                 const int pl = 16 * qr + (lane & 7) + 8 * (id >> 1);
                 const unsigned char *krow = kb + pl * (HD * 2);
-                uint4 qh[KSQ], ql[KSQ];
-                uint32_t kf[KSQ][4];
 #pragma unroll
-                for (int ks = 0; ks < KSQ; ++ks) {
-                    qh[ks] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][0]);
-                    ql[ks] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][4]);
-                    ldmatrix_x4(kf[ks], krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
-                }
+                for (int k0 = 0; k0 < KSQ; k0 += 4) {   // four k-steps of loads in flight, then their multiply-adds
+                    uint4 qh[4], ql[4];
+                    uint32_t kf[4][4];
 #pragma unroll
-                for (int ks = 0; ks < KSQ; ++ks) {
-                    const uint32_t ah[4] = {qh[ks].x, qh[ks].y, qh[ks].z, qh[ks].w}, al[4] = {ql[ks].x, ql[ks].y, ql[ks].z, ql[ks].w};
-                    mma16816(sh[0], ah, kf[ks][0], kf[ks][1]);
-                    mma16816(sh[1], ah, kf[ks][2], kf[ks][3]);
-                    mma16816(sl[0], al, kf[ks][0], kf[ks][1]);
-                    mma16816(sl[1], al, kf[ks][2], kf[ks][3]);
+                    for (int u = 0; u < 4; ++u) {
+                        const int ks = k0 + u;
+                        qh[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][0]);
+                        ql[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][4]);
+                        ldmatrix_x4(kf[u], krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t ah[4] = {qh[u].x, qh[u].y, qh[u].z, qh[u].w}, al[4] = {ql[u].x, ql[u].y, ql[u].z, ql[u].w};
+                        mma16816(sh[0], ah, kf[u][0], kf[u][1]);
+                        mma16816(sh[1], ah, kf[u][2], kf[u][3]);
+                        mma16816(sl[0], al, kf[u][0], kf[u][1]);
+                        mma16816(sl[1], al, kf[u][2], kf[u][3]);
+                    }
                 }
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt)
@@ -665,15 +669,19 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 const int id = lane >> 3;
                 const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
                 const unsigned char *vrow = vb + pl * (HD * 2);
-                uint32_t vf[NT / 2][4];
 #pragma unroll
-                for (int np = 0; np < NT / 2; ++np) ldmatrix_x4_trans(vf[np], vrow + ((((2 * np) | (id >> 1)) ^ (pl & 7)) << 4));
+                for (int n0 = 0; n0 < NT / 2; n0 += 4) {
+                    uint32_t vf[4][4];
 #pragma unroll
-                for (int np = 0; np < NT / 2; ++np) {
-                    mma16816(o[2 * np], ph, vf[np][0], vf[np][1]);
-                    mma16816(o[2 * np + 1], ph, vf[np][2], vf[np][3]);
-                    mma16816(o[2 * np], plo, vf[np][0], vf[np][1]);
-                    mma16816(o[2 * np + 1], plo, vf[np][2], vf[np][3]);
+                    for (int u = 0; u < 4; ++u) ldmatrix_x4_trans(vf[u], vrow + ((((2 * (n0 + u)) | (id >> 1)) ^ (pl & 7)) << 4));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int np = n0 + u;
+                        mma16816(o[2 * np], ph, vf[u][0], vf[u][1]);
+                        mma16816(o[2 * np + 1], ph, vf[u][2], vf[u][3]);
+                        mma16816(o[2 * np], plo, vf[u][0], vf[u][1]);
+                        mma16816(o[2 * np + 1], plo, vf[u][2], vf[u][3]);
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->x_empty[slot]);
@@ -842,7 +850,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     };
     // head over E* with the fused (max, sum exp, argmax) reduction; X = final-normed residual (or T output)
     auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols) {
-        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head;
+        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head; g.columns(cols ? cols : 1u << d.newest);
         x_ready();
         if (ROLE == 2) {
             if (ssq) compute_rstd(sm, ssq, ntd, d_model, c.eps);
@@ -913,7 +921,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             const unsigned mask = active_mask(d, l);
             // ---- QKV
             {
-                Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_qkv;
+                Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_qkv; g.columns(mask);
                 x_ready();
                 if (ROLE == 2) {
                     compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);
@@ -935,7 +943,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             phase_barrier(4);
             // ---- O projection + residual; prepares the FFN input
             {
-                Gemm g; g.W = ly.wo; g.X = reinterpret_cast<const uint4 *>(A.XO); g.N = d_model; g.K = qd; g.pair = 1; g.half = 0; g.ctas = n_d;
+                Gemm g; g.W = ly.wo; g.X = reinterpret_cast<const uint4 *>(A.XO); g.N = d_model; g.K = qd; g.pair = 1; g.half = 0; g.ctas = n_d; g.columns(mask);
                 x_ready();
                 if (ROLE == 2) {
                     const __nv_bfloat16 *gain = ly.ffn_norm;
@@ -973,7 +981,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             }
             // ---- gate / up + SwiGLU
             {
-                Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff; g.ctas = n_gu;
+                Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff; g.ctas = n_gu; g.columns(mask);
                 x_ready();
                 if (ROLE == 2) {
                     compute_rstd(sm, A.ssq_b, ntd, d_model, c.eps);
@@ -995,7 +1003,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             }
             // ---- down projection + residual; prepares the next layer's (and the head's) input
             {
-                Gemm g; g.W = ly.wdown; g.X = reinterpret_cast<const uint4 *>(A.XH); g.N = d_model; g.K = c.dff; g.pair = 1; g.half = 0; g.ctas = n_d;
+                Gemm g; g.W = ly.wdown; g.X = reinterpret_cast<const uint4 *>(A.XH); g.N = d_model; g.K = c.dff; g.pair = 1; g.half = 0; g.ctas = n_d; g.columns(mask);
                 x_ready();
                 if (ROLE == 2) {
                     const __nv_bfloat16 *gain_next = l + 1 < L ? M.layer[l + 1].attn_norm : nullptr;
@@ -1038,7 +1046,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             if (l + 1 < L && A.exit_at[l + 1] != 0 && d.head_ok) {
                 const MegaLayer &hl = M.layer[l + 1];
                 if (hl.wT) {
-                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_d;
+                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_d; g.columns(1u << d.newest);
                     x_ready();
                     if (ROLE == 2) {
                         compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);

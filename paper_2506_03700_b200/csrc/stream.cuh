@@ -31,7 +31,7 @@ constexpr int KSTEPS = KC / 16;                  // mma k-steps per stage
 constexpr int TILE_N = 16;                       // weight rows per stage (mma M)
 constexpr int KG = KC / 64;                      // 64-element (128-byte) k groups per stage
 constexpr int W_STAGE = TILE_N * KC * 2;         // 16384: [k group][row][128 B, 16-byte chunks xor-swizzled by row%8]
-constexpr int X_STAGE = KSTEPS * 32 * 16;        // 16384: [k-step][lane][b0.hi b1.hi b0.lo b1.lo]
+constexpr int X_STAGE = KSTEPS * 32 * 16;        // 16384: [column pair][k-step][8 slots][b0.hi b1.hi b0.lo b1.lo]
 constexpr int NW = 9;                            // weight stages in flight per CTA
 constexpr int NX = 3;                            // activation stages
 constexpr int CONS_WARPS = 8;
@@ -52,6 +52,7 @@ struct Smem {                                    // must start on a 1024-byte bo
     alignas(8) unsigned long long w_full[NW], w_empty[NW], x_full[NX], x_empty[NX];
     int abort;
     int bcast[8];
+    unsigned trace_n;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -143,10 +144,12 @@ __device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
 // ---------------------------------------------------------------- bounded waits
 
 // Optional event trace (test hook): records (globaltimer ns, code) pairs while `tr_on` is set.
+// Every CTA writes its own region of the buffer, so that recording costs a shared-memory counter
+// and one store.
 struct Trace {
-    unsigned long long *buf;   // [cap][2], or nullptr
-    unsigned *count;
-    unsigned cap;
+    unsigned long long *buf;   // [grid][cap][2], or nullptr
+    unsigned *count;           // [grid]
+    unsigned cap;              // events per CTA
 };
 
 struct Shared {            // what every role needs to wait safely
@@ -161,10 +164,12 @@ constexpr int EV_PHASE_BEGIN = 1, EV_X0 = 2, EV_W0 = 3, EV_MAIN_END = 4, EV_EPI_
 
 __device__ __forceinline__ void trace(const Shared &S, int ev, int arg) {
     if (S.tr_on && S.tr.buf) {
-        const unsigned i = atomicAdd(S.tr.count, 1u);
+        const unsigned i = atomicAdd(&S.sm->trace_n, 1u);
         if (i < S.tr.cap) {
-            S.tr.buf[2 * (size_t)i] = gtime();
-            S.tr.buf[2 * (size_t)i + 1] = ((unsigned long long)blockIdx.x << 32) | ((unsigned long long)(arg & 0xffff) << 8) | (unsigned)ev;
+            unsigned long long *e = S.tr.buf + 2 * ((size_t)blockIdx.x * S.tr.cap + i);
+            e[0] = gtime();
+            e[1] = ((unsigned long long)blockIdx.x << 32) | ((unsigned long long)(arg & 0xffff) << 8) | (unsigned)ev;
+            S.tr.count[blockIdx.x] = i + 1;
         }
     }
 }
@@ -217,13 +222,18 @@ __device__ __forceinline__ void grid_wait(const Shared &S, const unsigned *ctr, 
 
 // ---------------------------------------------------------------- activation layout
 
-// Activations for a GEMM of depth K live in global memory as ceil(K/KC) blocks of X_STAGE bytes;
-// block c, k-step s, lane l holds 16 bytes: the mma B fragment (b0, b1) of the bf16 high parts,
-// then of the bf16 low parts, for token column l/4 and k = 16 s + 2 (l%4) + {0,1} (+8 for b1).
+// Activations for a GEMM of depth K live in global memory as ceil(K/KC) blocks of X_STAGE bytes.
+// A block holds four sub-blocks of 4 KB, one per pair of token columns; in sub-block p, k-step s,
+// slot j (0..7) holds 16 bytes: the mma B fragment (b0, b1) of the bf16 high parts, then of the
+// bf16 low parts, for token column 2 p + j/4 and k = 16 s + 2 (j%4) + {0,1} (+8 for b1).  Lane l of
+// a warp reads slot l%8 of sub-block l/8.  A pass that carries few tokens fetches only the
+// sub-blocks of the column pairs in use: activations go through the same copy engine as the
+// weights, and for a CTA holding two weight tiles a full block per chunk would be half as many
+// bytes again as the weights.
 __device__ __forceinline__ size_t xfrag_index(int k, int col) {   // index in 2-byte units of the high part
     const int chunk = k / KC, ks = (k % KC) >> 4, kk = k & 15;
-    const int lane = col * 4 + ((kk & 7) >> 1);
-    return ((((size_t)chunk * KSTEPS + ks) * 32 + lane) << 3) + ((kk >> 3) << 1) + (kk & 1);
+    const int slot = (col & 1) * 4 + ((kk & 7) >> 1);
+    return (((((size_t)chunk * 4 + (col >> 1)) * KSTEPS + ks) * 8 + slot) << 3) + ((kk >> 3) << 1) + (kk & 1);
 }
 __device__ __forceinline__ void xfrag_store(__nv_bfloat16 *X, int k, int col, float v) {
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
@@ -248,6 +258,12 @@ struct Gemm {
     const uint4 *X;
     int N, K, pair, half;
     int ctas;   // CTAs 0 .. ctas-1 share the tiles (see balanced_ctas); 0 = the whole grid
+    int cp0, ncp;   // column pairs cp0 .. cp0+ncp-1 of the activations are fetched
+    __device__ __forceinline__ void columns(unsigned mask) {   // the pairs spanning the columns set in `mask`
+        if (mask == 0) { cp0 = 0; ncp = 1; return; }
+        cp0 = (__ffs(mask) - 1) >> 1;
+        ncp = ((31 - __clz(mask)) >> 1) - cp0 + 1;
+    }
     __device__ __forceinline__ int tiles() const { return pair == 2 ? half / TILE_N : (N + TILE_N - 1) / TILE_N; }
 };
 
@@ -309,13 +325,13 @@ __device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, i
     const int nch = (g.K + KC - 1) / KC;
     for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
         for (int kc = 0; kc < nch; ++kc) {
-            const int klen = min(KC, g.K - kc * KC);
             const int slot = r.xi % NX;
             mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
             if (lane == 0 && !aborted(S)) {
-                const uint32_t bytes = (uint32_t)(klen / 16) * 512u;
+                const uint32_t bytes = (uint32_t)g.ncp * 4096u;
                 mbar_expect_tx(&sm->x_full[slot], bytes);
-                bulk_g2s(sm->x[slot], reinterpret_cast<const unsigned char *>(g.X) + (size_t)kc * X_STAGE, bytes, &sm->x_full[slot], pol);
+                bulk_g2s(sm->x[slot] + g.cp0 * 4096, reinterpret_cast<const unsigned char *>(g.X) + (size_t)kc * X_STAGE + g.cp0 * 4096, bytes,
+                         &sm->x_full[slot], pol);
             }
             ++r.xi;
         }
@@ -335,7 +351,7 @@ __device__ __forceinline__ void stage_full(float (&acc)[4][4], const unsigned ch
     for (int j = 0; j < PF; ++j) {
         const int ks = ks_id + KS_ * j;
         ldmatrix_x4(a[j], ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
-        b[j] = xs[ks * 32];
+        b[j] = xs[ks * 8];
     }
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
@@ -345,7 +361,7 @@ __device__ __forceinline__ void stage_full(float (&acc)[4][4], const unsigned ch
         if (j + PF < NJ) {
             const int ks = ks_id + KS_ * (j + PF);
             ldmatrix_x4(a[cur], ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
-            b[cur] = xs[ks * 32];
+            b[cur] = xs[ks * 8];
         }
     }
 }
@@ -386,7 +402,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
             const int xslot = r.xi % NX;
             mbar_wait(S, &sm->x_full[xslot], (r.xi / NX) & 1);
             if (threadIdx.x == 0 && kc == 0 && g0 == t0) trace(S, EV_X0, 0);
-            const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + lane;
+            const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + (lane >> 3) * 256 + (lane & 7);
             for (int s = 0; s < ng; ++s) {
 #pragma unroll
                 for (int p = 0; p < PAIR; ++p) {
@@ -407,7 +423,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                             for (int ks = ks_id; ks < ksteps; ks += KS) {
                                 uint32_t a[4];
                                 ldmatrix_x4(a, ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
-                                const uint4 b = xs[ks * 32];
+                                const uint4 b = xs[ks * 8];
                                 if (par == 0) { mma16816(acc[p][0], a, b.x, b.y); mma16816(acc[p][2], a, b.z, b.w); }
                                 else { mma16816(acc[p][1], a, b.x, b.y); mma16816(acc[p][3], a, b.z, b.w); }
                                 par ^= 1;
@@ -475,6 +491,7 @@ __device__ __forceinline__ void smem_init(Smem *sm) {
         for (int i = 0; i < NW; ++i) { mbar_init(&sm->w_full[i], 1); mbar_init(&sm->w_empty[i], CONS_WARPS); }
         for (int i = 0; i < NX; ++i) { mbar_init(&sm->x_full[i], 1); mbar_init(&sm->x_empty[i], CONS_WARPS); }
         sm->abort = 0;
+        sm->trace_n = 0;
         fence_mbar_init();
         fence_proxy_async();
     }
