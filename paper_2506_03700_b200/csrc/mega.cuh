@@ -515,7 +515,6 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
 #pragma unroll
             for (int u = 0; u < VPT; ++u) nv[u] = __float2bfloat16_rn(vx[u]);
         }
-        if (tid == 0) trace(S, 15, 0);
         bar_consumers();   // the previous item is done with the shared buffers
         // ---- rotated, scaled queries -> A fragments (hi / lo)
 #pragma unroll
@@ -545,6 +544,13 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = qcol / group;
             lim[rh] = (cc < MAX_COLS && ((mask >> cc) & 1u)) ? d.pos[cc] : -1;
         }
+        // a query tile none of whose 16 (column, q head) pairs is in use does no arithmetic (uniform per warp)
+        bool tile_used = false;
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int cc = (mt * 16 + q) / group;
+            tile_used = tile_used || (cc < MAX_COLS && ((mask >> cc) & 1u));
+        }
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
         float o[NT][4];
 #pragma unroll
@@ -561,9 +567,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             float s[2][4];
             {   // ---- K block
                 const int slot = r.xi % NX;
-                if (tid == 0) trace(S, 11, sb);
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
-                if (tid == 0) trace(S, 12, sb);
                 unsigned char *kb = sm->x[slot];
                 if (newm) {
                     const size_t blk = ((((size_t)page * c.L + layer) * 2 + 0) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
@@ -590,6 +594,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 const int id = lane >> 3;
                 const int pl = 16 * qr + (lane & 7) + 8 * (id >> 1);
                 const unsigned char *krow = kb + pl * (HD * 2);
+                if (tile_used)
 #pragma unroll
                 for (int k0 = 0; k0 < KSQ; k0 += 4) {   // four k-steps of loads in flight, then their multiply-adds
                     uint4 qh[4], ql[4];
@@ -648,9 +653,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             }
             {   // ---- V block
                 const int slot = r.xi % NX;
-                if (tid == 0) trace(S, 13, sb);
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
-                if (tid == 0) trace(S, 14, sb);
                 unsigned char *vb = sm->x[slot];
                 if (newm) {
                     const size_t blk = ((((size_t)page * c.L + layer) * 2 + 1) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
@@ -669,6 +672,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 const int id = lane >> 3;
                 const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
                 const unsigned char *vrow = vb + pl * (HD * 2);
+                if (tile_used)
 #pragma unroll
                 for (int n0 = 0; n0 < NT / 2; n0 += 4) {
                     uint32_t vf[4][4];
@@ -688,7 +692,6 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 ++r.xi;
             }
         }
-        if (tid == 0) trace(S, 16, 0);
         // ---- row sums over the quad, then merge the four position quarters of each query tile:
         //      (q0 + q1) and (q2 + q3), then the two halves
 #pragma unroll

@@ -68,6 +68,9 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(bar)) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_n(unsigned long long *bar, uint32_t n) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(s32(bar)), "r"(n) : "memory");
+}
 __device__ __forceinline__ bool mbar_try(unsigned long long *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -274,20 +277,11 @@ __device__ __forceinline__ void cta_tile_range(int T, int cta, int G, int &t0, i
     t0 = (int)((long long)T * cta / G);
     t1 = (int)((long long)T * (cta + 1) / G);
 }
-// How many CTAs should share T equal tiles.  One SM's TMA unit moves at most about 58 GB/s of
-// 16 KB boxes, 1.3 times its fair share of HBM, so a CTA holding one tile more than the others
-// cannot catch up and everybody waits for it at the phase barrier.  About three quarters of the
-// SMs already saturate HBM, so the count in [0.76 G, G] that wastes the fewest tile slots
-// (ceil(T / g) g - T) is used; the idle CTAs prefetch the next phase meanwhile.
-__host__ __device__ inline int balanced_ctas(int T, int G) {
-    int lo = (G * 76 + 99) / 100, best = G;
-    long long best_waste = -1;
-    for (int g = G; g >= lo && g >= 1; --g) {
-        const long long waste = (long long)((T + g - 1) / g) * g - T;
-        if (best_waste < 0 || waste < best_waste) { best_waste = waste; best = g; }
-    }
-    return best;
-}
+// How many CTAs share the tiles of a GEMM: all of them.  (With its consumers attached one SM
+// sustains about 45 GB/s through the ring, roughly its fair share of HBM with all 148 SMs
+// streaming; giving equal tile counts to fewer CTAs was measured and lost more than the uneven
+// split costs.)
+__host__ __device__ inline int balanced_ctas(int T, int G) { (void)T; return G; }
 
 // Weight producer warp: streams this CTA's tiles of the GEMM through the weight ring.
 __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol) {
@@ -407,9 +401,9 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
 #pragma unroll
                 for (int p = 0; p < PAIR; ++p) {
                     const int wslot = r.wi % NW;
-                    mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
-                    if (threadIdx.x == 0 && kc == 0 && g0 == t0 && s == 0 && p == 0) trace(S, EV_W0, 0);
-                    if (s == slot_id) {
+                    if (s == slot_id) {   // only the warps that multiply a stage wait for it and release it
+                        mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
+                        if (threadIdx.x == 0 && kc == 0 && g0 == t0 && p == 0) trace(S, EV_W0, 0);
                         const unsigned char *ws = sm->w[wslot] + a_off;
                         if (ksteps == KSTEPS) {   // full chunk: software-pipelined, fully unrolled per k-split
                             switch (KS) {
@@ -429,9 +423,9 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                                 par ^= 1;
                             }
                         }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_n(&sm->w_empty[wslot], (uint32_t)TS);   // KS owners x TS = 8 arrivals
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->w_empty[wslot]);
                     ++r.wi;
                 }
             }
