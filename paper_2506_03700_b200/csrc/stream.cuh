@@ -267,6 +267,10 @@ struct Gemm {
         cp0 = (__ffs(mask) - 1) >> 1;
         ncp = ((31 - __clz(mask)) >> 1) - cp0 + 1;
     }
+    // k chunks whose activations share one 16 KB stage: 4 for one column pair, 2 for two, else 1.  (The
+    // ring holds three stages; with one chunk per stage a CTA that owns two weight tiles would wait
+    // for an activation copy every 96 KB of weights.)
+    __device__ __forceinline__ int xchunks() const { return ncp == 1 ? 4 : ncp == 2 ? 2 : 1; }
     __device__ __forceinline__ int tiles() const { return pair == 2 ? half / TILE_N : (N + TILE_N - 1) / TILE_N; }
 };
 
@@ -317,15 +321,18 @@ __device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, i
     int t0, t1;
     cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
     const int nch = (g.K + KC - 1) / KC;
+    const int XC = g.xchunks();
     for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
-        for (int kc = 0; kc < nch; ++kc) {
+        for (int kc = 0; kc < nch; kc += XC) {
+            const int nc = min(XC, nch - kc);
             const int slot = r.xi % NX;
             mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
             if (lane == 0 && !aborted(S)) {
                 const uint32_t bytes = (uint32_t)g.ncp * 4096u;
-                mbar_expect_tx(&sm->x_full[slot], bytes);
-                bulk_g2s(sm->x[slot] + g.cp0 * 4096, reinterpret_cast<const unsigned char *>(g.X) + (size_t)kc * X_STAGE + g.cp0 * 4096, bytes,
-                         &sm->x_full[slot], pol);
+                mbar_expect_tx(&sm->x_full[slot], bytes * nc);
+                for (int q = 0; q < nc; ++q)   // chunk kc+q: column pairs cp0.. at [q][pair - cp0] of the stage
+                    bulk_g2s(sm->x[slot] + q * bytes, reinterpret_cast<const unsigned char *>(g.X) + (size_t)(kc + q) * X_STAGE + g.cp0 * 4096,
+                             bytes, &sm->x_full[slot], pol);
             }
             ++r.xi;
         }
@@ -373,7 +380,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int t0, t1;
     cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
-    const int nch = (g.K + KC - 1) / KC;
+    const int nch = (g.K + KC - 1) / KC, XC = g.xchunks();
     // ldmatrix source of this lane inside a stage: row (lane%8) + 8 ((lane/8)%2), 16-byte chunk lane/16 of the k-step
     const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
     const int a_off = a_row * 128, a_hi = lane >> 4, a_sw = a_row & 7;
@@ -394,15 +401,22 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
         for (int kc = 0; kc < nch; ++kc) {
             const int ksteps = min(KC, g.K - kc * KC) >> 4;
             const int xslot = r.xi % NX;
-            mbar_wait(S, &sm->x_full[xslot], (r.xi / NX) & 1);
+            if (kc % XC == 0) mbar_wait(S, &sm->x_full[xslot], (r.xi / NX) & 1);
             if (threadIdx.x == 0 && kc == 0 && g0 == t0) trace(S, EV_X0, 0);
-            const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + (lane >> 3) * 256 + (lane & 7);
+            // this lane's column pair, if it was fetched (else any fetched pair: its column is not in use)
+            const int xp = min(max((lane >> 3) - g.cp0, 0), g.ncp - 1);
+            const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + ((kc % XC) * g.ncp + xp) * 256 + (lane & 7);
             for (int s = 0; s < ng; ++s) {
 #pragma unroll
                 for (int p = 0; p < PAIR; ++p) {
                     const int wslot = r.wi % NW;
-                    if (s == slot_id) {   // only the warps that multiply a stage wait for it and release it
-                        mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
+                    // Every warp waits for every stage in order, although only its owners use it: an
+                    // mbarrier tells phases apart by one parity bit, so a warp that skipped ahead by
+                    // more than a ring (in a gate/up group a warp's own stages are 14 apart, the ring
+                    // holds 9) would take an older phase of the slot for the one it wants.  Only the
+                    // owners release the stage, so a slot is free as soon as its math is done.
+                    mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
+                    if (s == slot_id) {
                         if (threadIdx.x == 0 && kc == 0 && g0 == t0 && p == 0) trace(S, EV_W0, 0);
                         const unsigned char *ws = sm->w[wslot] + a_off;
                         if (ksteps == KSTEPS) {   // full chunk: software-pipelined, fully unrolled per k-split
@@ -429,9 +443,11 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                     ++r.wi;
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm->x_empty[xslot]);
-            ++r.xi;
+            if (kc % XC == XC - 1 || kc == nch - 1) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->x_empty[xslot]);
+                ++r.xi;
+            }
         }
         if (threadIdx.x == 0 && g0 + CONS_WARPS >= t1) trace(S, EV_MAIN_END, 0);
         // fold the four partial accumulators in a fixed order: (even.hi + odd.hi) + (even.lo + odd.lo)
