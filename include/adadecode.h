@@ -197,6 +197,27 @@ int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const 
                    void *work_dev, size_t work_bytes, float *Y_dev, int32_t ldy, int32_t repeat, void *cuda_stream,
                    float *ms_out);
 
+/* The same streaming GEMM as ada_debug_gemm (modes, shapes and layouts as described there, one
+ * product per call), for callers that have no device memory to lend and must not allocate any.
+ * (The paper has no counterpart to this call; it exists for deployment.)  Think of a serving
+ * process whose framework has already handed every byte of HBM to its KV-cache pool, or of code
+ * running where a device allocation would stall every stream of the process: such a caller can
+ * still pass the weights, the activations and the output, and this call brings its own scratch.
+ *
+ * The scratch (activations re-laid for the tensor cores, an error word, a tensor map) is a fixed
+ * array of 512.5 KB inside the library image; every GPU that loads the library holds it until the
+ * process exits.  It bounds the depth: K <= 16384, larger K returns ADA_ECAPACITY.  The call
+ * performs no cudaMalloc / cudaFree and creates no events.
+ *
+ * The first call on each device looks up the array's device address and configures the kernel;
+ * make that first call outside any stream capture.  All calls on a device share the one array:
+ * it keeps the previous call's contents (the call clears the word that has to start at zero and
+ * rewrites the rest), and two calls whose kernels overlap on the GPU (different streams, or
+ * different host threads) race on it.  The call synchronises `cuda_stream` before returning.
+ * W_dev, X_dev, Y_dev are device pointers as in ada_debug_gemm. */
+int ada_gemm_noalloc(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols, float *Y_dev,
+                     int32_t ldy, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,7 @@ EXPORTS = [
     "ada_session_create", "ada_session_destroy", "ada_session_reset", "ada_prefill", "ada_plain_decode",
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
-    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace",
+    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace", "ada_gemm_noalloc",
 ]
 
 
@@ -105,6 +105,7 @@ def load() -> C.CDLL:
         L.ada_debug_get_path.argtypes = [vp, C.POINTER(i32)]
         L.ada_debug_set_launch_steps.argtypes = [vp, i32]
         L.ada_debug_trace.argtypes = [vp, vp, vp, C.c_uint32, i32, i32]
+        L.ada_gemm_noalloc.argtypes = [vp, i32, i32, i32, vp, i32, vp, i32, vp]
         L.ada_debug_profile.argtypes = [vp, i32]
         L.ada_debug_profile_read.argtypes = [vp, vp, vp, vp]
         L.ada_debug_gemm_work_bytes.restype = sz
@@ -137,6 +138,17 @@ def debug_gemm(W, X, mode: int = 0, repeat: int = 1):
     _ck(lib.ada_debug_gemm(W.data_ptr(), N, K, mode, X.data_ptr(), cols, work.data_ptr() + off, wb, Y.data_ptr(), n_out,
                            repeat, torch.cuda.current_stream().cuda_stream, C.byref(ms)), "ada_debug_gemm")
     return Y, ms.value
+
+
+def gemm_noalloc(W, X, Y, mode: int = 0):
+    """ada_gemm_noalloc: the streaming GEMM with the library's built-in scratch.  W bf16 [N, K], X
+    fp32 [cols, K], Y fp32 [cols, N or N/2], all on the current CUDA device; Y is written in place.
+    Nothing is allocated here or in the library."""
+    import torch
+    N, K = W.shape
+    _ck(load().ada_gemm_noalloc(W.data_ptr(), N, K, mode, X.data_ptr(), X.shape[0], Y.data_ptr(), Y.shape[1],
+                                torch.cuda.current_stream().cuda_stream), "ada_gemm_noalloc")
+    return Y
 
 
 class Model:

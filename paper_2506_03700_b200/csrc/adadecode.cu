@@ -1107,4 +1107,56 @@ int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const 
     return herr ? ADA_ETIMEOUT : ADA_OK;
 }
 
+// ---- streaming GEMM without caller scratch ---------------------------------------------------------
+
+#define ADA_NOALLOC_MAX_K 16384
+// Fragment-layout activations for K <= ADA_NOALLOC_MAX_K, then the error word (at +0) and the tensor
+// map (at +256) in a 512-byte tail.  Lives in every GPU context that loads this library.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[(ADA_NOALLOC_MAX_K / st::KC) * st::X_STAGE + 512];
+
+int ada_gemm_noalloc(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols, float *Y_dev,
+                     int32_t ldy, void *cuda_stream) {
+    if (!W_dev || !X_dev || !Y_dev || N < 1 || K < 64 || K % 64 || cols < 1 || cols > st::MAX_COLS) return ADA_EINVAL;
+    if (mode < 0 || mode > 1) return ADA_EINVAL;
+    if (mode == 1 && (N % 2 || (N / 2) % 16)) return ADA_EINVAL;
+    if ((uintptr_t)W_dev % 16 || ldy < (mode == 1 ? N / 2 : N)) return ADA_EINVAL;
+    if (K > ADA_NOALLOC_MAX_K) {
+        g_cuda_err = "ada_gemm_noalloc: K exceeds the built-in scratch (ADA_NOALLOC_MAX_K = 16384)";
+        return ADA_ECAPACITY;
+    }
+    // Once per device: the address of the scratch array in that device's memory.  The array's name
+    // in host code is only a handle; kernels must be given the address looked up here.
+    static unsigned char *scratch_of_device[64] = {nullptr};
+    static int sms_of_device[64] = {0};
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ADA_EUNSUPPORTED;
+    if (!scratch_of_device[dev]) {
+        unsigned char *ptr = nullptr;
+        CK(cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch));
+        CK(cudaDeviceGetAttribute(&sms_of_device[dev], cudaDevAttrMultiProcessorCount, dev));
+        CK(cudaFuncSetAttribute(k_gemm_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st::SMEM_BYTES));
+        scratch_of_device[dev] = ptr;
+    }
+    unsigned char *base = scratch_of_device[dev];
+    const size_t xb = st::xfrag_bytes(K);
+    int *err = (int *)(base + xb);
+    CUtensorMap *dmap = (CUtensorMap *)(base + xb + 256);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    CUtensorMap hmap;
+    int rc = make_weight_map(&hmap, W_dev, N, K);
+    if (rc) return rc;
+    CK(cudaMemsetAsync(err, 0, sizeof(int), stream));   // the one word that must start at zero
+    CK(cudaMemcpyAsync(dmap, &hmap, sizeof(hmap), cudaMemcpyHostToDevice, stream));
+    CK(cudaStreamSynchronize(stream));   // hmap lives on this stack frame
+    k_xfrag_pack<<<(K + 255) / 256, 256, 0, stream>>>(X_dev, K, cols, (__nv_bfloat16 *)base);
+    CK(cudaGetLastError());
+    k_gemm_probe<<<sms_of_device[dev], st::THREADS, st::SMEM_BYTES, stream>>>(dmap, N, K, mode, (const uint4 *)base, Y_dev, ldy, cols, 1, err);
+    CK(cudaGetLastError());
+    int herr = 0;
+    CK(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    CK(cudaStreamSynchronize(stream));
+    return herr ? ADA_ETIMEOUT : ADA_OK;
+}
+
 }  // extern "C"
