@@ -256,9 +256,45 @@ def run_ours(args):
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(cfg, w, args.cpu_tokens)
+    if not args.no_regime and world == 1 and args.workload == "8b":
+        del sess, model, w
+        torch.cuda.empty_cache()
+        line["confident_head_regime"] = confident_regime(cfg, args.regime_scale, args.regime_tokens)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def confident_regime(cfg, scale: float, n_tok: int) -> dict:
+    """Supplementary measurement.  With the configured o_proj/down_proj scale (0.2) and d_model 4096 the
+    random layers swamp the embedding, and an untrained head at layer 16 almost never agrees with the
+    final argmax (the paper's "original LM head" ablation).  Scaling those projections by `scale`
+    instead makes the intermediate heads predictive, as the paper's trained heads are (about 80 %
+    early exits, a few % rejected): same shape, same kernels, same byte counts per layer, measured
+    the same way on a shorter generation."""
+    import dataclasses
+    from paper_2506_03700_b200 import binding, synth
+    c2 = dataclasses.replace(cfg, resid_scale=scale)
+    w = synth.make_weights(c2, seed=1234, device="cuda")
+    model = binding.Model(c2, w)
+    for l in c2.exit_layers:
+        model.set_exit_head(l, None, c2.logit_scale)
+    prompt = synth.make_prompt(c2, seed=5678).numpy()
+    sess = binding.Session(model, 1, c2.prompt_len + n_tok + 16, 64, 5)
+    sess.prefill(prompt)
+    sess.plain_decode(8)
+    sess.prefill(prompt)
+    ps = binding.Stats()
+    pt = sess.plain_decode(n_tok, ps)[0]
+    sess.prefill(prompt)
+    st = binding.Stats()
+    at = sess.adaptive_decode(n_tok, c2.threshold, c2.exit_layers, 5, st)[0]
+    return {"o_down_scale": scale, "tokens": n_tok, "plain_tokens_per_s": n_tok / (ps.decode_ms * 1e-3),
+            "adaptive_tokens_per_s": n_tok / (st.decode_ms * 1e-3), "speedup_vs_plain": ps.decode_ms / st.decode_ms,
+            "adaptive_equals_plain": bool(np.array_equal(at, pt)), "distinct_tokens": len(set(pt.tolist())),
+            "early_exit_rate": st.early_exits / max(1, st.steps),
+            "rejection_rate": st.rejected / max(1, st.accepted + st.rejected),
+            "exits_at_layer": st.as_dict()["exits_at_layer"]}
 
 
 def cpu_baseline(cfg, w, n_tok: int, n_prompt: int = 16) -> dict:
@@ -325,6 +361,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=12)
     ap.add_argument("--ref-tokens", type=int, default=2)
+    ap.add_argument("--no-regime", action="store_true", help="skip the supplementary confident-head measurement")
+    ap.add_argument("--regime-scale", type=float, default=0.02)
+    ap.add_argument("--regime-tokens", type=int, default=512)
     ap.add_argument("--plain-only", action="store_true", help="time plain greedy decoding only (profiling runs)")
     ap.add_argument("--gen-len", type=int, default=0, help="generate this many tokens instead of the workload's (profiling runs)")
     ap.add_argument("--launch-steps", type=int, default=0, help="decode steps per launch of the persistent kernel (profiling runs)")

@@ -294,20 +294,27 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
         const int tokid = min(max(c.tokens[pos], 0), c.vocab - 1);
         const __nv_bfloat16 *erow = M.tok_embed + (size_t)tokid * c.d;
         const __nv_bfloat16 *g0 = M.layer[0].attn_norm;
-        for (int n0 = 0; n0 < c.d; n0 += CONS_THREADS) {
-            const int n = n0 + tid;
-            float v = 0.f;
-            if (n < c.d) {
-                v = __bfloat162float(erow[n]);
-                c.resid[(size_t)col * c.d + n] = v;
-                xfrag_store(A.XA, n, col, v * __bfloat162float(g0[n]));
+        for (int n0 = 0; n0 < c.d; n0 += 8 * CONS_THREADS) {   // eight loads of the embedding row in flight per thread
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int n = n0 + u * CONS_THREADS + tid;
+                v[u] = n < c.d ? __bfloat162float(erow[n]) * 1.0f : 0.f;
             }
-            float q = v * v;
-            q += __shfl_xor_sync(0xffffffffu, q, 1);
-            q += __shfl_xor_sync(0xffffffffu, q, 2);
-            q += __shfl_xor_sync(0xffffffffu, q, 4);
-            q += __shfl_xor_sync(0xffffffffu, q, 8);
-            if ((tid & 15) == 0 && n < c.d) A.ssq_a[(size_t)(n >> 4) * MAX_COLS + col] = q;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int n = n0 + u * CONS_THREADS + tid;
+                if (n < c.d) {
+                    c.resid[(size_t)col * c.d + n] = v[u];
+                    xfrag_store(A.XA, n, col, v[u] * __bfloat162float(g0[n]));
+                }
+                float q = v[u] * v[u];
+                q += __shfl_xor_sync(0xffffffffu, q, 1);
+                q += __shfl_xor_sync(0xffffffffu, q, 2);
+                q += __shfl_xor_sync(0xffffffffu, q, 4);
+                q += __shfl_xor_sync(0xffffffffu, q, 8);
+                if ((tid & 15) == 0 && n < c.d) A.ssq_a[(size_t)(n >> 4) * MAX_COLS + col] = q;
+            }
         }
         const int half = c.hd / 2;
         for (int i = tid; i < half; i += CONS_THREADS) {
