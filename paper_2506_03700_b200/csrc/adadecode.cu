@@ -908,6 +908,17 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
         int32_t zero = 0;
         CK(cudaMemcpyAsync(&S->c.st->capture_n, &zero, sizeof(int32_t), cudaMemcpyHostToDevice, S->stream));
     }
+    if (S->mega && S->path == 1) {
+        // prompt passes of eight positions through the persistent kernel
+        mg::k_prefill_arm<<<1, 32, 0, S->stream>>>(S->c, n_prompt);
+        CK(cudaGetLastError());
+        if ((rc = run_persistent(S, nullptr, 0, true))) return rc;
+        S->prefilled[seq] = 1;
+        S->h_prompt[seq] = n_prompt;
+        S->h_len[seq] = n_prompt + 1;
+        S->h_reported[seq] = 0;
+        return ADA_OK;
+    }
     const int chunk = std::min(S->rows_alloc, kMaxRows);
     for (int p0 = 0; p0 < n_prompt; p0 += chunk) {
         const int n = std::min(chunk, n_prompt - p0);

@@ -51,6 +51,8 @@ struct DevState {
     int32_t head_log_n;
     int32_t capture_cap, capture_n;     // final-logit capture (sequence 0)
     int32_t keep_rows;                  // rows of sequence 0 whose logits the last verification kept
+    int32_t keep_row0;                  // first of those rows in the logits staging buffer
+    int32_t pf_pos, pf_end;             // persistent-kernel prefill: next prompt position, prompt length (0: not prefilling)
     DevStats st;
 };
 

@@ -38,6 +38,8 @@ struct StepDesc {
     int newest;                // column of the newest token
     int head_ok;               // the newest token may consult intermediate heads in this step
     int pmax;                  // position of the newest token
+    int fresh;                 // columns whose token enters at layer 1 in this step (their embedding is set up by the control point)
+    int run_final;             // the step ends with the final head (0: a prompt pass that is not the last)
     int first_layer[MAX_COLS]; // 0-based layer at which the column resumes (INT_MAX: no token)
     int pos[MAX_COLS];
 };
@@ -46,7 +48,7 @@ struct Pub {                   // what CTA 0 publishes at a control point
     unsigned seq;
     int action;
     StepDesc d;
-    int pad[10];
+    int pad[8];
 };
 
 struct MegaLayer {
@@ -207,7 +209,26 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
                 st->st.layer_passes += e;
             }
         }
-        if (action != ACT_STOP && kind == CTRL_TOP) {
+        const bool prefilling = st->pf_end > 0;
+        if (action != ACT_STOP && kind == CTRL_TOP && prefilling) {
+            // a pass over prompt positions [pf_pos, pf_pos + n) is complete at every layer
+            const int n = dprev.n_cols, end = st->pf_pos + n;
+            for (int l = 0; l < c.L; ++l) c.fill[l] = end;
+            st->pf_pos = end;
+            if (end >= st->pf_end) {   // KV cache <- LM(x) done: the full-depth argmax at the last prompt token is the first generated token
+                const int np = st->pf_end;
+                tok[np] = min(max(c.head_res[n - 1].token, 0), c.vocab - 1);
+                st->len[0] = np + 1;
+                st->base[0] = np;
+                st->n_prompt[0] = np;
+                st->done[0] = 1;
+                st->pf_end = 0;
+                st->keep_rows = 1;
+                st->keep_row0 = n - 1;
+                verified = 1;
+            }
+        }
+        if (action != ACT_STOP && kind == CTRL_TOP && !prefilling) {
             const int len = st->len[0], base = st->base[0], nrow = len - base;
             for (int l = 0; l < c.L; ++l) st->st.row_layers += len - c.fill[l];
             int bad = -1;
@@ -241,19 +262,40 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
             st->st.layer_passes += c.L;
             if (new_len >= st->target_len[0]) st->done[0] = 1;
             st->keep_rows = keep;
+            st->keep_row0 = 0;
             verified = 1;
         }
         if (action == ACT_NEWSTEP) {
             if (st->done[0]) { action = ACT_STOP; st->n_done = 1; }
             else if (steps_started >= A.step_budget) action = ACT_STOP;
         }
-        if (action == ACT_NEWSTEP) {
+        if (action == ACT_NEWSTEP && st->pf_end > 0) {   // next pass over the prompt: up to eight positions, all from layer 1
+            ++steps_started;
+            StepDesc nd;
+            nd.n_cols = min(MAX_COLS, st->pf_end - st->pf_pos);
+            nd.newest = nd.n_cols - 1;
+            nd.pmax = st->pf_pos + nd.n_cols - 1;
+            nd.head_ok = 0;
+            nd.fresh = (1 << nd.n_cols) - 1;
+            nd.run_final = st->pf_pos + nd.n_cols >= st->pf_end;
+            if (nd.n_cols < 1 || nd.pmax >= c.max_seq) {
+                atomicCAS(A.err, 0, ERR_BAD_STATE);
+                action = ACT_STOP;
+            }
+            for (int j = 0; j < MAX_COLS; ++j) {
+                nd.first_layer[j] = j < nd.n_cols ? 0 : INT_MAX;
+                nd.pos[j] = st->pf_pos + j;
+            }
+            pub->d = nd;
+        } else if (action == ACT_NEWSTEP) {
             ++steps_started;
             const int len = st->len[0], base = st->base[0];
             StepDesc nd;
             nd.n_cols = len - base;
             nd.newest = len - 1 - base;
             nd.pmax = len - 1;
+            nd.fresh = 1 << (len - 1 - base);
+            nd.run_final = 1;
             nd.head_ok = (len - 1 - base) < st->max_early && len < st->target_len[0];
             if (nd.n_cols < 1 || nd.n_cols > c.slots || nd.n_cols > MAX_COLS || len > c.max_seq || base < 0) {
                 atomicCAS(A.err, 0, ERR_BAD_STATE);
@@ -281,7 +323,7 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
     if (kind == CTRL_TOP && c.capture && sm->bcast[3]) {
         const int keep = st->keep_rows, at = st->capture_n;
         for (int j = 0; j < keep && at + j < st->capture_cap; ++j) {
-            const float *src = c.logit_stage + (size_t)j * c.vocab;
+            const float *src = c.logit_stage + (size_t)(st->keep_row0 + j) * c.vocab;
             float *dst = c.capture + (size_t)(at + j) * c.vocab;
             for (int i = tid; i < c.vocab; i += CONS_THREADS) dst[i] = __ldcg(src + i);
         }
@@ -290,39 +332,42 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
     }
     if (action == ACT_NEWSTEP) {
         const StepDesc &nd = pub->d;
-        const int col = nd.newest, pos = nd.pmax;
-        const int tokid = min(max(c.tokens[pos], 0), c.vocab - 1);
-        const __nv_bfloat16 *erow = M.tok_embed + (size_t)tokid * c.d;
         const __nv_bfloat16 *g0 = M.layer[0].attn_norm;
-        for (int n0 = 0; n0 < c.d; n0 += 8 * CONS_THREADS) {   // eight loads of the embedding row in flight per thread
-            float v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int n = n0 + u * CONS_THREADS + tid;
-                v[u] = n < c.d ? __bfloat162float(erow[n]) * 1.0f : 0.f;
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int n = n0 + u * CONS_THREADS + tid;
-                if (n < c.d) {
-                    c.resid[(size_t)col * c.d + n] = v[u];
-                    xfrag_store(A.XA, n, col, v[u] * __bfloat162float(g0[n]));
-                }
-                float q = v[u] * v[u];
-                q += __shfl_xor_sync(0xffffffffu, q, 1);
-                q += __shfl_xor_sync(0xffffffffu, q, 2);
-                q += __shfl_xor_sync(0xffffffffu, q, 4);
-                q += __shfl_xor_sync(0xffffffffu, q, 8);
-                if ((tid & 15) == 0 && n < c.d) A.ssq_a[(size_t)(n >> 4) * MAX_COLS + col] = q;
-            }
-        }
         const int half = c.hd / 2;
-        for (int i = tid; i < half; i += CONS_THREADS) {
-            const double freq = pow((double)M.rope_base, -2.0 * i / c.hd);
-            double sn, cs;
-            sincos((double)pos * freq, &sn, &cs);
-            c.rope_cs[((size_t)col * half + i) * 2 + 0] = (float)cs;
-            c.rope_cs[((size_t)col * half + i) * 2 + 1] = (float)sn;
+        for (int col = 0; col < MAX_COLS; ++col) {
+            if (!((nd.fresh >> col) & 1)) continue;
+            const int pos = nd.pos[col];
+            const int tokid = min(max(c.tokens[pos], 0), c.vocab - 1);
+            const __nv_bfloat16 *erow = M.tok_embed + (size_t)tokid * c.d;
+            for (int n0 = 0; n0 < c.d; n0 += 8 * CONS_THREADS) {   // eight loads of the embedding row in flight per thread
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int n = n0 + u * CONS_THREADS + tid;
+                    v[u] = n < c.d ? __bfloat162float(erow[n]) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int n = n0 + u * CONS_THREADS + tid;
+                    if (n < c.d) {
+                        c.resid[(size_t)col * c.d + n] = v[u];
+                        xfrag_store(A.XA, n, col, v[u] * __bfloat162float(g0[n]));
+                    }
+                    float q = v[u] * v[u];
+                    q += __shfl_xor_sync(0xffffffffu, q, 1);
+                    q += __shfl_xor_sync(0xffffffffu, q, 2);
+                    q += __shfl_xor_sync(0xffffffffu, q, 4);
+                    q += __shfl_xor_sync(0xffffffffu, q, 8);
+                    if ((tid & 15) == 0 && n < c.d) A.ssq_a[(size_t)(n >> 4) * MAX_COLS + col] = q;
+                }
+            }
+            for (int i = tid; i < half; i += CONS_THREADS) {
+                const double freq = pow((double)M.rope_base, -2.0 * i / c.hd);
+                double sn, cs;
+                sincos((double)pos * freq, &sn, &cs);
+                c.rope_cs[((size_t)col * half + i) * 2 + 0] = (float)cs;
+                c.rope_cs[((size_t)col * half + i) * 2 + 1] = (float)sn;
+            }
         }
     }
     __threadfence();
@@ -826,7 +871,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     const int n_qkv = balanced_ctas((c.qkv_rows + 15) / 16, G), n_d = balanced_ctas(ntd, G), n_gu = balanced_ctas(c.dff / 16, G),
               n_head = balanced_ctas((c.vocab + 15) / 16, G);
     StepDesc d;
-    d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0;
+    d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0; d.fresh = 0; d.run_final = 1;
 #pragma unroll
     for (int i = 0; i < MAX_COLS; ++i) { d.first_layer[i] = INT_MAX; d.pos[i] = 0; }
 
@@ -1082,11 +1127,26 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
         }
         if (!restart) {
             // ---- final head for every column, then verification (Eq. 2 at temperature zero) in the control point
-            head_phase(A.XF, A.ssq_a, 1.0f, active_mask(d, L - 1));
+            if (d.run_final) head_phase(A.XF, A.ssq_a, 1.0f, active_mask(d, L - 1));
             action = control_point<ROLE>(A, S, CTRL_TOP, 0, pub_no, d, steps_started);
             book_control();
         }
     }
+}
+
+// Arms the prompt passes of the persistent kernel for sequence 0 (KV cache <- LM(x), first line of Algorithm 1).
+__global__ void k_prefill_arm(Ctx c, int n_prompt) {
+    DevState *st = c.st;
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    st->pf_pos = 0;
+    st->pf_end = n_prompt;
+    st->done[0] = 0;
+    st->n_done = 0;
+    st->len[0] = 0;
+    st->base[0] = 0;
+    st->tape_n = 0;
+    st->tape_i = 0;
+    for (int l = 0; l < c.L; ++l) c.fill[l] = 0;
 }
 
 template <int HD>
