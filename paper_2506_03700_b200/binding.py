@@ -39,7 +39,7 @@ class AdaError(RuntimeError):
             lib = _LIB
             if lib is not None:
                 msg += f" ({lib.ada_strerror(code).decode()})"
-                if code == -4:
+                if code in (-4, -5, -2) and lib.ada_last_cuda_error():
                     msg += f" [{lib.ada_last_cuda_error().decode()}]"
         except Exception:
             pass

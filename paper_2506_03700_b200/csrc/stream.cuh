@@ -410,11 +410,12 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
 #pragma unroll
                 for (int p = 0; p < PAIR; ++p) {
                     const int wslot = r.wi % NW;
-                    // Every warp waits for every stage in order, although only its owners use it: an
-                    // mbarrier tells phases apart by one parity bit, so a warp that skipped ahead by
-                    // more than a ring (in a gate/up group a warp's own stages are 14 apart, the ring
-                    // holds 9) would take an older phase of the slot for the one it wants.  Only the
-                    // owners release the stage, so a slot is free as soon as its math is done.
+                    // Every warp waits for and releases every stage in order, although only its owners
+                    // use it.  An mbarrier tells phases apart by one parity bit: a warp that ran ahead
+                    // of, or fell behind, the others by a ring would mistake one phase of a slot for
+                    // another (releasing stages by their owners alone was tried: a lagging warp then
+                    // waits for a refill that needs its own release).  With all eight arrivals per
+                    // stage no warp is ever more than one ring away from any other.
                     mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
                     if (s == slot_id) {
                         if (threadIdx.x == 0 && kc == 0 && g0 == t0 && p == 0) trace(S, EV_W0, 0);
@@ -437,9 +438,9 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                                 par ^= 1;
                             }
                         }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_n(&sm->w_empty[wslot], (uint32_t)TS);   // KS owners x TS = 8 arrivals
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->w_empty[wslot]);
                     ++r.wi;
                 }
             }
