@@ -163,8 +163,8 @@ int ada_debug_profile(ada_session *s, int32_t on);
 int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out, double *bytes_out);
 /* Select the decode path: 1 = the persistent kernel (one cooperative launch runs many steps of
  * Algorithm 1; bf16 models, one sequence, at most 8 tokens per pass, 64-token KV pages, head_dim 64
- * or 128, at most 4 q heads per kv head, d_model / n_q_heads*head_dim / d_ff multiples of 64,
- * max_seq_len at most 256 * head_dim); it is the default wherever a session qualifies.  0 = one
+ * or 128, at most 4 q heads per kv head, d_model / n_q_heads*head_dim / d_ff multiples of 64); it is
+ * the default wherever a session qualifies.  0 = one
  * kernel per operation on CUDA cores (any dtype, any batch; also what prefill uses).
  * ADA_EUNSUPPORTED if path 1 is asked of a session that does not qualify. */
 int ada_debug_set_path(ada_session *s, int32_t path);

@@ -425,7 +425,6 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     if (g.dtype != ADA_DTYPE_BF16 || S->batch != 1 || S->slots > st::MAX_COLS || S->page_tokens != mg::ATT_PAGE) return ADA_OK;
     if ((g.head_dim != 64 && g.head_dim != 128) || group > 4) return ADA_OK;
     if (g.d_model % 64 || qd % 64 || g.d_ff % 64) return ADA_OK;
-    if (S->n_chunks > g.head_dim) return ADA_OK;   // the chunk merge stages 2 x 32 x n_chunks floats in shared memory
     int dev = 0, sms = 0, coop = 0, nb = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return ADA_OK; }
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

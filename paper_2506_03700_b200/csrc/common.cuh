@@ -10,7 +10,7 @@
 namespace ada {
 
 constexpr int kMaxRows = 64;        // rows (tokens) one layer pass can carry
-constexpr int kAttnChunk = 256;     // attention split size; chunk c covers positions [256c, 256c+255]
+constexpr int kAttnChunk = 128;     // attention split size; chunk c covers positions [128c, 128c+127]
 constexpr int kMaxTape = 4096;
 constexpr int kHeadLogCap = 1 << 16;
 

@@ -497,7 +497,7 @@ __device__ __forceinline__ void attn_merge_to(const float (&o)[NT][4], const flo
 }
 
 // Consumers: causal attention of every active column over the cache plus the in-flight rows.
-// Work item = (kv head, 256-position chunk).  Within a 64-position sub-block warp (mt, qr) handles
+// Work item = (kv head, 128-position chunk).  Within a 64-position sub-block warp (mt, qr) handles
 // query tile mt (16 of the up to 32 (column, q head) pairs of the kv head) and positions
 // [16 qr, 16 qr + 16).  K and V rows of the columns processed in this pass are not in the cache
 // yet: they are rotated / rounded here from the QKV output, patched into the shared-memory copy
@@ -775,62 +775,51 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
         }
         // ---- the CTA that finishes a kv head's last item merges the chunks of that head
         if (tid == 0) trace(S, EV_ITEM, item);
-        __threadfence();
         bar_consumers();
-        if (tid == 0) sm->bcast[2] = (int)atomicAdd(A.attn_cnt + kvh, 1u);
+        if (tid == 0) {   // release this block's partials and acquire the others' in one step
+            unsigned old;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + kvh) : "memory");
+            sm->bcast[2] = (int)old;
+        }
         bar_consumers();
         if (sm->bcast[2] == nchunk - 1) {
-            __threadfence();
-            // (1) every (max, sum) pair of the head's chunks -> shared memory, all loads in flight at once
-            float *sm_m = &as->o[0][0][0][0];                       // [32][nchunk]
-            float *sm_e = sm_m + 32 * nchunk;                        // [32][nchunk]: sum, then exp(max_k - max)
-            float *sm_den = &as->ml[0][0][0][0];                     // [32]
+            // Four features of one (column, q head) per thread and pass; the chunk partials are folded in
+            // ascending order, eight at a time with all their loads in flight, by the usual running-max rule.
             const int nqc = MAX_COLS * group;
-            for (int idx = tid; idx < nqc * nchunk; idx += CONS_THREADS) {
-                const int qcol = idx / nchunk, k = idx - qcol * nchunk, cc = qcol / group, g = qcol - cc * group;
-                float2 v = make_float2(-INFINITY, 0.f);
-                if (((mask >> cc) & 1u) && k <= d.pos[cc] / ATT_CHUNK)
-                    v = __ldcg(reinterpret_cast<const float2 *>(A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + k) * ATT_STRIDE + HD));
-                sm_m[idx] = v.x;
-                sm_e[idx] = v.y;
-            }
-            bar_consumers();
-            // (2) per (column, q head): weights exp(m_k - max) and the denominator, chunks in ascending order
-            if (tid < nqc) {
-                float Mx = -INFINITY;
-                for (int k = 0; k < nchunk; ++k) Mx = fmaxf(Mx, sm_m[tid * nchunk + k]);
-                float den = 0.f;
-                for (int k = 0; k < nchunk; ++k) {
-                    const float mk = sm_m[tid * nchunk + k];
-                    const float w = mk == -INFINITY ? 0.f : __expf(mk - Mx);
-                    den += sm_e[tid * nchunk + k] * w;
-                    sm_e[tid * nchunk + k] = w;
-                }
-                sm_den[tid] = den;
-            }
-            bar_consumers();
-            // (3) outputs, four features per thread and pass, eight chunk loads in flight
             for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
                 const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = qcol / group, g = qcol - cc * group;
                 if (!((mask >> cc) & 1u)) continue;
                 const int h = kvh * group + g;
                 const int nch = d.pos[cc] / ATT_CHUNK + 1;
-                const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE + dim;
+                const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE;
+                float Mx = -INFINITY, den = 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int k0 = 0; k0 < nch; k0 += 8) {
+                    float2 ml[8];
                     float4 ov[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        ov[u] = k0 + u < nch ? __ldcg(reinterpret_cast<const float4 *>(part + (size_t)(k0 + u) * ATT_STRIDE)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int u = 0; u < 8; ++u) {
+                        const bool ok = k0 + u < nch;
+                        const float *pk = part + (size_t)(k0 + u) * ATT_STRIDE;
+                        ml[u] = ok ? __ldcg(reinterpret_cast<const float2 *>(pk + HD)) : make_float2(-INFINITY, 0.f);
+                        ov[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(pk + dim)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    float Mn = Mx;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, ml[u].x);
+                    if (Mn == -INFINITY) continue;
+                    const float sc = Mx == -INFINITY ? 0.f : __expf(Mx - Mn);
+                    den *= sc; acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        if (k0 + u < nch) {
-                            const float w = sm_e[qcol * nchunk + k0 + u];
+                        if (ml[u].x != -INFINITY) {
+                            const float w = __expf(ml[u].x - Mn);
+                            den += ml[u].y * w;
                             acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
                         }
                     }
+                    Mx = Mn;
                 }
-                const float den = sm_den[qcol];
                 xfrag_store(A.XO, h * HD + dim, cc, acc.x / den);
                 xfrag_store(A.XO, h * HD + dim + 1, cc, acc.y / den);
                 xfrag_store(A.XO, h * HD + dim + 2, cc, acc.z / den);

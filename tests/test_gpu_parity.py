@@ -264,7 +264,7 @@ def test_chained_and_mixed_calls():
 
 
 def test_context_across_pages_and_attention_chunks():
-    """Prompt + generation cross several KV pages and the 256-position attention split."""
+    """Prompt + generation cross several KV pages and the 128-position attention split."""
     cfg = small("bf16", n_layers=2, exit_layers=(1,))
     pair = Pair(cfg)
     prompt = synth.make_prompt(cfg, n=250).numpy()

@@ -209,7 +209,7 @@ def test_chained_calls_and_both_paths_mixed():
 
 
 def test_context_across_pages_and_attention_chunks():
-    """Prompt + generation cross several 64-token KV pages and the 256-position attention split."""
+    """Prompt + generation cross several 64-token KV pages and the 128-position attention split."""
     cfg = mha(n_layers=2, exit_layers=(1,))
     pair = Pair(cfg)
     prompt = synth.make_prompt(cfg, n=250).numpy()
