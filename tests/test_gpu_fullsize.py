@@ -1,0 +1,92 @@
+"""The benchmark's own configuration (8B-shaped model, the launch shape bench.py times) at full size.
+
+The oracle cannot recompute a 1024-token context of an 8B-shaped model in test time, so full-size
+parity is checked two ways: (1) sampled outputs the oracle can compute one by one: the same weights
+on a short prompt, final logits and tokens against the oracle; (2) properties that hold at any size
+on the full prompt: adaptive decoding equals the library's plain decoding bit for bit (tokens and
+final-logit bits), the counters add up, and the cache state after rollbacks equals that of a run
+that never left the plain path."""
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle
+from paper_2506_03700_b200 import binding, synth
+from test_gpu_parity import check_against_oracle
+
+
+class BigPair:
+    _cache = None
+
+    def __init__(self):
+        self.cfg = synth.CONFIGS["8b"]
+        self.w = synth.make_weights(self.cfg, seed=1234, device="cuda")
+        self.gm = binding.Model(self.cfg, self.w)
+        for l in self.cfg.exit_layers:
+            self.gm.set_exit_head(l, None, self.cfg.logit_scale)
+        self._om = None
+
+    @property
+    def om(self):
+        if self._om is None:
+            self._om = oracle.model_from_torch(self.cfg, {k: v.cpu() for k, v in self.w.items()})
+        return self._om
+
+
+@pytest.fixture(scope="module")
+def big():
+    if torch.cuda.get_device_properties(0).total_memory < 40e9:
+        pytest.skip("needs a GPU with room for the 8B-shaped weights")
+    p = BigPair()
+    yield p
+    del p
+    torch.cuda.empty_cache()
+
+
+def test_8b_short_prompt_logits_and_tokens_match_the_oracle(big):
+    cfg = big.cfg
+    prompt = synth.make_prompt(cfg, n=12).numpy()
+    n = 4
+    S = binding.Session(big.gm, 1, 64, 64, 5)
+    assert S.get_path() == 1
+    S.capture_logits(n + 2)
+    S.prefill(prompt)
+    out = S.plain_decode(n)[0]
+    check_against_oracle(big, prompt, out, S.captured_logits().cpu().numpy())
+
+
+def test_8b_full_prompt_adaptive_equals_plain_bit_for_bit(big):
+    cfg = big.cfg
+    prompt = synth.make_prompt(cfg, seed=5678).numpy()          # the benchmark's 1024-token prompt
+    n = 96
+    max_seq = cfg.prompt_len + cfg.gen_len + 16                  # the benchmark's session shape
+    P = binding.Session(big.gm, 1, max_seq, 64, 5)
+    assert P.get_path() == 1
+    P.capture_logits(n + 8)
+    P.prefill(prompt)
+    ref = P.plain_decode(n)[0]
+    ref_lg = P.captured_logits()[:n].clone()
+    lp, fp_ = P.state()
+    assert len(set(ref.tolist())) > 8
+    for gamma, tape in [(cfg.threshold, None), (0.0, None), (0.5, [1] * 64)]:
+        S = binding.Session(big.gm, 1, max_seq, 64, 5)
+        S.capture_logits(n + 8)
+        S.prefill(prompt)
+        if tape:
+            S.set_exit_tape(tape)
+        st = binding.Stats()
+        out = S.adaptive_decode(n, gamma, cfg.exit_layers, 5, st)[0]
+        assert np.array_equal(out, ref), gamma
+        assert torch.equal(S.captured_logits()[:n], ref_lg), gamma
+        ls, fs = S.state()
+        assert ls == lp and np.array_equal(fs, fp_)
+        assert st.early_exits == st.accepted + st.rejected + st.discarded
+        assert st.accepted + st.verify_steps - st.truncated == n - 1
+        assert st.early_exits > 0 and st.rejected > 0
+        for l in (0, 15, 31):                                    # rolled-back rows left nothing behind
+            for pos in (0, 700, cfg.prompt_len + 3, cfg.prompt_len + n - 2):
+                assert np.array_equal(S.read_kv(0, l, pos), P.read_kv(0, l, pos))
+                assert np.array_equal(S.read_kv(1, l, pos), P.read_kv(1, l, pos))
