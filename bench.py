@@ -93,6 +93,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of `values` over the ranks of the job (the slowest replica sets the time).
+    The decode path does not shard: N GPUs run N independent replicas and exchange nothing else."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_max: float) -> float:
+    """Throughput of the whole job: all replicas' tokens over the slowest replica's time."""
+    return tokens_per_rank * world / (ms_max * 1e-3)
+
+
 def byte_model(cfg, stats, ctx_mean: float) -> float:
     """Algorithmic HBM bytes of a decode call: every layer pass streams one layer's weights and
     reads that layer's K/V once for all rows; every head evaluation and every verification streams
@@ -201,10 +216,7 @@ def run_ours(args):
     prof = sess.profile_read()
     sess.profile(False)
 
-    tms = torch.tensor([a_ms, p_ms, a_wall, p_wall], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    a_ms, p_ms, a_wall, p_wall = [float(x) for x in tms.cpu()]
+    a_ms, p_ms, a_wall, p_wall = max_over_ranks([a_ms, p_ms, a_wall, p_wall], dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -223,7 +235,7 @@ def run_ours(args):
     dom = "k_decode_persistent"
     dom_gbs = a_bytes / (a_st.decode_ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": n_tok / (a_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "metric": METRIC, "value": whole_job_tokens_per_s(gen_len, world, a_ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": a_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": f"{cfg.name}-shaped decoder bs1, {cfg.prompt_len}-token uniform-random prompt, "
@@ -231,7 +243,7 @@ def run_ours(args):
                                f"tied head logit scale {cfg.logit_scale}, max_early 5",
                    "tokens_per_step": per_step, "l2": "inputs_larger_than_l2 (weights stream >> 126 MB)",
                    "parallelism": "replicas" if world > 1 else "single"},
-        "e2e": {"value": n_tok / (a_wall * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 64 + 4 * 16,
+        "e2e": {"value": whole_job_tokens_per_s(gen_len, world, a_wall), "unit": UNIT, "h2d_bytes_per_step": 64 + 4 * 16,
                 "d2h_bytes_per_step": int(per_step * 4 + 8 * (9 + 256 + 4))},
         "gpu_launches": int(a_st.kernel_launches),
         "clocks": clocks,
