@@ -2,6 +2,7 @@
 // loops that issue the kernels of Algorithm 1.  All decoding state lives on the device; the host
 // only decides how far to launch and reads back a few counters.
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <memory>
@@ -126,7 +127,7 @@ namespace {
 // Scratch layout (all offsets 256-byte aligned).
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
-        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qkvraw, attn_cnt,
+        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qkvraw, attn_cnt, rope_freq,
         grid_ctr, pub, err, total;
 };
 
@@ -174,6 +175,7 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
         L.ssq_b = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
         L.qkvraw = take(sizeof(float) * (size_t)st::MAX_COLS * qkv_rows);
         L.attn_cnt = take(sizeof(unsigned) * g.n_kv_heads);
+        L.rope_freq = take(sizeof(double) * (g.head_dim / 2));
         L.grid_ctr = take(256);
         L.pub = take(sizeof(mg::Pub) * 2);
         L.err = take(256);
@@ -467,6 +469,9 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     M.rope_base = g.rope_base;
     CK(cudaMemcpyAsync(S->maps_dev, S->maps_host.data(), sizeof(CUtensorMap) * S->maps_host.size(), cudaMemcpyHostToDevice, S->stream));
     CK(cudaMemcpyAsync(S->mm_dev, &M, sizeof(M), cudaMemcpyHostToDevice, S->stream));
+    std::vector<double> freq(g.head_dim / 2);
+    for (int i = 0; i < g.head_dim / 2; ++i) freq[i] = pow((double)g.rope_base, -2.0 * i / g.head_dim);
+    CK(cudaMemcpyAsync(b + lay.rope_freq, freq.data(), sizeof(double) * freq.size(), cudaMemcpyHostToDevice, S->stream));
     CK(cudaStreamSynchronize(S->stream));
     mg::MegaArgs &a = S->margs;
     a.c = S->c;
@@ -479,6 +484,7 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.attn_part = S->c.attn_part;
     a.head_part = S->c.head_part;
     a.attn_cnt = (unsigned *)(b + lay.attn_cnt);
+    a.rope_freq = (const double *)(b + lay.rope_freq);
     a.grid_ctr = (unsigned *)(b + lay.grid_ctr);
     a.pub = (mg::Pub *)(b + lay.pub);
     a.err = (int *)(b + lay.err);

@@ -75,6 +75,7 @@ struct MegaArgs {
     float *qkvraw;             // [8][qkv_rows]
     float *attn_part;          // [8 * nq][n_chunks][hd + 4]
     float *head_part;          // [grid][8][4]
+    const double *rope_freq;   // [hd/2]: base^(-2i/hd), computed once on the host
     unsigned *attn_cnt;        // [nkv]
     unsigned *grid_ctr;
     Pub *pub;                  // [2]
@@ -362,11 +363,14 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
                 }
             }
             for (int i = tid; i < half; i += CONS_THREADS) {
-                const double freq = pow((double)M.rope_base, -2.0 * i / c.hd);
-                double sn, cs;
-                sincos((double)pos * freq, &sn, &cs);
-                c.rope_cs[((size_t)col * half + i) * 2 + 0] = (float)cs;
-                c.rope_cs[((size_t)col * half + i) * 2 + 1] = (float)sn;
+                // angle = pos * freq in double, reduced to [-pi, pi] in double, then single-precision sin / cos
+                // (double-precision transcendentals with large arguments are slow on this GPU)
+                const double a = (double)pos * A.rope_freq[i];
+                const double r = a - 6.283185307179586476925 * rint(a * 0.15915494309189533577);
+                float sn, cs;
+                sincosf((float)r, &sn, &cs);
+                c.rope_cs[((size_t)col * half + i) * 2 + 0] = cs;
+                c.rope_cs[((size_t)col * half + i) * 2 + 1] = sn;
             }
         }
     }
