@@ -369,7 +369,7 @@ __device__ __forceinline__ void stage_full(float (&acc)[4][4], const unsigned ch
 
 // Consumer warps.  Within a group of up to eight tiles the warps are arranged as TS tile slots x
 // KS k-splits (TS * KS = 8, TS the smallest power of two holding the group); a warp multiplies
-// the k-steps s = ks_id (mod KS) of its slot's stages.  The k-splits of a tile are summed in a
+// the stages of its slot whose k chunk is ks_id (mod KS).  The k-splits of a tile are summed in a
 // fixed order through shared memory, then `epi(tile, acc)` runs in the slot's first warp with
 //   acc[p][i]: fragment element i of matrix p: rows lane/4 (i<2) or lane/4+8, columns 2(lane%4)+(i&1).
 // The arrangement depends only on the tile partition, never on which token columns are in use.
@@ -417,19 +417,17 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                     // waits for a refill that needs its own release).  With all eight arrivals per
                     // stage no warp is ever more than one ring away from any other.
                     mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
-                    if (s == slot_id) {
+                    // the k-splits of a tile take whole stages in turn (chunk kc belongs to split kc % KS):
+                    // a warp then multiplies all 32 k-steps of a stage, which amortises the per-stage
+                    // waiting and set-up (splitting every stage among the warps streamed 20-30 % slower)
+                    if (s == slot_id && (kc % KS) == ks_id) {
                         if (threadIdx.x == 0 && kc == 0 && g0 == t0 && p == 0) trace(S, EV_W0, 0);
                         const unsigned char *ws = sm->w[wslot] + a_off;
-                        if (ksteps == KSTEPS) {   // full chunk: software-pipelined, fully unrolled per k-split
-                            switch (KS) {
-                                case 1: stage_full<1>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
-                                case 2: stage_full<2>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
-                                case 4: stage_full<4>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
-                                default: stage_full<8>(acc[p], ws, xs, ks_id, a_hi, a_sw); break;
-                            }
+                        if (ksteps == KSTEPS) {   // full chunk: software-pipelined, fully unrolled
+                            stage_full<1>(acc[p], ws, xs, 0, a_hi, a_sw);
                         } else {                  // short last chunk of K
                             int par = 0;
-                            for (int ks = ks_id; ks < ksteps; ks += KS) {
+                            for (int ks = 0; ks < ksteps; ++ks) {
                                 uint32_t a[4];
                                 ldmatrix_x4(a, ws + (ks >> 2) * 2048 + (((((ks & 3) << 1) | a_hi) ^ a_sw) << 4));
                                 const uint4 b = xs[ks * 8];
