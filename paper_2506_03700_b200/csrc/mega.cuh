@@ -98,22 +98,29 @@ __device__ __forceinline__ unsigned active_mask(const StepDesc &d, int layer) {
 }
 
 // rstd[c] = 1 / sqrt(sum_tiles ssq[tile][c] / d + eps), one warp per column, fixed summation order.
-__device__ __forceinline__ void compute_rstd(Smem *sm, const float *ssq, int ntiles, int d, float eps) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// RMSNorm factors 1/sqrt(mean square + eps) of the eight columns from the per-tile sums of squares
+// ssq[tile][column], by the activation producer warp: lane l sums column l%8 over the tiles
+// l/8 + 4u in ascending order (32 loads in flight), the four lanes of a column are folded by a
+// butterfly.  The order is fixed, so the factor of a column does not depend on the other columns.
+__device__ __forceinline__ void rstd_produce(Smem *sm, const float *ssq, int ntiles, int d, float eps, unsigned seq) {
+    const int lane = threadIdx.x & 31, col = lane & 7, sub = lane >> 3;
     float s = 0.f;
-    for (int t0 = 0; t0 < ntiles; t0 += 256) {   // eight loads in flight per lane; the order of the sum is fixed
-        float v[8];
+    for (int t0 = 0; t0 < ntiles; t0 += 128) {
+        float v[32];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int t = t0 + lane + 32 * u;
-            v[u] = t < ntiles ? ldcg(ssq + (size_t)t * MAX_COLS + warp) : 0.f;
+        for (int u = 0; u < 32; ++u) {
+            const int t = t0 + sub + 4 * u;
+            v[u] = t < ntiles ? ldcg(ssq + (size_t)t * MAX_COLS + col) : 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) s += v[u];
+        for (int u = 0; u < 32; ++u) s += v[u];
     }
-    s = warp_sum(s);
-    if (lane == 0) sm->vec[warp] = 1.0f / sqrtf(s / (float)d + eps);
-    bar_consumers();
+    s += __shfl_xor_sync(0xffffffffu, s, 8);
+    s += __shfl_xor_sync(0xffffffffu, s, 16);
+    if (lane < MAX_COLS) sm->vec[lane] = 1.0f / sqrtf(s / (float)d + eps);
+    __threadfence_block();
+    __syncwarp();
+    if (lane == 0) *(volatile unsigned *)&sm->vec_seq = seq;
 }
 
 // Grid barrier as seen by the consumers of a CTA.
@@ -900,13 +907,15 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols) {
         Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head; g.columns(cols ? cols : 1u << d.newest);
         x_ready();
+        const unsigned vseq = bar_no + 1;
         if (ROLE == 2) {
-            if (ssq) compute_rstd(sm, ssq, ntd, d_model, c.eps);
             Msa run[2];
             run[0].m = run[1].m = -INFINITY; run[0].s = run[1].s = 0.f; run[0].i = run[1].i = INT_MAX;
             const int c0 = 2 * (lane & 3);
-            const float r0 = ssq ? sm->vec[c0] * scale : scale, r1 = ssq ? sm->vec[c0 + 1] * scale : scale;
+            float r0 = scale, r1 = scale;
+            bool have_r = ssq == nullptr;
             gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0] * scale; r1 = sm->vec[c0 + 1] * scale; have_r = true; }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8;
@@ -951,6 +960,8 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                 float *o = A.head_part + ((size_t)blockIdx.x * MAX_COLS + threadIdx.x) * 4;
                 o[0] = a.m; o[1] = a.s; o[2] = __int_as_float(a.i);
             }
+        } else if (ROLE == 1) {
+            gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { if (ssq) rstd_produce(sm, ssq, ntd, d_model, c.eps, vseq); });
         } else {
             gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
         }
@@ -971,18 +982,21 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             {
                 Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_qkv; g.columns(mask);
                 x_ready();
+                const unsigned vseq = bar_no + 1;
                 if (ROLE == 2) {
-                    compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);
                     const int c0 = 2 * (lane & 3);
-                    const float r0 = sm->vec[c0], r1 = sm->vec[c0 + 1];
+                    float r0 = 0.f, r1 = 0.f;
+                    bool have_r = false;
                     gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                        if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0]; r1 = sm->vec[c0 + 1]; have_r = true; }
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
                             if (n < c.qkv_rows && ((mask >> cc) & 1u)) A.qkvraw[(size_t)cc * c.qkv_rows + n] = acc[0][i] * ((i & 1) ? r1 : r0);
                         }
                     });
-                } else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+                } else if (ROLE == 1) gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { rstd_produce(sm, A.ssq_a, ntd, d_model, c.eps, vseq); });
+                else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
                 phase_barrier(2);
             }
             // ---- attention (the KV producer may run ahead: rows of this pass are patched in by the consumers)
@@ -1031,11 +1045,13 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             {
                 Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff; g.ctas = n_gu; g.columns(mask);
                 x_ready();
+                const unsigned vseq = bar_no + 1;
                 if (ROLE == 2) {
-                    compute_rstd(sm, A.ssq_b, ntd, d_model, c.eps);
                     const int c0 = 2 * (lane & 3);
-                    const float r0 = sm->vec[c0], r1 = sm->vec[c0 + 1];
+                    float r0 = 0.f, r1 = 0.f;
+                    bool have_r = false;
                     gemm_consume<2>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[2][4]) {
+                        if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0]; r1 = sm->vec[c0 + 1]; have_r = true; }
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
@@ -1046,7 +1062,8 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                             }
                         }
                     });
-                } else gemm_phase<ROLE, 2>(S, g, r, pol, NoEpi());
+                } else if (ROLE == 1) gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { rstd_produce(sm, A.ssq_b, ntd, d_model, c.eps, vseq); });
+                else gemm_phase<ROLE, 2>(S, g, r, pol, NoEpi());
                 phase_barrier(6);
             }
             // ---- down projection + residual; prepares the next layer's (and the head's) input
@@ -1096,18 +1113,21 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                 if (hl.wT) {
                     Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_d; g.columns(1u << d.newest);
                     x_ready();
+                    const unsigned vseq = bar_no + 1;
                     if (ROLE == 2) {
-                        compute_rstd(sm, A.ssq_a, ntd, d_model, c.eps);
                         const int c0 = 2 * (lane & 3);
-                        const float r0 = sm->vec[c0], r1 = sm->vec[c0 + 1];
+                        float r0 = 0.f, r1 = 0.f;
+                        bool have_r = false;
                         gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
+                            if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0]; r1 = sm->vec[c0 + 1]; have_r = true; }
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
                                 xfrag_store(A.XT, n, cc, acc[0][i] * ((i & 1) ? r1 : r0));
                             }
                         });
-                    } else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
+                    } else if (ROLE == 1) gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { rstd_produce(sm, A.ssq_a, ntd, d_model, c.eps, vseq); });
+                    else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
                     phase_barrier(10);
                     head_phase(A.XT, nullptr, hl.head_scale, 0u);
                 } else {

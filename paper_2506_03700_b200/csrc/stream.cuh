@@ -53,6 +53,7 @@ struct Smem {                                    // must start on a 1024-byte bo
     int abort;
     int bcast[8];
     unsigned trace_n;
+    unsigned vec_seq;                             // phase for which vec[] holds the normalisation factors (see vec_wait)
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -202,9 +203,26 @@ __device__ __forceinline__ void mbar_wait(const Shared &S, unsigned long long *b
     }
 }
 
+// The consumers wait until the activation producer warp has left the per-column factors of phase
+// `seq` in vec[] (it computes them while the first weight stages are being multiplied).
+__device__ __forceinline__ void vec_wait(const Shared &S, unsigned seq) {
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (*(volatile unsigned *)&S.sm->vec_seq == seq) return;
+        if ((it & 127u) == 127u) {
+            if (aborted(S)) return;
+            if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
+            unsigned long long t = gtime();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > WAIT_NS) { raise_error(S, ERR_TIMEOUT_MBAR); return; }
+        }
+    }
+}
+
 // Grid barrier on a monotonically increasing counter: arrive once per CTA, wait for `target`.
 __device__ __forceinline__ void grid_arrive(unsigned *ctr) {
-    __threadfence();
+    // the release of the reduction orders this thread's earlier writes, and through the block-level
+    // barrier before it those of the whole CTA; a separate fence before it only adds its latency
     fence_proxy_async();
     red_release_add(ctr, 1u);
 }
@@ -315,13 +333,17 @@ __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, i
 }
 
 // Activation producer warp: one stage per (tile group, k chunk).
-__device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol) {
+// `after_first` runs once, after the first stage has been issued: work of the phase that is not
+// needed before the epilogues (the normalisation factors) and must not delay the first copy.
+template <class Hook>
+__device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol, Hook &&after_first) {
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31;
     int t0, t1;
     cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
     const int nch = (g.K + KC - 1) / KC;
     const int XC = g.xchunks();
+    bool hooked = false;
     for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
         for (int kc = 0; kc < nch; kc += XC) {
             const int nc = min(XC, nch - kc);
@@ -335,8 +357,16 @@ __device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, i
                              bytes, &sm->x_full[slot], pol);
             }
             ++r.xi;
+            if (!hooked) { after_first(); hooked = true; }
         }
     }
+    if (!hooked) after_first();
+}
+struct NoHook {
+    __device__ __forceinline__ void operator()() const {}
+};
+__device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol) {
+    gemm_produce_x(S, g, cta, G, r, pol, NoHook());
 }
 
 // The k-steps ks_id + KS_ j (j < 32 / KS_) of one full weight stage: fragment loads run PF steps
@@ -501,6 +531,7 @@ __device__ __forceinline__ void smem_init(Smem *sm) {
         for (int i = 0; i < NX; ++i) { mbar_init(&sm->x_full[i], 1); mbar_init(&sm->x_empty[i], CONS_WARPS); }
         sm->abort = 0;
         sm->trace_n = 0;
+        sm->vec_seq = 0;
         fence_mbar_init();
         fence_proxy_async();
     }
