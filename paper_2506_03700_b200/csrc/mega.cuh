@@ -1009,24 +1009,27 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                 x_ready();
                 if (ROLE == 2) {
                     const __nv_bfloat16 *gain = ly.ffn_norm;
-                    float rv[4] = {0.f, 0.f, 0.f, 0.f};
-                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile) {   // the residual is fetched while the weights stream
+                    uint32_t *stash = stash_of(sm);
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile) {   // residual and gain are fetched while the weights stream
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = 2 * (lane & 3) + (i & 1);
-                            rv[i] = ((mask >> cc) & 1u) ? c.resid[(size_t)cc * d_model + n] : 0.f;
+                            if ((mask >> cc) & 1u) cp_async4(stash + i * 32, c.resid + (size_t)cc * d_model + n);
                         }
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) cp_async4(stash + (4 + h) * 32, gain + ((tile * 16 + (lane >> 2) + h * 8) & ~1));
                     }, [&](int tile, float (&acc)[1][4]) {
                         const int c0 = 2 * (lane & 3);
                         float sq[2] = {0.f, 0.f};
+                        cp_async_wait_all();
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
                             if ((mask >> cc) & 1u) {
                                 float *rp = c.resid + (size_t)cc * d_model + n;
-                                const float v = rv[i] + acc[0][i];
+                                const float v = __uint_as_float(stash[i * 32]) + acc[0][i];
                                 *rp = v;
-                                xfrag_store(A.XB, n, cc, v * __bfloat162float(gain[n]));
+                                xfrag_store(A.XB, n, cc, v * bf16_of_word(stash[(4 + (i >> 1)) * 32], n));
                                 sq[i & 1] += v * v;
                             }
                         }
@@ -1074,25 +1077,32 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                     const __nv_bfloat16 *gain_next = l + 1 < L ? M.layer[l + 1].attn_norm : nullptr;
                     const bool want_f = l + 1 == L || A.exit_at[l + 1] != 0;
                     const __nv_bfloat16 *gain_f = M.final_norm;
-                    float rv[4] = {0.f, 0.f, 0.f, 0.f};
+                    uint32_t *stash = stash_of(sm);
                     gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile) {
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = 2 * (lane & 3) + (i & 1);
-                            rv[i] = ((mask >> cc) & 1u) ? c.resid[(size_t)cc * d_model + n] : 0.f;
+                            if ((mask >> cc) & 1u) cp_async4(stash + i * 32, c.resid + (size_t)cc * d_model + n);
+                        }
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int n2 = (tile * 16 + (lane >> 2) + h * 8) & ~1;
+                            if (gain_next) cp_async4(stash + (4 + h) * 32, gain_next + n2);
+                            if (want_f) cp_async4(stash + (6 + h) * 32, gain_f + n2);
                         }
                     }, [&](int tile, float (&acc)[1][4]) {
                         const int c0 = 2 * (lane & 3);
                         float sq[2] = {0.f, 0.f};
+                        cp_async_wait_all();
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
                             if ((mask >> cc) & 1u) {
                                 float *rp = c.resid + (size_t)cc * d_model + n;
-                                const float v = rv[i] + acc[0][i];
+                                const float v = __uint_as_float(stash[i * 32]) + acc[0][i];
                                 *rp = v;
-                                if (gain_next) xfrag_store(A.XA, n, cc, v * __bfloat162float(gain_next[n]));
-                                if (want_f) xfrag_store(A.XF, n, cc, v * __bfloat162float(gain_f[n]));
+                                if (gain_next) xfrag_store(A.XA, n, cc, v * bf16_of_word(stash[(4 + (i >> 1)) * 32], n));
+                                if (want_f) xfrag_store(A.XF, n, cc, v * bf16_of_word(stash[(6 + (i >> 1)) * 32], n));
                                 sq[i & 1] += v * v;
                             }
                         }

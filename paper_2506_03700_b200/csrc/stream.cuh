@@ -203,6 +203,23 @@ __device__ __forceinline__ void mbar_wait(const Shared &S, unsigned long long *b
     }
 }
 
+// Epilogue operands are fetched while the weights stream, by 4-byte asynchronous copies into a
+// per-warp corner of the scratch area (word k of lane l at [k][l]) rather than into registers: a
+// value held in a register across the main loop ties up the register file, and wherever the
+// compiler has to move it the warp first waits for the load.  Each lane reads back only its own
+// words, after cp_async_wait_all().  The k-split reduction uses the first 8 KB of the scratch area.
+constexpr int STASH_OFFSET = 8192, STASH_WORDS = 8;
+static_assert(STASH_OFFSET + CONS_WARPS * STASH_WORDS * 32 * 4 <= SCRATCH_BYTES, "stash exceeds the scratch area");
+__device__ __forceinline__ uint32_t *stash_of(Smem *sm) {
+    return reinterpret_cast<uint32_t *>(sm->scratch + STASH_OFFSET) + (threadIdx.x >> 5) * (STASH_WORDS * 32) + (threadIdx.x & 31);
+}
+__device__ __forceinline__ void cp_async4(uint32_t *dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// element n of a bf16 vector from the aligned 32-bit word that holds it
+__device__ __forceinline__ float bf16_of_word(uint32_t w, int n) { return __uint_as_float((n & 1) ? (w & 0xffff0000u) : (w << 16)); }
+
 // The consumers wait until the activation producer warp has left the per-column factors of phase
 // `seq` in vec[] (it computes them while the first weight stages are being multiplied).
 __device__ __forceinline__ void vec_wait(const Shared &S, unsigned seq) {
