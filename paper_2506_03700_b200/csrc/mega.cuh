@@ -398,25 +398,35 @@ __device__ __forceinline__ int control_point(const MegaArgs &A, const Shared &S,
     ++pub_no;
     const Pub *pub = A.pub + (pub_no & 1);
     int action;
+    // the new step descriptor is copied into the role's shared copy `d` by one thread (by every lane of a
+    // producer warp: same values), and checked before anything is indexed with it
+    auto fetch = [&]() -> int {
+        int act = aborted(S) ? ACT_STOP : *(volatile const int *)&pub->action;
+        if (act == ACT_NEWSTEP) {
+            const volatile int *src = reinterpret_cast<const volatile int *>(&pub->d);
+            int *dst = reinterpret_cast<int *>(&d);
+#pragma unroll
+            for (int i = 0; i < (int)(sizeof(StepDesc) / 4); ++i) dst[i] = src[i];
+            if (d.n_cols < 1 || d.n_cols > MAX_COLS || d.newest < 0 || d.newest >= MAX_COLS || d.pmax < 0 || d.pmax >= A.c.max_seq)
+                act = ACT_STOP;   // cannot happen unless memory was corrupted; never index with it
+        }
+        return act;
+    };
     if (ROLE == 2) {
-        if (blockIdx.x == 0) control_cta0(A, sm, kind, e, pub_no, d, steps_started);
+        if (blockIdx.x == 0) {
+            control_cta0(A, sm, kind, e, pub_no, d, steps_started);
+            bar_consumers();   // every thread is done with the old descriptor before thread 0 replaces it
+        }
         if (threadIdx.x == 0) {
             grid_wait(S, &pub->seq, pub_no);
-            sm->bcast[1] = aborted(S) ? ACT_STOP : *(volatile const int *)&pub->action;
+            sm->bcast[1] = fetch();
         }
         bar_consumers();
         action = sm->bcast[1];
     } else {
         grid_wait(S, &pub->seq, pub_no);
-        action = aborted(S) ? ACT_STOP : *(volatile const int *)&pub->action;
-    }
-    if (action == ACT_NEWSTEP) {
-        const volatile int *src = reinterpret_cast<const volatile int *>(&pub->d);
-        int *dst = reinterpret_cast<int *>(&d);
-#pragma unroll
-        for (int i = 0; i < (int)(sizeof(StepDesc) / 4); ++i) dst[i] = src[i];
-        if (d.n_cols < 1 || d.n_cols > MAX_COLS || d.newest < 0 || d.newest >= MAX_COLS || d.pmax < 0 || d.pmax >= A.c.max_seq)
-            action = ACT_STOP;   // cannot happen unless memory was corrupted; never index with it
+        action = fetch();
+        __syncwarp();
     }
     return action;
 }
@@ -513,6 +523,12 @@ __device__ __forceinline__ void attn_merge_to(const float (&o)[NT][4], const flo
 // [16 qr, 16 qr + 16).  K and V rows of the columns processed in this pass are not in the cache
 // yet: they are rotated / rounded here from the QKV output, patched into the shared-memory copy
 // and written to the cache by the item that owns their position.
+// x / group for the q heads per kv head the persistent path admits (1..4) and x < 128, without the
+// general integer division (some thirty of those sat on the critical path of every attention item)
+__device__ __forceinline__ int div_group(int x, int group) {
+    return group == 4 ? x >> 2 : group == 2 ? x >> 1 : group == 1 ? x : (x * 43) >> 7;
+}
+
 template <int HD>
 __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, unsigned mask, Rings &r) {
     const Ctx &c = A.c;
@@ -544,7 +560,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
         for (int u = 0; u < QPT; ++u) {
             const int idx = tid + u * CONS_THREADS;
             const int qcol = idx / HALF, jj = idx - qcol * HALF;
-            const int cc = qcol / group, g = qcol - cc * group;
+            const int cc = div_group(qcol, group), g = qcol - cc * group;
             qx0[u] = 0.f; qx1[u] = 0.f; qco[u] = 1.f; qsi[u] = 0.f;
             if (cc < MAX_COLS && ((mask >> cc) & 1u)) {
                 const float *q = A.qkvraw + (size_t)cc * c.qkv_rows + (size_t)(kvh * group + g) * HD;
@@ -600,18 +616,19 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             }
         }
         bar_consumers();
+        if (tid == 0) trace(S, EV_ATT, 2);   // queries ready
         // ---- per-warp online softmax state: rows (lane/4) and (lane/4)+8 of query tile mt
         int lim[2];
 #pragma unroll
         for (int rh = 0; rh < 2; ++rh) {
-            const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = qcol / group;
+            const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = div_group(qcol, group);
             lim[rh] = (cc < MAX_COLS && ((mask >> cc) & 1u)) ? d.pos[cc] : -1;
         }
         // a query tile none of whose 16 (column, q head) pairs is in use does no arithmetic (uniform per warp)
         bool tile_used = false;
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
-            const int cc = (mt * 16 + q) / group;
+            const int cc = div_group(mt * 16 + q, group);
             tile_used = tile_used || (cc < MAX_COLS && ((mask >> cc) & 1u));
         }
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
@@ -762,6 +779,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 1);
             l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 2);
         }
+        if (tid == 0) trace(S, EV_ATT, 5);   // sub-blocks done
         bar_consumers();   // every warp is done with the query fragments, whose space the merge reuses
         if (qr & 1) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
         bar_consumers();
@@ -774,7 +792,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             // ---- chunk partial (unnormalised output, max, sum) of every valid (column, q head)
 #pragma unroll
             for (int rh = 0; rh < 2; ++rh) {
-                const int qcol = mt * 16 + (lane >> 2) + 8 * rh, cc = qcol / group, g = qcol - cc * group;
+                const int qcol = mt * 16 + (lane >> 2) + 8 * rh, cc = div_group(qcol, group), g = qcol - cc * group;
                 if (cc < MAX_COLS && ((mask >> cc) & 1u) && d.pos[cc] >= p_base) {
                     float *out = A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + j) * ATT_STRIDE;
 #pragma unroll
@@ -798,7 +816,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             // ascending order, eight at a time with all their loads in flight, by the usual running-max rule.
             const int nqc = MAX_COLS * group;
             for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
-                const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = qcol / group, g = qcol - cc * group;
+                const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = div_group(qcol, group), g = qcol - cc * group;
                 if (!((mask >> cc) & 1u)) continue;
                 const int h = kvh * group + g;
                 const int nch = d.pos[cc] / ATT_CHUNK + 1;
@@ -870,10 +888,17 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     // CTAs that share the tiles of each kind of GEMM (the rest idle through that phase)
     const int n_qkv = balanced_ctas((c.qkv_rows + 15) / 16, G), n_d = balanced_ctas(ntd, G), n_gu = balanced_ctas(c.dff / 16, G),
               n_head = balanced_ctas((c.vocab + 15) / 16, G);
-    StepDesc d;
-    d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0; d.fresh = 0; d.run_final = 1;
+    // The step descriptor lives in shared memory, one copy per role (the roles pass a control point at
+    // different times): indexed by a run-time column it would otherwise sit in local memory, whose
+    // cached lines do not survive the acquire of a grid barrier -- every first touch after a barrier
+    // then costs a round trip to L2 on the critical path.
+    StepDesc &d = *reinterpret_cast<StepDesc *>(sm->desc[ROLE]);
+    if (ROLE != 2 || threadIdx.x == 0) {
+        d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0; d.fresh = 0; d.run_final = 1;
 #pragma unroll
-    for (int i = 0; i < MAX_COLS; ++i) { d.first_layer[i] = INT_MAX; d.pos[i] = 0; }
+        for (int i = 0; i < MAX_COLS; ++i) { d.first_layer[i] = INT_MAX; d.pos[i] = 0; }
+    }
+    if (ROLE == 2) bar_consumers(); else __syncwarp();
 
     // barrier between phases, per role; CTA 0 books the time since the previous one to the phase's class
     unsigned long long t_last = gtime();

@@ -50,6 +50,7 @@ struct Smem {                                    // must start on a 1024-byte bo
     alignas(16) unsigned char scratch[SCRATCH_BYTES];
     alignas(16) float vec[64];                    // per-column scalars (rstd, ...)
     alignas(8) unsigned long long w_full[NW], w_empty[NW], x_full[NX], x_empty[NX];
+    alignas(16) int desc[3][32];                  // per-role copy of the step descriptor (persistent decode kernel)
     int abort;
     int bcast[8];
     unsigned trace_n;
@@ -164,7 +165,7 @@ struct Shared {            // what every role needs to wait safely
 };
 
 constexpr int EV_PHASE_BEGIN = 1, EV_X0 = 2, EV_W0 = 3, EV_MAIN_END = 4, EV_EPI_END = 5, EV_WP_BEGIN = 6, EV_WP_END = 7,
-              EV_ITEM = 8, EV_COMBINE = 9, EV_ARRIVE = 10;
+              EV_ITEM = 8, EV_COMBINE = 9, EV_ARRIVE = 10, EV_ATT = 14;
 
 __device__ __forceinline__ void trace(const Shared &S, int ev, int arg) {
     if (S.tr_on && S.tr.buf) {
