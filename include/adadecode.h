@@ -192,6 +192,15 @@ int ada_debug_trace(ada_session *s, uint64_t *dev_buf, uint32_t *count_dev, uint
  * bytes, 256-byte aligned.  The product is launched `repeat` >= 1 times back to back inside one
  * kernel; *ms_out (nullable) receives the device time of that kernel.  All pointers except ms_out
  * are device pointers.  Returns ADA_ETIMEOUT if a bounded device-side wait expired. */
+/* Host-only: how the streaming GEMM of shape N x K (mode as in ada_debug_gemm) divides its work
+ * over `grid` CTAs, for CTA `cta`.  out9 (host) receives {split, t0, t1, n, ta, tb, s0_own_k0,
+ * s0_pub_k1, sl_k1}: split == 0: whole 16-row tiles [t0, t1); split == 1 (only if `split` is
+ * nonzero and the shape allows it): one group of n tile slots, slot s holding tile ta + s, where
+ * slot 0 multiplies k chunks >= s0_own_k0 of its tile and, before them, chunks < s0_pub_k1 of
+ * tile tb (published to the next CTA), and the last slot (if not slot 0) only chunks < sl_k1.
+ * A k chunk is 512 wide.  No GPU is touched.  ADA_EINVAL on bad arguments. */
+int ada_debug_gemm_plan(int32_t N, int32_t K, int32_t mode, int32_t grid, int32_t cta, int32_t split, int32_t *out9);
+
 size_t ada_debug_gemm_work_bytes(int32_t K);
 int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols,
                    void *work_dev, size_t work_bytes, float *Y_dev, int32_t ldy, int32_t repeat, void *cuda_stream,

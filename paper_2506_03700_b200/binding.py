@@ -27,7 +27,7 @@ EXPORTS = [
     "ada_session_create", "ada_session_destroy", "ada_session_reset", "ada_prefill", "ada_plain_decode",
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
-    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace", "ada_gemm_noalloc",
+    "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_plan", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace", "ada_gemm_noalloc",
 ]
 
 
@@ -108,6 +108,7 @@ def load() -> C.CDLL:
         L.ada_gemm_noalloc.argtypes = [vp, i32, i32, i32, vp, i32, vp, i32, vp]
         L.ada_debug_profile.argtypes = [vp, i32]
         L.ada_debug_profile_read.argtypes = [vp, vp, vp, vp]
+        L.ada_debug_gemm_plan.argtypes = [i32, i32, i32, i32, i32, i32, C.POINTER(i32)]
         L.ada_debug_gemm_work_bytes.restype = sz
         L.ada_debug_gemm_work_bytes.argtypes = [i32]
         L.ada_debug_gemm.argtypes = [vp, i32, i32, i32, vp, i32, vp, sz, vp, i32, i32, vp, C.POINTER(C.c_float)]
@@ -118,6 +119,14 @@ def load() -> C.CDLL:
 def _ck(rc: int, where: str):
     if rc != 0:
         raise AdaError(rc, where)
+
+
+def debug_gemm_plan(N: int, K: int, mode: int, grid: int, cta: int, split: bool = True) -> dict:
+    """ada_debug_gemm_plan: the share of CTA `cta` of `grid` in the streaming GEMM (host only, no GPU)."""
+    out = (C.c_int32 * 9)()
+    _ck(load().ada_debug_gemm_plan(N, K, mode, grid, cta, 1 if split else 0, out), "ada_debug_gemm_plan")
+    keys = ("split", "t0", "t1", "n", "ta", "tb", "s0_own_k0", "s0_pub_k1", "sl_k1")
+    return dict(zip(keys, list(out)))
 
 
 def debug_gemm(W, X, mode: int = 0, repeat: int = 1):

@@ -127,11 +127,15 @@ namespace {
 // Scratch layout (all offsets 256-byte aligned).
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
-        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qkvraw, attn_cnt, rope_freq,
+        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qkvraw, attn_cnt, rope_freq, part,
         grid_ctr, pub, err, total;
 };
 
 int rows_alloc_for(int batch, int max_early) { return std::max(batch * (max_early + 1), 32); }
+
+// exchange area of weight tiles split between two CTAs: 8 k-splits x 256 tagged words per CTA
+constexpr size_t kPartBytesPerCta = (size_t)st::CONS_WARPS * 256 * sizeof(unsigned long long);
+constexpr int kPartMaxGrid = 256;
 
 Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, int head_blocks) {
     Layout L{};
@@ -176,6 +180,7 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
         L.qkvraw = take(sizeof(float) * (size_t)st::MAX_COLS * qkv_rows);
         L.attn_cnt = take(sizeof(unsigned) * g.n_kv_heads);
         L.rope_freq = take(sizeof(double) * (g.head_dim / 2));
+        L.part = take(kPartBytesPerCta * kPartMaxGrid);
         L.grid_ctr = take(256);
         L.pub = take(sizeof(mg::Pub) * 2);
         L.err = take(256);
@@ -485,6 +490,7 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.head_part = S->c.head_part;
     a.attn_cnt = (unsigned *)(b + lay.attn_cnt);
     a.rope_freq = (const double *)(b + lay.rope_freq);
+    a.part = S->grid <= kPartMaxGrid ? (unsigned long long *)(b + lay.part) : nullptr;
     a.grid_ctr = (unsigned *)(b + lay.grid_ctr);
     a.pub = (mg::Pub *)(b + lay.pub);
     a.err = (int *)(b + lay.err);
@@ -533,6 +539,7 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
         if (guard > (1ll << 24)) return ADA_ETIMEOUT;
         CK(cudaMemsetAsync(a.grid_ctr, 0, sizeof(unsigned), S->stream));
         CK(cudaMemsetAsync(a.pub, 0, sizeof(mg::Pub) * 2, S->stream));
+        if (a.part) CK(cudaMemsetAsync(a.part, 0, kPartBytesPerCta * (size_t)S->grid, S->stream));
         void *params[] = {(void *)&a};
         CK(cudaLaunchCooperativeKernel(kern, dim3(S->grid), dim3(st::THREADS), params, st::SMEM_BYTES, S->stream));
         S->launches++;
@@ -1077,9 +1084,23 @@ int ada_debug_trace(ada_session *S, uint64_t *dev_buf, uint32_t *count_dev, uint
     return ADA_OK;
 }
 
+int ada_debug_gemm_plan(int32_t N, int32_t K, int32_t mode, int32_t grid, int32_t cta, int32_t split, int32_t *out9) {
+    if (!out9 || N < 1 || K < 64 || K % 64 || mode < 0 || mode > 1 || grid < 1 || cta < 0 || cta >= grid) return ADA_EINVAL;
+    if (mode == 1 && (N % 2 || (N / 2) % 16)) return ADA_EINVAL;
+    st::Gemm g;
+    memset(&g, 0, sizeof(g));
+    g.N = N; g.K = K; g.pair = mode == 1 ? 2 : 1; g.half = mode == 1 ? N / 2 : 0; g.ctas = grid;
+    static unsigned long long dummy;
+    g.part = split ? &dummy : nullptr;   // only tested for null by the plan
+    const st::Plan p = st::make_plan(g, cta, grid);
+    const int32_t v[9] = {p.split, p.t0, p.t1, p.n, p.ta, p.tb, p.s0_own_k0, p.s0_pub_k1, p.sl_k1};
+    memcpy(out9, v, sizeof(v));
+    return ADA_OK;
+}
+
 size_t ada_debug_gemm_work_bytes(int32_t K) {
     if (K < 64) return 0;
-    return st::xfrag_bytes(K) + 512;
+    return st::xfrag_bytes(K) + 512 + kPartBytesPerCta * kPartMaxGrid + 256;
 }
 
 int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols, void *work_dev,
@@ -1108,7 +1129,10 @@ int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const 
     CK(cudaEventCreate(&e0));
     CK(cudaEventCreate(&e1));
     cudaEventRecord(e0, stream);
-    k_gemm_probe<<<sms, st::THREADS, st::SMEM_BYTES, stream>>>(dmap, N, K, mode, (const uint4 *)work_dev, Y_dev, ldy, cols, repeat, err);
+    unsigned long long *part = (unsigned long long *)((char *)work_dev + st::xfrag_bytes(K) + 512);
+    if (sms > kPartMaxGrid || repeat != 1) part = nullptr;
+    else CK(cudaMemsetAsync(part, 0, kPartBytesPerCta * (size_t)sms, stream));
+    k_gemm_probe<<<sms, st::THREADS, st::SMEM_BYTES, stream>>>(dmap, N, K, mode, (const uint4 *)work_dev, Y_dev, ldy, cols, repeat, err, part);
     cudaError_t le = cudaGetLastError();
     cudaEventRecord(e1, stream);
     int herr = 0;
@@ -1167,7 +1191,7 @@ int ada_gemm_noalloc(const void *W_dev, int32_t N, int32_t K, int32_t mode, cons
     CK(cudaStreamSynchronize(stream));   // hmap lives on this stack frame
     k_xfrag_pack<<<(K + 255) / 256, 256, 0, stream>>>(X_dev, K, cols, (__nv_bfloat16 *)base);
     CK(cudaGetLastError());
-    k_gemm_probe<<<sms_of_device[dev], st::THREADS, st::SMEM_BYTES, stream>>>(dmap, N, K, mode, (const uint4 *)base, Y_dev, ldy, cols, 1, err);
+    k_gemm_probe<<<sms_of_device[dev], st::THREADS, st::SMEM_BYTES, stream>>>(dmap, N, K, mode, (const uint4 *)base, Y_dev, ldy, cols, 1, err, nullptr);
     CK(cudaGetLastError());
     int herr = 0;
     CK(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, stream));

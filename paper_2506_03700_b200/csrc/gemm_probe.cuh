@@ -17,7 +17,7 @@ __global__ void k_xfrag_pack(const float *__restrict__ X, int K, int cols, __nv_
 // mode 1: Y[col][n] = silu(g) * u, g = W[n].X, u = W[half + n].X     (half = N/2 rows of each)
 __global__ void __launch_bounds__(st::THREADS, 1)
 k_gemm_probe(const CUtensorMap *__restrict__ W, int N, int K, int mode, const uint4 *__restrict__ X, float *__restrict__ Y,
-             int ldy, int cols, int repeat, int *err) {
+             int ldy, int cols, int repeat, int *err, unsigned long long *part) {
     extern __shared__ unsigned char smem_raw[];
     st::Smem *sm = st::smem_base(smem_raw);
     st::smem_init(sm);
@@ -27,6 +27,8 @@ k_gemm_probe(const CUtensorMap *__restrict__ W, int N, int K, int mode, const ui
     g.W = W; g.X = X; g.N = N; g.K = K; g.pair = mode == 1 ? 2 : 1; g.half = mode == 1 ? N / 2 : 0;
     g.ctas = st::balanced_ctas(g.tiles(), gridDim.x);
     g.cp0 = 0; g.ncp = (cols + 1) / 2;
+    // tiles split between CTAs need a grid-wide meeting between products: only for a single product
+    g.part = repeat == 1 ? part : nullptr; g.phase_id = 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x, G = gridDim.x;
     st::Rings r{0, 0};

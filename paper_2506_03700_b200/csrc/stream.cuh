@@ -297,6 +297,14 @@ struct Gemm {
     const uint4 *X;
     int N, K, pair, half;
     int ctas;   // CTAs 0 .. ctas-1 share the tiles (see balanced_ctas); 0 = the whole grid
+    // Exchange area for tiles split between two CTAs (null: whole tiles only): [grid][CONS_WARPS][8][32]
+    // words of 8 bytes, each a partial sum (low half) tagged with the phase that wrote it (high half).
+    // A word is written and read by one 8-byte access, so a reader that sees the tag sees the sum:
+    // no fence is needed on either side (a fence in the middle of the stream stalls the publishing
+    // warp, and with it the whole ring, for microseconds).  phase_id is unique per GEMM of a launch
+    // and never 0; the area is zeroed before each launch.
+    unsigned long long *part;
+    unsigned phase_id;
     int cp0, ncp;   // column pairs cp0 .. cp0+ncp-1 of the activations are fetched
     __device__ __forceinline__ void columns(unsigned mask) {   // the pairs spanning the columns set in `mask`
         if (mask == 0) { cp0 = 0; ncp = 1; return; }
@@ -307,16 +315,88 @@ struct Gemm {
     // ring holds three stages; with one chunk per stage a CTA that owns two weight tiles would wait
     // for an activation copy every 96 KB of weights.)
     __device__ __forceinline__ int xchunks() const { return ncp == 1 ? 4 : ncp == 2 ? 2 : 1; }
-    __device__ __forceinline__ int tiles() const { return pair == 2 ? half / TILE_N : (N + TILE_N - 1) / TILE_N; }
+    __host__ __device__ __forceinline__ int tiles() const { return pair == 2 ? half / TILE_N : (N + TILE_N - 1) / TILE_N; }
 };
 
 struct Rings { uint32_t wi, xi; };   // stage counters of one role (slot = i % N, parity = (i / N) & 1)
 
-__device__ __forceinline__ void cta_tile_range(int T, int cta, int G, int &t0, int &t1) {
+__host__ __device__ __forceinline__ void cta_tile_range(int T, int cta, int G, int &t0, int &t1) {
     if (cta >= G) { t0 = t1 = 0; return; }
     t0 = (int)((long long)T * cta / G);
     t1 = (int)((long long)T * (cta + 1) / G);
 }
+// ---------------------------------------------------------------- unit-balanced split of a GEMM
+// With whole tiles some CTAs stream one tile more than the others (7 against 6 in the 8B gate-up
+// GEMM) and the phase lasts as long as they do.  When g.part is set the work is instead measured in
+// units of (tile, k chunk): CTA c takes the units [U c / C, U (c + 1) / C) of the tile-major order,
+// so every CTA streams the same number of stages (+- one).  A tile cut by a CTA boundary is
+// computed in two parts.  The CTA with its chunks from 0 (the head part, [0, kb)) meets them early
+// in its k loop and publishes its partial sums as soon as they are complete; the CTA with the later
+// chunks (the tail part, [ka, nch)) finishes them at the end of its loop, adds the published part
+// (own + published, the published k-splits in index order: the sum does not depend on timing) and
+// runs the epilogue.  All tiles of a CTA, partial ones included, form one group that shares every
+// activation chunk; when the head part ends before the tail part begins they take turns in slot 0.
+// GEMMs with fewer units per CTA than chunks per tile, or more tiles per CTA than consumer warps,
+// keep whole tiles.  The plan is a function of the GEMM's shape and the grid only.
+struct Plan {
+    int split;       // 0: whole tiles [t0, t1) in groups of CONS_WARPS
+    int t0, t1;
+    // split: one group of n slots; slot s holds tile ta + s, except that
+    int n, ta, tb;
+    int s0_own_k0;   //   slot 0 multiplies its own tile from chunk s0_own_k0 on (0: a whole tile),
+    int s0_pub_k1;   //   and before that the chunks below s0_pub_k1 of tile tb, to publish (0: none);
+    int sl_k1;       //   the last slot (if not slot 0) multiplies chunks below sl_k1 only, to publish (nch: a whole tile)
+};
+__host__ __device__ __forceinline__ Plan make_plan(const Gemm &g, int cta, int G) {
+    Plan p;
+    p.split = 0;
+    p.t0 = p.t1 = p.n = p.ta = p.tb = p.s0_own_k0 = p.s0_pub_k1 = 0;
+    const int C = g.ctas > 0 ? g.ctas : G, T = g.tiles(), nch = (g.K + KC - 1) / KC;
+    p.sl_k1 = nch;
+    if (cta < 0 || cta >= C) return p;
+    // 32-bit arithmetic throughout (a 64-bit division costs hundreds of cycles); GEMMs whose unit
+    // count times the CTA count does not fit keep whole tiles
+    const unsigned U = (unsigned)T * (unsigned)nch;
+    const bool fits = (unsigned long long)T * nch * (unsigned)(C + 1) < 0x7fffffffull;
+    const unsigned L = (U + C - 1) / C;      // most units of one CTA; a run of L units touches <= (L + nch - 2) / nch + 1 tiles
+    if (!g.part || !fits || U / C < (unsigned)nch || (L + nch - 2) / nch + 1 > (unsigned)CONS_WARPS) {
+        cta_tile_range(T, cta, C, p.t0, p.t1);
+        return p;
+    }
+    p.split = 1;
+    const unsigned u0 = U * (unsigned)cta / C, u1 = U * (unsigned)(cta + 1) / C;
+    p.ta = (int)(u0 / nch);
+    p.tb = (int)((u1 - 1) / nch);
+    const int ka = (int)(u0 - p.ta * nch), kb = (int)((u1 - 1) - p.tb * nch) + 1;
+    const bool has_tail = ka > 0, has_head = kb < nch;
+    const bool shared = has_tail && has_head && kb <= ka;
+    p.s0_own_k0 = ka;
+    p.n = p.tb - p.ta + 1;
+    if (shared) { p.s0_pub_k1 = kb; p.n -= 1; }
+    else if (has_head) p.sl_k1 = kb;
+    return p;
+}
+// the tile slot s of a split plan multiplies at chunk kc (-1: none)
+__host__ __device__ __forceinline__ int plan_tile(const Plan &p, int s, int kc) {
+    if (s == 0) return kc < p.s0_pub_k1 ? p.tb : (kc >= p.s0_own_k0 ? p.ta : -1);
+    if (s == p.n - 1 && kc >= p.sl_k1) return -1;
+    return p.ta + s;
+}
+// the k-splits of a group of ng slots
+__host__ __device__ __forceinline__ int group_ks(int ng) {
+    int TS = 1;
+    while (TS < ng) TS <<= 1;
+    return CONS_WARPS / TS;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 // How many CTAs share the tiles of a GEMM: all of them.  (With its consumers attached one SM
 // sustains about 45 GB/s through the ring, roughly its fair share of HBM with all 148 SMs
 // streaming; giving equal tile counts to fewer CTAs was measured and lost more than the uneven
@@ -327,24 +407,31 @@ __host__ __device__ inline int balanced_ctas(int T, int G) { (void)T; return G; 
 __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol) {
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31;
-    int t0, t1;
-    cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
+    const Plan pl = make_plan(g, cta, G);
     const int nch = (g.K + KC - 1) / KC;
     if (lane == 0) trace(S, EV_WP_BEGIN, 0);
-    for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
-        const int ng = min(CONS_WARPS, t1 - g0);
-        for (int kc = 0; kc < nch; ++kc) {
-            for (int s = 0; s < ng; ++s) {
-                for (int p = 0; p < g.pair; ++p) {
-                    const int slot = r.wi % NW;
-                    mbar_wait(S, &sm->w_empty[slot], ((r.wi / NW) & 1) ^ 1);
-                    if (lane == 0 && !aborted(S)) {
-                        mbar_expect_tx(&sm->w_full[slot], (uint32_t)W_STAGE);
-                        tma_load_3d(sm->w[slot], g.W, 0, (g0 + s) * TILE_N + p * g.half, kc * KG, &sm->w_full[slot], pol);
-                    }
-                    ++r.wi;
-                }
+    auto stage = [&](int tile, int p, int kc) {
+        const int slot = r.wi % NW;
+        mbar_wait(S, &sm->w_empty[slot], ((r.wi / NW) & 1) ^ 1);
+        if (lane == 0 && !aborted(S)) {
+            mbar_expect_tx(&sm->w_full[slot], (uint32_t)W_STAGE);
+            tma_load_3d(sm->w[slot], g.W, 0, tile * TILE_N + p * g.half, kc * KG, &sm->w_full[slot], pol);
+        }
+        ++r.wi;
+    };
+    if (pl.split) {
+        for (int kc = 0; kc < nch; ++kc)
+            for (int s = 0; s < pl.n; ++s) {
+                const int tile = plan_tile(pl, s, kc);
+                if (tile < 0) continue;
+                for (int p = 0; p < g.pair; ++p) stage(tile, p, kc);
             }
+    } else {
+        for (int g0 = pl.t0; g0 < pl.t1; g0 += CONS_WARPS) {
+            const int ng = min(CONS_WARPS, pl.t1 - g0);
+            for (int kc = 0; kc < nch; ++kc)
+                for (int s = 0; s < ng; ++s)
+                    for (int p = 0; p < g.pair; ++p) stage(g0 + s, p, kc);
         }
     }
     if (lane == 0) trace(S, EV_WP_END, 0);
@@ -357,12 +444,12 @@ template <class Hook>
 __device__ __forceinline__ void gemm_produce_x(const Shared &S, const Gemm &g, int cta, int G, Rings &r, uint64_t pol, Hook &&after_first) {
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31;
-    int t0, t1;
-    cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
+    const Plan pl = make_plan(g, cta, G);
     const int nch = (g.K + KC - 1) / KC;
     const int XC = g.xchunks();
+    const int ngroups = pl.split ? (pl.n > 0 ? 1 : 0) : (pl.t1 - pl.t0 + CONS_WARPS - 1) / CONS_WARPS;
     bool hooked = false;
-    for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
+    for (int gi = 0; gi < ngroups; ++gi) {
         for (int kc = 0; kc < nch; kc += XC) {
             const int nc = min(XC, nch - kc);
             const int slot = r.xi % NX;
@@ -426,19 +513,26 @@ template <int PAIR, class Pre, class Epi>
 __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int cta, int G, Rings &r, Pre &&pre, Epi &&epi) {
     Smem *sm = S.sm;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int t0, t1;
-    cta_tile_range(g.tiles(), cta, g.ctas > 0 ? g.ctas : G, t0, t1);
     const int nch = (g.K + KC - 1) / KC, XC = g.xchunks();
+    bool first_group = true;
     // ldmatrix source of this lane inside a stage: row (lane%8) + 8 ((lane/8)%2), 16-byte chunk lane/16 of the k-step
     const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
     const int a_off = a_row * 128, a_hi = lane >> 4, a_sw = a_row & 7;
-    for (int g0 = t0; g0 < t1; g0 += CONS_WARPS) {
-        const int ng = min(CONS_WARPS, t1 - g0);
+    // One group of ng tile slots; slot s holds tile g0 + s.  Whole tiles: s0_own_k0 = s0_pub_k1 = 0,
+    // sl_k1 = nch.  The group of a split plan: see Plan; ksp = k-splits of the CTA before (0: no tail part).
+    auto group = [&](int g0, int ng, int s0_own_k0, int s0_pub_k1, int sl_k1, int ksp, bool last_group) {
         int TS = 1;
         while (TS < ng) TS <<= 1;
         const int KS = CONS_WARPS / TS;
         const int slot_id = warp % TS, ks_id = warp / TS;
-        if (ks_id == 0 && slot_id < ng) pre(g0 + slot_id);
+        const bool mine = slot_id < ng;
+        const bool pub_only = slot_id > 0 && slot_id == ng - 1 && sl_k1 < nch;
+        // this warp's slot: chunks below my_pub_k1 go to the published part, chunks from my_own_k0 to its own tile
+        const int my_pub_k1 = !mine ? 0 : slot_id == 0 ? s0_pub_k1 : pub_only ? sl_k1 : 0;
+        const int my_own_k0 = (!mine || pub_only) ? nch : slot_id == 0 ? s0_own_k0 : 0;
+        const int own_tile = (mine && !pub_only) ? g0 + slot_id : -1;
+        const bool tail = own_tile >= 0 && my_own_k0 > 0;   // the head part of this tile comes from CTA cta - 1
+        if (ks_id == 0 && own_tile >= 0) pre(own_tile);
         float acc[PAIR][4][4];   // [matrix][even/odd step x hi/lo][fragment]
 #pragma unroll
         for (int p = 0; p < PAIR; ++p)
@@ -450,26 +544,30 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
             const int ksteps = min(KC, g.K - kc * KC) >> 4;
             const int xslot = r.xi % NX;
             if (kc % XC == 0) mbar_wait(S, &sm->x_full[xslot], (r.xi / NX) & 1);
-            if (threadIdx.x == 0 && kc == 0 && g0 == t0) trace(S, EV_X0, 0);
+            if (threadIdx.x == 0 && kc == 0 && first_group) trace(S, EV_X0, 0);
             // this lane's column pair, if it was fetched (else any fetched pair: its column is not in use)
             const int xp = min(max((lane >> 3) - g.cp0, 0), g.ncp - 1);
             const uint4 *xs = reinterpret_cast<const uint4 *>(sm->x[xslot]) + ((kc % XC) * g.ncp + xp) * 256 + (lane & 7);
+            // the k-splits of a slot take whole stages in turn, counted from the first chunk of the part
+            // (chunk kc belongs to split (kc - first) mod KS): a warp then multiplies all 32 k-steps of
+            // a stage, which amortises the per-stage waiting and set-up (splitting every stage among
+            // the warps streamed 20-30 % slower)
+            const int kbase = kc < my_pub_k1 ? 0 : my_own_k0;
+            const bool my_turn = mine && ((kc - kbase) & (KS - 1)) == ks_id;
             for (int s = 0; s < ng; ++s) {
+                if (s == 0 ? (kc >= s0_pub_k1 && kc < s0_own_k0) : (s == ng - 1 && kc >= sl_k1)) continue;   // no stage: outside the parts
 #pragma unroll
                 for (int p = 0; p < PAIR; ++p) {
                     const int wslot = r.wi % NW;
-                    // Every warp waits for and releases every stage in order, although only its owners
-                    // use it.  An mbarrier tells phases apart by one parity bit: a warp that ran ahead
+                    // Every warp waits for and releases every stage in order, although only its owner
+                    // uses it.  An mbarrier tells phases apart by one parity bit: a warp that ran ahead
                     // of, or fell behind, the others by a ring would mistake one phase of a slot for
                     // another (releasing stages by their owners alone was tried: a lagging warp then
                     // waits for a refill that needs its own release).  With all eight arrivals per
                     // stage no warp is ever more than one ring away from any other.
                     mbar_wait(S, &sm->w_full[wslot], (r.wi / NW) & 1);
-                    // the k-splits of a tile take whole stages in turn (chunk kc belongs to split kc % KS):
-                    // a warp then multiplies all 32 k-steps of a stage, which amortises the per-stage
-                    // waiting and set-up (splitting every stage among the warps streamed 20-30 % slower)
-                    if (s == slot_id && (kc % KS) == ks_id) {
-                        if (threadIdx.x == 0 && kc == 0 && g0 == t0 && p == 0) trace(S, EV_W0, 0);
+                    if (s == slot_id && my_turn) {
+                        if (threadIdx.x == 0 && kc == 0 && first_group && p == 0) trace(S, EV_W0, 0);
                         const unsigned char *ws = sm->w[wslot] + a_off;
                         if (ksteps == KSTEPS) {   // full chunk: software-pipelined, fully unrolled
                             stage_full<1>(acc[p], ws, xs, 0, a_hi, a_sw);
@@ -495,14 +593,70 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                 if (lane == 0) mbar_arrive(&sm->x_empty[xslot]);
                 ++r.xi;
             }
+            if (kc + 1 == my_pub_k1) {
+                // The head part of a split tile is complete: every k-split warp publishes its own sums
+                // (no meeting inside the CTA in the middle of the stream) and starts over for the tail
+                // part that may follow in this slot.
+                unsigned long long *pb = g.part + (size_t)(cta * CONS_WARPS + ks_id) * 256;
+#pragma unroll
+                for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float v = (acc[p][0][i] + acc[p][1][i]) + (acc[p][2][i] + acc[p][3][i]);
+                        st_relaxed_u64(pb + (p * 4 + i) * 32 + lane, ((unsigned long long)g.phase_id << 32) | __float_as_uint(v));
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) acc[p][q][i] = 0.f;
+                    }
+            }
         }
-        if (threadIdx.x == 0 && g0 + CONS_WARPS >= t1) trace(S, EV_MAIN_END, 0);
+        if (threadIdx.x == 0 && last_group) trace(S, EV_MAIN_END, 0);
+        first_group = false;
         // fold the four partial accumulators in a fixed order: (even.hi + odd.hi) + (even.lo + odd.lo)
         float d[PAIR][4];
 #pragma unroll
         for (int p = 0; p < PAIR; ++p)
 #pragma unroll
             for (int i = 0; i < 4; ++i) d[p][i] = (acc[p][0][i] + acc[p][1][i]) + (acc[p][2][i] + acc[p][3][i]);
+        // The head part published by CTA cta - 1, in ksp k-splits: this slot's k-split warp j fetches
+        // the published splits j, j + KS, ... (all at once: one round trip) and adds them to its own
+        // sums in index order; the fixed-order reduction below then covers both parts.
+        if (tail) {
+            unsigned long long t0 = 0;
+            for (uint32_t it = 0;; ++it) {
+                bool ok = true;
+                float add[PAIR][4];
+#pragma unroll
+                for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) add[p][i] = 0.f;
+                for (int q = ks_id; q < ksp; q += KS) {
+                    const unsigned long long *pb = g.part + (size_t)((cta - 1) * CONS_WARPS + q) * 256;
+#pragma unroll
+                    for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const unsigned long long v = ld_relaxed_u64(pb + (p * 4 + i) * 32 + lane);
+                            ok = ok && (unsigned)(v >> 32) == g.phase_id;
+                            add[p][i] += __uint_as_float((unsigned)v);
+                        }
+                }
+                if (__all_sync(0xffffffffu, ok)) {
+#pragma unroll
+                    for (int p = 0; p < PAIR; ++p)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) d[p][i] += add[p][i];
+                    break;
+                }
+                if ((it & 15u) == 15u) {   // bounded like every other wait on another CTA
+                    bool stop = aborted(S) || *(volatile int *)S.err != 0;
+                    const unsigned long long t = gtime();
+                    if (t0 == 0) t0 = t;
+                    else if (t - t0 > WAIT_NS) { if (lane == 0) raise_error(S, ERR_TIMEOUT_GRID); stop = true; }
+                    if (__any_sync(0xffffffffu, stop)) { *(volatile int *)&S.sm->abort = 1; break; }
+                }
+                __nanosleep(64);
+            }
+        }
         if (KS > 1) {
             float *red = reinterpret_cast<float *>(sm->scratch) + (size_t)warp * (PAIR * 128);
 #pragma unroll
@@ -520,8 +674,18 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                 }
             }
         }
-        if (ks_id == 0 && slot_id < ng) epi(g0 + slot_id, d);
+        if (ks_id == 0 && own_tile >= 0) epi(own_tile, d);
         if (KS > 1) bar_consumers();
+    };
+    {
+        const Plan pl = make_plan(g, cta, G);
+        if (pl.split) {
+            const int ksp = pl.s0_own_k0 > 0 ? group_ks(make_plan(g, cta - 1, G).n) : 0;
+            if (pl.n > 0) group(pl.ta, pl.n, pl.s0_own_k0, pl.s0_pub_k1, pl.sl_k1, ksp, true);
+        } else {
+            for (int g0 = pl.t0; g0 < pl.t1; g0 += CONS_WARPS)
+                group(g0, min(CONS_WARPS, pl.t1 - g0), 0, 0, nch, 0, g0 + CONS_WARPS >= pl.t1);
+        }
     }
 }
 
