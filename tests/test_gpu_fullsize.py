@@ -90,3 +90,97 @@ def test_8b_full_prompt_adaptive_equals_plain_bit_for_bit(big):
             for pos in (0, 700, cfg.prompt_len + 3, cfg.prompt_len + n - 2):
                 assert np.array_equal(S.read_kv(0, l, pos), P.read_kv(0, l, pos))
                 assert np.array_equal(S.read_kv(1, l, pos), P.read_kv(1, l, pos))
+
+
+def test_8b_long_context_adaptive_equals_plain_bit_for_bit(big):
+    """The long-context configuration: an 8192-token prompt (65 attention chunks per kv head, so a
+    CTA takes several work items and the chunk merge folds more partials than it loads at once)."""
+    cfg = synth.CONFIGS["8b-long"]
+    prompt = synth.make_prompt(cfg, seed=91).numpy()
+    assert len(prompt) == 8192
+    n = 40
+    max_seq = cfg.prompt_len + 256
+    P = binding.Session(big.gm, 1, max_seq, 64, 5)
+    assert P.get_path() == 1
+    P.capture_logits(n + 8)
+    P.prefill(prompt)
+    ref = P.plain_decode(n)[0]
+    ref_lg = P.captured_logits()[:n].clone()
+    lp, fp_ = P.state()
+    assert torch.isfinite(ref_lg).all()
+    for gamma, tape in [(cfg.threshold, None), (0.0, [1] * 32)]:
+        S = binding.Session(big.gm, 1, max_seq, 64, 5)
+        S.capture_logits(n + 8)
+        S.prefill(prompt)
+        if tape:
+            S.set_exit_tape(tape)
+        st = binding.Stats()
+        out = S.adaptive_decode(n, gamma, cfg.exit_layers, 5, st)[0]
+        assert np.array_equal(out, ref), gamma
+        assert torch.equal(S.captured_logits()[:n], ref_lg), gamma
+        ls, fs = S.state()
+        assert ls == lp and np.array_equal(fs, fp_)
+        assert st.early_exits == st.accepted + st.rejected + st.discarded
+        assert st.early_exits > 0
+        for l in (0, 31):
+            for pos in (0, 4097, cfg.prompt_len - 1, cfg.prompt_len + n - 2):
+                assert np.array_equal(S.read_kv(0, l, pos), P.read_kv(0, l, pos))
+                assert np.array_equal(S.read_kv(1, l, pos), P.read_kv(1, l, pos))
+    del P, S
+    torch.cuda.empty_cache()
+
+
+def test_13b_shape_adaptive_equals_plain_and_matches_the_oracle_on_a_short_prompt():
+    """The 13B-shaped configuration at batch 1 on the persistent path: multi-head attention (one q
+    head per kv head), d_model 5120, a 13824-wide FFN (27 k chunks), vocabulary 32000."""
+    if torch.cuda.get_device_properties(0).total_memory < 60e9:
+        pytest.skip("needs a GPU with room for the 13B-shaped weights")
+    cfg = synth.CONFIGS["13b"]
+    w = synth.make_weights(cfg, seed=77, device="cuda")
+    gm = binding.Model(cfg, w)
+    for l in cfg.exit_layers:
+        gm.set_exit_head(l, None, cfg.logit_scale)
+    prompt = synth.make_prompt(cfg, n=200, seed=5).numpy()
+    n = 48
+    P = binding.Session(gm, 1, 512, 64, 5)
+    assert P.get_path() == 1
+    P.capture_logits(n + 8)
+    P.prefill(prompt)
+    ref = P.plain_decode(n)[0]
+    ref_lg = P.captured_logits()[:n].clone()
+    lp, fp_ = P.state()
+    assert torch.isfinite(ref_lg).all() and len(set(ref.tolist())) > 4
+    for gamma, tape in [(cfg.threshold, None), (0.3, None), (0.0, [1] * 32)]:
+        S = binding.Session(gm, 1, 512, 64, 5)
+        S.capture_logits(n + 8)
+        S.prefill(prompt)
+        if tape:
+            S.set_exit_tape(tape)
+        st = binding.Stats()
+        out = S.adaptive_decode(n, gamma, cfg.exit_layers, 5, st)[0]
+        assert np.array_equal(out, ref), gamma
+        assert torch.equal(S.captured_logits()[:n], ref_lg), gamma
+        ls, fs = S.state()
+        assert ls == lp and np.array_equal(fs, fp_)
+        assert st.early_exits == st.accepted + st.rejected + st.discarded
+    del P, S
+    # a short prompt against the oracle (sampled outputs the oracle can compute one by one); the host
+    # copy of the weights takes twice 26 GB for a moment
+    import psutil
+    if psutil.virtual_memory().available < 90e9:
+        del gm, w
+        torch.cuda.empty_cache()
+        pytest.skip("adaptive == plain checked; not enough host memory for the oracle's copy of the 13B-shaped weights")
+    class Pair:
+        pass
+    pr = Pair()
+    pr.cfg, pr.gm = cfg, gm
+    pr.om = oracle.model_from_torch(cfg, {k: v.cpu() for k, v in w.items()})
+    sp = synth.make_prompt(cfg, n=10, seed=6).numpy()
+    Q = binding.Session(gm, 1, 64, 64, 5)
+    Q.capture_logits(8)
+    Q.prefill(sp)
+    out = Q.plain_decode(3)[0]
+    check_against_oracle(pr, sp, out, Q.captured_logits().cpu().numpy())
+    del Q, gm, w, pr
+    torch.cuda.empty_cache()
