@@ -70,9 +70,6 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(bar)) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_n(unsigned long long *bar, uint32_t n) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(s32(bar)), "r"(n) : "memory");
-}
 __device__ __forceinline__ bool mbar_try(unsigned long long *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
