@@ -908,8 +908,9 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             barrier_consumers(S, A.grid_ctr, bar_no, G, cls);
             if (blockIdx.x == 0 && threadIdx.x == 0) {
                 const unsigned long long t = gtime();
-                c.st->st.phase_ns[cls] += (long long)(t - t_last);
-                c.st->st.phase_count[cls] += 1;
+                // reductions, not read-modify-write: thread 0 of CTA 0 must not wait for a load from L2 at every barrier
+                atomicAdd(reinterpret_cast<unsigned long long *>(&c.st->st.phase_ns[cls]), t - t_last);
+                atomicAdd(reinterpret_cast<unsigned long long *>(&c.st->st.phase_count[cls]), 1ull);
                 t_last = t;
             }
         } else ++bar_no;
@@ -917,8 +918,8 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     auto book_control = [&]() {
         if (ROLE == 2 && blockIdx.x == 0 && threadIdx.x == 0) {
             const unsigned long long t = gtime();
-            c.st->st.phase_ns[0] += (long long)(t - t_last);
-            c.st->st.phase_count[0] += 1;
+            atomicAdd(reinterpret_cast<unsigned long long *>(&c.st->st.phase_ns[0]), t - t_last);
+            atomicAdd(reinterpret_cast<unsigned long long *>(&c.st->st.phase_count[0]), 1ull);
             t_last = t;
         }
     };
