@@ -144,10 +144,20 @@ __device__ __forceinline__ void barrier_consumers(const Shared &S, unsigned *ctr
 __device__ __forceinline__ HeadResult merge_head(const float *head_part, int G, int col) {
     const int lane = threadIdx.x & 31;
     Msa a; a.m = -INFINITY; a.s = 0.f; a.i = INT_MAX;
-    for (int b = lane; b < G; b += 32) {
-        const float *o = head_part + ((size_t)b * MAX_COLS + col) * 4;
-        Msa x; x.m = ldcg(o); x.s = ldcg(o + 1); x.i = __float_as_int(ldcg(o + 2));
-        a = msa_merge(a, x);
+    for (int b0 = lane; b0 < G; b0 += 32 * 8) {   // eight CTAs' partials in flight per lane, merged in ascending order
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int b = b0 + 32 * u;
+            v[u] = b < G ? __ldcg(reinterpret_cast<const float4 *>(head_part + ((size_t)b * MAX_COLS + col) * 4)) : make_float4(-INFINITY, 0.f, __int_as_float(INT_MAX), 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (b0 + 32 * u < G) {
+                Msa x; x.m = v[u].x; x.s = v[u].y; x.i = __float_as_int(v[u].z);
+                a = msa_merge(a, x);
+            }
+        }
     }
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -166,69 +176,95 @@ __device__ __forceinline__ HeadResult merge_head(const float *head_part, int G, 
 // Applies the outcome of the step that just ended (Eq. 1 after a head; verification and rollback,
 // Eq. 2 at temperature zero, after the final head), then sets up the next step: its columns, the
 // embedding of its newest token, that token's rotary table; finally publishes the action.
-__device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind, int e, unsigned pub_no, const StepDesc &dprev,
+__device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind, int e, unsigned pub_no, const StepDesc &dprev,
                                           int &steps_started) {
     const Ctx &c = A.c;
     DevState *st = c.st;
     const MegaModel &M = *A.mm;
     const int tid = threadIdx.x, G = gridDim.x;
     Pub *pub = A.pub + (pub_no & 1);
+    // Shared-memory copies for the bookkeeping thread (fetched by many threads at once: a single
+    // thread reading them from global memory one after the other spent 30 us here on round trips to L2):
+    // the fill levels, the head results, and the tokens the verification compares with.
+    int *fill_s = reinterpret_cast<int *>(sm->scratch);                                // [L]
+    HeadResult *hr_s = reinterpret_cast<HeadResult *>(sm->scratch + 1024);             // [MAX_COLS]
+    int *tok_s = reinterpret_cast<int *>(sm->scratch + 1024 + sizeof(HeadResult) * MAX_COLS);   // [MAX_COLS]: tokens base+1 ..
+    for (int l = tid; l < c.L; l += CONS_THREADS) fill_s[l] = c.fill[l];
+    if (tid >= CONS_THREADS - MAX_COLS) {
+        const int j = tid - (CONS_THREADS - MAX_COLS), at = st->base[0] + j + 1;
+        tok_s[j] = at < c.max_seq ? c.tokens[at] : -1;
+    }
     // (a) head results of the columns that matter: warp w merges column w
     if (kind != CTRL_START) {
         const int w = tid >> 5;
         const bool want = kind == CTRL_HEAD ? w == dprev.newest : w < dprev.n_cols;
         if (want) {
             const HeadResult hr = merge_head(A.head_part, G, w);
-            if ((tid & 31) == 0) c.head_res[w] = hr;
+            if ((tid & 31) == 0) { c.head_res[w] = hr; hr_s[w] = hr; }
         }
     }
     __threadfence_block();
     bar_consumers();
-    // (b) bookkeeping, one thread
+    // (b) bookkeeping, one thread.  Every scalar it may need is read up front (the loads overlap);
+    // counters are bumped by reductions, which do not wait for memory.
     if (tid == 0) {
+        auto bump = [](long long *p, long long v) { atomicAdd(reinterpret_cast<unsigned long long *>(p), (unsigned long long)v); };
+        const int err0 = *(volatile int *)A.err;
+        const int len0 = st->len[0], base0 = st->base[0], target0 = st->target_len[0], done0 = st->done[0];
+        const int pf_end0 = st->pf_end, pf_pos0 = st->pf_pos, max_early0 = st->max_early;
+        const int tape_n0 = st->tape_n, tape_i0 = st->tape_i, hl_n0 = st->head_log_n;
+        const float gamma0 = st->gamma;
+        const long long steps0 = __ldcg(&st->st.steps);   // past the L1: the counters are bumped by reductions
         int action = ACT_NEWSTEP, verified = 0;
+        int len = len0, base = base0, done = done0, pf_end = pf_end0, pf_pos = pf_pos0;
         int32_t *tok = c.tokens;
-        if (*(volatile int *)A.err != 0) action = ACT_STOP;
+        if (err0 != 0) action = ACT_STOP;
         if (action != ACT_STOP && kind == CTRL_HEAD) {
-            const int len = st->len[0];
-            const HeadResult hr = c.head_res[dprev.newest];
-            bool decide = hr.p > st->gamma;
-            if (st->tape_i < st->tape_n) {
-                const uint8_t t = st->tape[st->tape_i++];
+            const HeadResult hr = hr_s[dprev.newest];
+            bool decide = hr.p > gamma0;
+            if (tape_i0 < tape_n0) {
+                const uint8_t t = st->tape[tape_i0];
+                st->tape_i = tape_i0 + 1;
                 if (t == 0) decide = false;
                 if (t == 1) decide = true;
             }
-            st->st.head_evals++;
-            if (c.head_log && st->head_log_n < kHeadLogCap) {
-                float *hl = c.head_log + 4 * (size_t)st->head_log_n;
-                hl[0] = (float)st->st.steps; hl[1] = (float)e; hl[2] = (float)hr.token; hl[3] = hr.p;
-                st->head_log_n++;
+            bump(&st->st.head_evals, 1);
+            if (c.head_log && hl_n0 < kHeadLogCap) {
+                float *hl = c.head_log + 4 * (size_t)hl_n0;
+                hl[0] = (float)steps0; hl[1] = (float)e; hl[2] = (float)hr.token; hl[3] = hr.p;
+                st->head_log_n = hl_n0 + 1;
             }
             if (!decide) action = ACT_CONTINUE;
             else {
+                long long rl = 0;
                 for (int l = 0; l < e; ++l) {
-                    st->st.row_layers += len - c.fill[l];
+                    rl += len - fill_s[l];
+                    fill_s[l] = len;
                     c.fill[l] = len;
                 }
+                bump(&st->st.row_layers, rl);
                 tok[len] = min(max(hr.token, 0), c.vocab - 1);
-                st->len[0] = len + 1;
-                st->st.early_exits++;
-                st->st.exits_at_layer[e]++;
-                st->st.steps++;
-                st->st.layer_passes += e;
+                len = len + 1;
+                st->len[0] = len;
+                bump(&st->st.early_exits, 1);
+                bump(&st->st.exits_at_layer[e], 1);
+                bump(&st->st.steps, 1);
+                bump(&st->st.layer_passes, e);
             }
         }
-        const bool prefilling = st->pf_end > 0;
+        const bool prefilling = pf_end > 0;
         if (action != ACT_STOP && kind == CTRL_TOP && prefilling) {
             // a pass over prompt positions [pf_pos, pf_pos + n) is complete at every layer
-            const int n = dprev.n_cols, end = st->pf_pos + n;
-            for (int l = 0; l < c.L; ++l) c.fill[l] = end;
+            const int n = dprev.n_cols, end = pf_pos + n;
+            for (int l = 0; l < c.L; ++l) { fill_s[l] = end; c.fill[l] = end; }
+            pf_pos = end;
             st->pf_pos = end;
-            if (end >= st->pf_end) {   // KV cache <- LM(x) done: the full-depth argmax at the last prompt token is the first generated token
-                const int np = st->pf_end;
-                tok[np] = min(max(c.head_res[n - 1].token, 0), c.vocab - 1);
-                st->len[0] = np + 1;
-                st->base[0] = np;
+            if (end >= pf_end) {   // KV cache <- LM(x) done: the full-depth argmax at the last prompt token is the first generated token
+                const int np = pf_end;
+                tok[np] = min(max(hr_s[n - 1].token, 0), c.vocab - 1);
+                len = np + 1; base = np; done = 1; pf_end = 0;
+                st->len[0] = len;
+                st->base[0] = base;
                 st->n_prompt[0] = np;
                 st->done[0] = 1;
                 st->pf_end = 0;
@@ -238,74 +274,76 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
             }
         }
         if (action != ACT_STOP && kind == CTRL_TOP && !prefilling) {
-            const int len = st->len[0], base = st->base[0], nrow = len - base;
-            for (int l = 0; l < c.L; ++l) st->st.row_layers += len - c.fill[l];
+            const int nrow = len - base;
+            long long rl = 0;
+            for (int l = 0; l < c.L; ++l) rl += len - fill_s[l];
+            bump(&st->st.row_layers, rl);
             int bad = -1;
             for (int j = 0; j + 1 < nrow; ++j)
-                if (c.head_res[j].token != tok[base + j + 1]) { bad = j; break; }
+                if (hr_s[j].token != tok_s[j]) { bad = j; break; }
             int new_base, keep;
             if (bad < 0) {
-                st->st.accepted += nrow - 1;
-                tok[len] = min(max(c.head_res[nrow - 1].token, 0), c.vocab - 1);
+                bump(&st->st.accepted, nrow - 1);
+                tok[len] = min(max(hr_s[nrow - 1].token, 0), c.vocab - 1);
                 new_base = len;
                 keep = nrow;
             } else {
-                st->st.accepted += bad;
-                st->st.rejected += 1;
-                st->st.discarded += nrow - 2 - bad;
+                bump(&st->st.accepted, bad);
+                bump(&st->st.rejected, 1);
+                bump(&st->st.discarded, nrow - 2 - bad);
                 new_base = base + bad + 1;
-                tok[new_base] = min(max(c.head_res[bad].token, 0), c.vocab - 1);
+                tok[new_base] = min(max(hr_s[bad].token, 0), c.vocab - 1);
                 keep = bad + 1;
             }
             int new_len = new_base + 1;
-            if (new_len > st->target_len[0]) {
-                st->st.truncated += new_len - st->target_len[0];
-                new_len = st->target_len[0];
+            if (new_len > target0) {
+                bump(&st->st.truncated, new_len - target0);
+                new_len = target0;
                 new_base = new_len - 1;
             }
-            for (int l = 0; l < c.L; ++l) c.fill[l] = new_base;
-            st->len[0] = new_len;
-            st->base[0] = new_base;
-            st->st.verify_steps++;
-            st->st.steps++;
-            st->st.layer_passes += c.L;
-            if (new_len >= st->target_len[0]) st->done[0] = 1;
+            for (int l = 0; l < c.L; ++l) { fill_s[l] = new_base; c.fill[l] = new_base; }
+            len = new_len; base = new_base;
+            st->len[0] = len;
+            st->base[0] = base;
+            bump(&st->st.verify_steps, 1);
+            bump(&st->st.steps, 1);
+            bump(&st->st.layer_passes, c.L);
+            if (new_len >= target0) { done = 1; st->done[0] = 1; }
             st->keep_rows = keep;
             st->keep_row0 = 0;
             verified = 1;
         }
         if (action == ACT_NEWSTEP) {
-            if (st->done[0]) { action = ACT_STOP; st->n_done = 1; }
+            if (done) { action = ACT_STOP; st->n_done = 1; }
             else if (steps_started >= A.step_budget) action = ACT_STOP;
         }
-        if (action == ACT_NEWSTEP && st->pf_end > 0) {   // next pass over the prompt: up to eight positions, all from layer 1
+        if (action == ACT_NEWSTEP && pf_end > 0) {   // next pass over the prompt: up to eight positions, all from layer 1
             ++steps_started;
             StepDesc nd;
-            nd.n_cols = min(MAX_COLS, st->pf_end - st->pf_pos);
+            nd.n_cols = min(MAX_COLS, pf_end - pf_pos);
             nd.newest = nd.n_cols - 1;
-            nd.pmax = st->pf_pos + nd.n_cols - 1;
+            nd.pmax = pf_pos + nd.n_cols - 1;
             nd.head_ok = 0;
             nd.fresh = (1 << nd.n_cols) - 1;
-            nd.run_final = st->pf_pos + nd.n_cols >= st->pf_end;
+            nd.run_final = pf_pos + nd.n_cols >= pf_end;
             if (nd.n_cols < 1 || nd.pmax >= c.max_seq) {
                 atomicCAS(A.err, 0, ERR_BAD_STATE);
                 action = ACT_STOP;
             }
             for (int j = 0; j < MAX_COLS; ++j) {
                 nd.first_layer[j] = j < nd.n_cols ? 0 : INT_MAX;
-                nd.pos[j] = st->pf_pos + j;
+                nd.pos[j] = pf_pos + j;
             }
             pub->d = nd;
         } else if (action == ACT_NEWSTEP) {
             ++steps_started;
-            const int len = st->len[0], base = st->base[0];
             StepDesc nd;
             nd.n_cols = len - base;
             nd.newest = len - 1 - base;
             nd.pmax = len - 1;
             nd.fresh = 1 << (len - 1 - base);
             nd.run_final = 1;
-            nd.head_ok = (len - 1 - base) < st->max_early && len < st->target_len[0];
+            nd.head_ok = (len - 1 - base) < max_early0 && len < target0;
             if (nd.n_cols < 1 || nd.n_cols > c.slots || nd.n_cols > MAX_COLS || len > c.max_seq || base < 0) {
                 atomicCAS(A.err, 0, ERR_BAD_STATE);
                 action = ACT_STOP;
@@ -315,7 +353,7 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
                 const int pos = base + j;
                 if (j < nd.n_cols) {
                     fl = 0;
-                    for (int l = 0; l < c.L; ++l) fl += c.fill[l] > pos;
+                    for (int l = 0; l < c.L; ++l) fl += fill_s[l] > pos;
                 }
                 nd.first_layer[j] = fl;
                 nd.pos[j] = pos;
@@ -348,19 +386,20 @@ __device__ __noinline__ void control_cta0(const MegaArgs &A, Smem *sm, int kind,
             const int pos = nd.pos[col];
             const int tokid = min(max(c.tokens[pos], 0), c.vocab - 1);
             const __nv_bfloat16 *erow = M.tok_embed + (size_t)tokid * c.d;
-            for (int n0 = 0; n0 < c.d; n0 += 8 * CONS_THREADS) {   // eight loads of the embedding row in flight per thread
-                float v[8];
+            for (int n0 = 0; n0 < c.d; n0 += 8 * CONS_THREADS) {   // eight loads of the embedding row and of the gain in flight per thread
+                float v[8], gn[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const int n = n0 + u * CONS_THREADS + tid;
                     v[u] = n < c.d ? __bfloat162float(erow[n]) : 0.f;
+                    gn[u] = n < c.d ? __bfloat162float(g0[n]) : 0.f;
                 }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const int n = n0 + u * CONS_THREADS + tid;
                     if (n < c.d) {
                         c.resid[(size_t)col * c.d + n] = v[u];
-                        xfrag_store(A.XA, n, col, v[u] * __bfloat162float(g0[n]));
+                        xfrag_store(A.XA, n, col, v[u] * gn[u]);
                     }
                     float q = v[u] * v[u];
                     q += __shfl_xor_sync(0xffffffffu, q, 1);
