@@ -585,6 +585,54 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     const int mt = warp >> 2, qr = warp & 3;
     const float scale = rsqrtf((float)HD);
     __nv_bfloat16 *pool = reinterpret_cast<__nv_bfloat16 *>(c.kv_pool);
+    // Merge of the chunk partials of one kv head into the O-projection's input (by a whole CTA).
+    auto merge_chunks = [&](int kvh) {
+        // Four features of one (column, q head) per thread and pass; the chunk partials are folded in
+        // ascending order, eight at a time with all their loads in flight, by the usual running-max rule.
+        const int nqc = MAX_COLS * group;
+        for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
+            const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = div_group(qcol, group), g = qcol - cc * group;
+            if (!((mask >> cc) & 1u)) continue;
+            const int h = kvh * group + g;
+            const int nch = d.pos[cc] / ATT_CHUNK + 1;
+            const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE;
+            float Mx = -INFINITY, den = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k0 = 0; k0 < nch; k0 += 8) {
+                float2 ml[8];
+                float4 ov[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const bool ok = k0 + u < nch;
+                    const float *pk = part + (size_t)(k0 + u) * ATT_STRIDE;
+                    ml[u] = ok ? __ldcg(reinterpret_cast<const float2 *>(pk + HD)) : make_float2(-INFINITY, 0.f);
+                    ov[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(pk + dim)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float Mn = Mx;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, ml[u].x);
+                if (Mn == -INFINITY) continue;
+                const float sc = Mx == -INFINITY ? 0.f : __expf(Mx - Mn);
+                den *= sc; acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (ml[u].x != -INFINITY) {
+                        const float w = __expf(ml[u].x - Mn);
+                        den += ml[u].y * w;
+                        acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
+                    }
+                }
+                Mx = Mn;
+            }
+            xfrag_store(A.XO, h * HD + dim, cc, acc.x / den);
+            xfrag_store(A.XO, h * HD + dim + 1, cc, acc.y / den);
+            xfrag_store(A.XO, h * HD + dim + 2, cc, acc.z / den);
+            xfrag_store(A.XO, h * HD + dim + 3, cc, acc.w / den);
+        }
+    };
+    // With at most one work item per CTA the CTA that completes a head last merges it at once; with more,
+    // designated CTAs do (see below).  Who merges does not change what is computed.
+    const bool last_arriver_merges = n_items <= G;
     for (int item = cta; item < n_items; item += G) {
         const int kvh = item / nchunk, j = item - kvh * nchunk;
         const int p_base = j * ATT_CHUNK;
@@ -842,60 +890,40 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 }
             }
         }
-        // ---- the CTA that finishes a kv head's last item merges the chunks of that head
+        // ---- this item's partials are complete: count it (a release that returns nothing, so nobody waits for it)
         if (tid == 0) trace(S, EV_ITEM, item);
         bar_consumers();
-        if (tid == 0) {   // release this block's partials and acquire the others' in one step
-            unsigned old;
-            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + kvh) : "memory");
-            sm->bcast[2] = (int)old;
-        }
-        bar_consumers();
-        if (sm->bcast[2] == nchunk - 1) {
-            // Four features of one (column, q head) per thread and pass; the chunk partials are folded in
-            // ascending order, eight at a time with all their loads in flight, by the usual running-max rule.
-            const int nqc = MAX_COLS * group;
-            for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
-                const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = div_group(qcol, group), g = qcol - cc * group;
-                if (!((mask >> cc) & 1u)) continue;
-                const int h = kvh * group + g;
-                const int nch = d.pos[cc] / ATT_CHUNK + 1;
-                const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE;
-                float Mx = -INFINITY, den = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int k0 = 0; k0 < nch; k0 += 8) {
-                    float2 ml[8];
-                    float4 ov[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const bool ok = k0 + u < nch;
-                        const float *pk = part + (size_t)(k0 + u) * ATT_STRIDE;
-                        ml[u] = ok ? __ldcg(reinterpret_cast<const float2 *>(pk + HD)) : make_float2(-INFINITY, 0.f);
-                        ov[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(pk + dim)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    float Mn = Mx;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, ml[u].x);
-                    if (Mn == -INFINITY) continue;
-                    const float sc = Mx == -INFINITY ? 0.f : __expf(Mx - Mn);
-                    den *= sc; acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (ml[u].x != -INFINITY) {
-                            const float w = __expf(ml[u].x - Mn);
-                            den += ml[u].y * w;
-                            acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
-                        }
-                    }
-                    Mx = Mn;
-                }
-                xfrag_store(A.XO, h * HD + dim, cc, acc.x / den);
-                xfrag_store(A.XO, h * HD + dim + 1, cc, acc.y / den);
-                xfrag_store(A.XO, h * HD + dim + 2, cc, acc.z / den);
-                xfrag_store(A.XO, h * HD + dim + 3, cc, acc.w / den);
+        if (last_arriver_merges) {
+            if (tid == 0) {   // release this block's partials and acquire the others' in one step
+                unsigned old;
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + kvh) : "memory");
+                sm->bcast[2] = (int)old;
             }
+            bar_consumers();
+            if (sm->bcast[2] == nchunk - 1) {
+                merge_chunks(kvh);
+                if (tid == 0) { A.attn_cnt[kvh] = 0u; trace(S, EV_COMBINE, kvh); }
+            }
+        } else if (tid == 0) {
+            __threadfence();
+            red_release_add(A.attn_cnt + kvh, 1u);
+        }
+    }
+    if (last_arriver_merges) return;
+    // ---- The chunk partials of kv head h are merged by one designated CTA, G - 1 - h (the high CTAs
+    // have the fewest work items), once all nchunk items of the head have been counted.  (Letting
+    // whichever CTA arrives last do it looks cheaper but piles up at long contexts: the CTA that
+    // merges one head is late for its next item, so it is last again for the next head, and ends up
+    // merging every head in turn while the rest of the grid waits.)
+    for (int kvh = 0; kvh < c.nkv; ++kvh) {
+        if ((G - 1 - kvh % G + G) % G != cta) continue;
+        if (tid == 0) grid_wait(S, A.attn_cnt + kvh, (unsigned)nchunk);
+        bar_consumers();
+        {
+            merge_chunks(kvh);
             if (tid == 0) { A.attn_cnt[kvh] = 0u; trace(S, EV_COMBINE, kvh); }
         }
+        bar_consumers();   // the next head's wait must not start before every thread is done with this one
     }
 }
 
