@@ -239,3 +239,28 @@ def test_long_context_many_chunks():
     A = session(pair, max_seq=1200)
     A.prefill(prompt)
     assert np.array_equal(A.adaptive_decode(n, 0.0, cfg.exit_layers, 5)[0], out)
+
+
+def test_more_attention_work_items_than_ctas():
+    """Sixteen kv heads at a context of 1600 positions: 13 chunks x 16 heads = 208 work items, more than
+    any GPU has SMs, so CTAs take several items each and the chunk partials are merged by the
+    designated CTAs (with fewer items than CTAs the last CTA to finish a head merges it)."""
+    cfg = mha(n_layers=2, d_model=1024, n_q_heads=16, n_kv_heads=16, d_ff=704, exit_layers=(1,))
+    assert 16 * (1600 // 128 + 1) > torch.cuda.get_device_properties(0).multi_processor_count
+    pair = Pair(cfg)
+    prompt = synth.make_prompt(cfg, n=1600).numpy()
+    n = 10
+    S = session(pair, max_seq=1700)
+    S.capture_logits(n + 4)
+    S.prefill(prompt)
+    out = S.plain_decode(n)[0]
+    lg = S.captured_logits()[:n].clone()
+    check_against_oracle(pair, prompt, out, lg.cpu().numpy())
+    for gamma, tape in [(0.0, None), (0.5, [1] * 16)]:
+        A = session(pair, max_seq=1700)
+        A.capture_logits(n + 4)
+        A.prefill(prompt)
+        if tape:
+            A.set_exit_tape(tape)
+        assert np.array_equal(A.adaptive_decode(n, gamma, cfg.exit_layers, 5)[0], out)
+        assert torch.equal(A.captured_logits()[:n], lg)
