@@ -16,8 +16,8 @@
  *     string saved by the last ADA_ECUDA on the calling thread.
  *   - "dev" pointers are device memory owned by the CALLER (allocated e.g. through PyTorch); the
  *     library borrows them and they must outlive the object they were given to.  "host" pointers
- *     are ordinary host memory.  The library never allocates device memory itself, except in
- *     ada_*_create for tensor-map/handle bookkeeping on the host.
+ *     are ordinary host memory.  The library never allocates device memory itself: weights it has to
+ *     repack go into an arena the caller provides, everything else into the session's scratch.
  *   - All matrices are row-major [out_features, in_features]; every tensor of a model has the
  *     model's dtype (fp32 or bf16 bit patterns).
  *   - One session is used from one host thread at a time.  All device work of a session is issued
@@ -74,6 +74,9 @@ typedef struct {
     int64_t host_syncs;      /* stream synchronisations the decode loop needed */
     int64_t kernel_launches; /* kernels of this library launched by the decode calls */
     double decode_ms;        /* device time of the decode calls (CUDA events on the session stream) */
+    int64_t emitted[ADA_MAX_BATCH]; /* tokens returned per sequence (fewer than asked for only after an end-of-sequence token) */
+    int64_t finished;        /* sequences that ended on a verified end-of-sequence token during these calls */
+    int64_t path;            /* decode path of the last call: 1 = persistent kernel, 0 = one kernel per operation */
 } ada_stats;
 
 const char *ada_strerror(int code);
@@ -86,19 +89,35 @@ int ada_model_create(const ada_config *cfg, ada_model **out);
 /* Lend one tensor (device pointer, exact byte size checked).  Names:
  *   tok_embed [vocab, d]         final_norm [d]          lm_head [vocab, d] (only if not tied)
  *   layers.N.attn_norm [d]       layers.N.ffn_norm [d]
- *   layers.N.wqkv [(n_q+2 n_kv) head_dim, d]   rows: all q heads, then all k heads, then all v heads
+ *   layers.N.wq [n_q head_dim, d]    layers.N.wk, layers.N.wv [n_kv head_dim, d]
  *   layers.N.wo [d, n_q head_dim]
- *   layers.N.w_gate_up [2 d_ff, d]             rows: gate, then up
+ *   layers.N.w_gate, layers.N.w_up [d_ff, d]
  *   layers.N.w_down [d, d_ff]
+ * and, for callers that already hold them stacked (nothing is gained or lost either way):
+ *   layers.N.wqkv [(n_q+2 n_kv) head_dim, d]   rows: all q heads, then all k heads, then all v heads
+ *   layers.N.w_gate_up [2 d_ff, d]             rows: gate, then up
  * Pointers must be 16-byte aligned. */
 int ada_model_set_tensor(ada_model *m, const char *name, const void *dev_ptr, size_t bytes);
+
+/* Repack on load.  The persistent decode kernel finishes q, k and v (rotary embedding, cache write)
+ * in the epilogue of the QKV product, which needs the rows of every q and k head in an order that
+ * puts the two partners (i, i + head_dim/2) of a rotation into one tensor-core tile.
+ * ada_model_finalize() writes that reordered copy of q | k | v of every layer into an arena the
+ * caller provides: ada_model_arena_bytes() device bytes, 256-byte aligned, which must outlive the
+ * model (0 bytes for models the persistent kernel does not take: fp32, head_dim other than 64 / 128,
+ * more than 4 q heads per kv head, d_model / n_q head_dim / d_ff not multiples of 64; such models
+ * need no arena).  The lent tensors themselves are never written. */
+size_t ada_model_arena_bytes(const ada_model *m);
+int ada_model_set_arena(ada_model *m, void *arena_dev, size_t bytes);
 
 /* Register the intermediate head of Section 2.1 at 1-based `layer` (1 <= layer < n_layers):
  * logits = logit_scale * E* (T RMSNorm_f(h)), E^(i) = E* T^(i).  T_dev is a dense [d, d] matrix in
  * the model dtype, or NULL for T = I. */
 int ada_model_set_exit_head(ada_model *m, int32_t layer, const void *T_dev, float logit_scale);
 
-int ada_model_finalize(ada_model *m); /* ADA_ESTATE if a tensor is missing */
+/* Checks that every tensor is present and repacks into the arena (on the device that is current;
+ * synchronises that device).  ADA_ESTATE if a tensor or a required arena is missing. */
+int ada_model_finalize(ada_model *m);
 void ada_model_destroy(ada_model *m);
 
 /* ---- session ------------------------------------------------------------------------------ */
@@ -129,13 +148,20 @@ int ada_prefill(ada_session *s, int32_t seq, const int32_t *prompt_host, int32_t
  * out_host[batch][n_tokens] (counting from the first generated token, which prefill produced),
  * synchronise the stream before returning, and leave the same logical state: K/V present at all
  * layers for every token before the last returned one, which stays pending.  Calls can be chained
- * and mixed.  Every sequence must have been prefilled. */
-int ada_plain_decode(ada_session *s, int32_t n_tokens, int32_t *out_host, ada_stats *stats /* nullable */);
+ * and mixed.  Every sequence must have been prefilled.
+ *
+ * eos_id (Algorithm 1: "while t_i != [EOS]"): a token id, or -1 for none.  A sequence ends at its first
+ * VERIFIED end-of-sequence token, i.e. one that is the full-depth argmax; an early-predicted one stops
+ * nothing until the verification accepts it.  The row of a sequence that ended holds its tokens up to
+ * and including that token, then eos_id up to n_tokens; stats->emitted[seq] counts the real ones.
+ * Later calls return only padding for it, and ADA_ESTATE once every sequence of the session has
+ * ended (ada_prefill or ada_session_reset starts a sequence afresh). */
+int ada_plain_decode(ada_session *s, int32_t n_tokens, int32_t eos_id, int32_t *out_host, ada_stats *stats /* nullable */);
 
 /* Algorithm 1.  threshold = gamma of Eq. 1 (strict: exit iff p > gamma).  exit_layers: ascending
  * 1-based layers, each < n_layers, each with a registered head.  max_early <= the session's. */
 int ada_adaptive_decode(ada_session *s, int32_t n_tokens, float threshold, const int32_t *exit_layers,
-                        int32_t n_exit_layers, int32_t max_early, int32_t *out_host, ada_stats *stats);
+                        int32_t n_exit_layers, int32_t max_early, int32_t eos_id, int32_t *out_host, ada_stats *stats);
 
 /* ---- test hooks --------------------------------------------------------------------------- */
 
@@ -164,14 +190,22 @@ int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out
 /* Select the decode path: 1 = the persistent kernel (one cooperative launch runs many steps of
  * Algorithm 1; bf16 models, one sequence, at most 8 tokens per pass, 64-token KV pages, head_dim 64
  * or 128, at most 4 q heads per kv head, d_model / n_q_heads*head_dim / d_ff multiples of 64); it is
- * the default wherever a session qualifies.  0 = one
- * kernel per operation on CUDA cores (any dtype, any batch; also what prefill uses).
- * ADA_EUNSUPPORTED if path 1 is asked of a session that does not qualify. */
+ * the default wherever a session qualifies; a session that qualifies but cannot be set up fails in
+ * ada_session_create instead of taking the other path).  0 = one kernel per operation on CUDA cores
+ * (any dtype, any batch).  ADA_EUNSUPPORTED if path 1 is asked of a session that does not qualify.
+ * ada_stats.path reports the path a decode call ran on. */
 int ada_debug_set_path(ada_session *s, int32_t path);
 int ada_debug_get_path(ada_session *s, int32_t *path_out);
 /* Steps of Algorithm 1 one launch of the persistent kernel may start before it returns to the host
  * (default 256; the host relaunches until the call is complete). */
 int ada_debug_set_launch_steps(ada_session *s, int32_t steps);
+/* Every wait inside the persistent kernel (on a shared-memory barrier, on the grid-wide counter, on
+ * another CTA's partial sums) gives up after `ns` nanoseconds (default 2 s): the kernel then sets an
+ * error word, lets every other wait fall through, ends, and the decode call returns ADA_ETIMEOUT.
+ * The sequence state is undefined after that; ada_session_reset + ada_prefill make the session
+ * usable again.  A limit shorter than a grid-wide wait normally lasts (a few microseconds) makes the
+ * next decode call time out: that is how the give-up path is tested. */
+int ada_debug_set_wait_limit(ada_session *s, uint64_t ns);
 /* Event trace of the persistent kernel: while the kernel runs the steps [step0, step1) of a launch
  * (counted from 0 in every launch), every CTA appends (nanosecond timestamp, code) pairs of
  * uint64 to its own region of dev_buf [SMs][cap_events][2]; code = CTA << 32 | argument << 8 | event (1 phase begin, 2
@@ -180,6 +214,15 @@ int ada_debug_set_launch_steps(ada_session *s, int32_t steps);
  * chunks merged, 10 barrier arrival, 11.. attention sub-steps).  count_dev [SMs] receives the number of
  * events of each CTA in the last traced launch.  NULL stops. */
 int ada_debug_trace(ada_session *s, uint64_t *dev_buf, uint32_t *count_dev, uint32_t cap_events, int32_t step0, int32_t step1);
+
+/* Host-only: how the streaming GEMM of shape N x K (mode as in ada_debug_gemm) divides its work
+ * over `grid` CTAs, for CTA `cta`.  out9 (host) receives {split, t0, t1, n, ta, tb, s0_own_k0,
+ * s0_pub_k1, sl_k1}: split == 0: whole 16-row tiles [t0, t1); split == 1 (only if `split` is
+ * nonzero and the shape allows it): one group of n tile slots, slot s holding tile ta + s, where
+ * slot 0 multiplies k chunks >= s0_own_k0 of its tile and, before them, chunks < s0_pub_k1 of
+ * tile tb (published to the next CTA), and the last slot (if not slot 0) only chunks < sl_k1.
+ * A k chunk is 512 wide.  No GPU is touched.  ADA_EINVAL on bad arguments. */
+int ada_debug_gemm_plan(int32_t N, int32_t K, int32_t mode, int32_t grid, int32_t cta, int32_t split, int32_t *out9);
 
 /* Run the weight-streaming skinny GEMM of the decode kernel by itself (the kernel behind the QKV,
  * O, gate/up, down and LM-head products of a layer pass, Algorithm 1 "process all tokens in P[l]
@@ -192,15 +235,6 @@ int ada_debug_trace(ada_session *s, uint64_t *dev_buf, uint32_t *count_dev, uint
  * bytes, 256-byte aligned.  The product is launched `repeat` >= 1 times back to back inside one
  * kernel; *ms_out (nullable) receives the device time of that kernel.  All pointers except ms_out
  * are device pointers.  Returns ADA_ETIMEOUT if a bounded device-side wait expired. */
-/* Host-only: how the streaming GEMM of shape N x K (mode as in ada_debug_gemm) divides its work
- * over `grid` CTAs, for CTA `cta`.  out9 (host) receives {split, t0, t1, n, ta, tb, s0_own_k0,
- * s0_pub_k1, sl_k1}: split == 0: whole 16-row tiles [t0, t1); split == 1 (only if `split` is
- * nonzero and the shape allows it): one group of n tile slots, slot s holding tile ta + s, where
- * slot 0 multiplies k chunks >= s0_own_k0 of its tile and, before them, chunks < s0_pub_k1 of
- * tile tb (published to the next CTA), and the last slot (if not slot 0) only chunks < sl_k1.
- * A k chunk is 512 wide.  No GPU is touched.  ADA_EINVAL on bad arguments. */
-int ada_debug_gemm_plan(int32_t N, int32_t K, int32_t mode, int32_t grid, int32_t cta, int32_t split, int32_t *out9);
-
 size_t ada_debug_gemm_work_bytes(int32_t K);
 int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols,
                    void *work_dev, size_t work_bytes, float *Y_dev, int32_t ldy, int32_t repeat, void *cuda_stream,
@@ -218,11 +252,15 @@ int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const 
  * process exits.  It bounds the depth: K <= 16384, larger K returns ADA_ECAPACITY.  The call
  * performs no cudaMalloc / cudaFree and creates no events.
  *
- * The first call on each device looks up the array's device address and configures the kernel;
- * make that first call outside any stream capture.  All calls on a device share the one array:
+ * The scratch comes into being when the library's device code is first used on a GPU (the driver
+ * then places the array and the kernels there; that one-time placement is the driver's, not a call
+ * this function makes).  The first call on each device also looks up the array's device address and
+ * configures the kernel: make that first call before any stream capture begins.  Every call, the
+ * first and the later ones alike, waits for `cuda_stream` twice and copies an error word back to
+ * the host before it returns.  All calls on a device share the one array:
  * it keeps the previous call's contents (the call clears the word that has to start at zero and
  * rewrites the rest), and two calls whose kernels overlap on the GPU (different streams, or
- * different host threads) race on it.  The call synchronises `cuda_stream` before returning.
+ * different host threads) race on it.
  * W_dev, X_dev, Y_dev are device pointers as in ada_debug_gemm. */
 int ada_gemm_noalloc(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols, float *Y_dev,
                      int32_t ldy, void *cuda_stream);

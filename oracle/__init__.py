@@ -79,9 +79,10 @@ def _lib():
         L.orc_full_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_hidden_after.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         L.orc_head_eval.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(C.c_double), C.c_void_p]
-        L.orc_plain_decode.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(Stats)]
+        L.orc_plain_decode.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_int32), C.POINTER(Stats)]
         L.orc_adaptive_decode.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_int, C.c_int,
-                                          C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.POINTER(Stats)]
+                                          C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_int32),
+                                          C.POINTER(Stats)]
         _LIB = L
     return _LIB
 
@@ -232,17 +233,23 @@ class Session:
         if rc:
             raise RuntimeError(f"orc_prefill -> {rc}")
 
-    def plain_decode(self, n: int, stats: Optional[Stats] = None) -> np.ndarray:
+    def plain_decode(self, n: int, stats: Optional[Stats] = None, eos_id: int = -1) -> np.ndarray:
+        """Next n greedy tokens; with eos_id >= 0 generation stops at the first such token, `self.emitted`
+        holds the number produced and the rest of the row is eos_id."""
         out = np.empty(n, dtype=np.int32)
-        rc = _lib().orc_plain_decode(self.h, n, out.ctypes.data, C.byref(stats) if stats is not None else None)
+        got = C.c_int32(0)
+        rc = _lib().orc_plain_decode(self.h, n, eos_id, out.ctypes.data, C.byref(got),
+                                     C.byref(stats) if stats is not None else None)
         if rc:
             raise RuntimeError(f"orc_plain_decode -> {rc}")
+        self.emitted = got.value
         return out
 
     def adaptive_decode(self, n: int, gamma: float, exit_layers: Sequence[int], max_early: int = 5,
                         tape: Optional[Sequence[int]] = None, tape_tok: Optional[Sequence[int]] = None,
-                        stats: Optional[Stats] = None) -> np.ndarray:
+                        stats: Optional[Stats] = None, eos_id: int = -1) -> np.ndarray:
         out = np.empty(n, dtype=np.int32)
+        got = C.c_int32(0)
         ex = np.ascontiguousarray(np.asarray(exit_layers, dtype=np.int32))
         n_tape = 0
         tp = tt = None
@@ -257,10 +264,11 @@ class Session:
             assert len(tp) == len(tt)
         rc = _lib().orc_adaptive_decode(self.h, n, gamma, ex.ctypes.data, len(ex), max_early,
                                         tp.ctypes.data if tp is not None else None,
-                                        tt.ctypes.data if tt is not None else None, n_tape,
-                                        out.ctypes.data, C.byref(stats) if stats is not None else None)
+                                        tt.ctypes.data if tt is not None else None, n_tape, eos_id,
+                                        out.ctypes.data, C.byref(got), C.byref(stats) if stats is not None else None)
         if rc:
             raise RuntimeError(f"orc_adaptive_decode -> {rc}")
+        self.emitted = got.value
         return out
 
     def __del__(self):

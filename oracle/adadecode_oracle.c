@@ -430,15 +430,18 @@ static void report(orc_session *s, int n, int32_t *out) {
 }
 
 /* Standard greedy autoregressive decoding: returns the next n generated tokens.  After the call
-   every token before the last returned one has K/V at all layers and the last one is pending. */
-int orc_plain_decode(orc_session *s, int n, int32_t *out, orc_stats *st) {
+   every token before the last returned one has K/V at all layers and the last one is pending.
+   eos_id >= 0: generation stops at the first end-of-sequence token ("while t_i != [EOS]" of
+   Algorithm 1, which plain decoding shares): *n_out receives the number of tokens produced, the
+   rest of `out` is filled with eos_id. */
+int orc_plain_decode(orc_session *s, int n, int eos_id, int32_t *out, int32_t *n_out, orc_stats *st) {
     const orc_config *c = &s->m->c;
     if (s->n_inflight) return -3;
     int target_len = s->n_prompt + s->n_reported + n;
     if (target_len > s->max_seq) return -4;
     double *h = (double *)malloc(sizeof(double) * c->d_model);
     double *z = (double *)malloc(sizeof(double) * c->vocab);
-    while (s->len < target_len) {
+    while (s->len < target_len && !(eos_id >= 0 && s->tokens[s->len - 1] == eos_id)) {
         int pos = s->len - 1;
         embed(s->m, s->tokens[pos], h);
         for (int l = 0; l < c->n_layers; ++l) {
@@ -451,7 +454,13 @@ int orc_plain_decode(orc_session *s, int n, int32_t *out, orc_stats *st) {
         s->tokens[s->len++] = tok;
         if (st) { st->steps++; st->verify_steps++; }
     }
-    report(s, n, out);
+    {
+        int got = s->len - (s->n_prompt + s->n_reported);
+        if (got > n) got = n;
+        report(s, got, out);
+        for (int i = got; i < n; ++i) out[i] = eos_id;
+        if (n_out) *n_out = got;
+    }
     free(h); free(z);
     return 0;
 }
@@ -474,8 +483,8 @@ int orc_plain_decode(orc_session *s, int n, int32_t *out, orc_stats *st) {
  * requested count is already reached by tentative tokens, the newest token runs to layer L.
  */
 int orc_adaptive_decode(orc_session *s, int n, double gamma, const int32_t *exit_layers, int n_exit,
-                        int max_early, const uint8_t *tape, const int32_t *tape_tok, int n_tape,
-                        int32_t *out, orc_stats *st) {
+                        int max_early, const uint8_t *tape, const int32_t *tape_tok, int n_tape, int eos_id,
+                        int32_t *out, int32_t *n_out, orc_stats *st) {
     const orc_config *c = &s->m->c;
     const int L = c->n_layers, d = c->d_model;
     if (max_early < 0 || max_early > ORC_MAX_INFLIGHT) return -5;
@@ -486,6 +495,8 @@ int orc_adaptive_decode(orc_session *s, int n, double gamma, const int32_t *exit
     }
     int target_len = s->n_prompt + s->n_reported + n;
     if (target_len + 1 > s->max_seq) return -4;
+    /* while t_i != [EOS]: the pending token is verified; if it is the end-of-sequence token nothing more is generated */
+    if (eos_id >= 0 && s->len >= 1 && s->len <= target_len && s->tokens[s->len - 1] == eos_id) target_len = s->len;
 
     /* P[l]: positions of tokens pending at layer l (1-based l), in sequence order */
     int32_t(*P)[ORC_MAX_INFLIGHT + 1] = calloc(L + 1, sizeof(*P));
@@ -601,6 +612,12 @@ int orc_adaptive_decode(orc_session *s, int n, double gamma, const int32_t *exit
                 Pn[L] = 0;
                 s->n_inflight = 0;
                 if (st) st->verify_steps++;
+                /* while t_i != [EOS]: every token after position pos0 is now verified (each equals the full
+                   model's greedy choice); the first end-of-sequence token among them ends the sequence.  An
+                   early-predicted end-of-sequence token has stopped nothing until this point. */
+                if (eos_id >= 0)
+                    for (int q = pos0 + 1; q < s->len; ++q)
+                        if (s->tokens[q] == eos_id) { if (q + 1 < target_len) target_len = q + 1; break; }
             }
         }
         if (st) st->steps++;
@@ -615,7 +632,13 @@ int orc_adaptive_decode(orc_session *s, int n, double gamma, const int32_t *exit
         s->len = target_len;
         for (int l2 = 0; l2 < L; ++l2) if (s->kv_len[l2] > target_len - 1) s->kv_len[l2] = target_len - 1;
     }
-    report(s, n, out);
+    {
+        int got = s->len - (s->n_prompt + s->n_reported);
+        if (got > n) got = n;
+        report(s, got, out);
+        for (int i = got; i < n; ++i) out[i] = eos_id;
+        if (n_out) *n_out = got;
+    }
 done:
     free(P); free(Pn); free(H); free(z); free(argm);
     return rc;

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libadadecode.so")
 _LIB = None
 
 ADA_MAX_LAYERS = 256
+ADA_MAX_BATCH = 16
 ERRORS = {0: "ADA_OK", -1: "ADA_EINVAL", -2: "ADA_ESTATE", -3: "ADA_ECAPACITY", -4: "ADA_ECUDA",
           -5: "ADA_ETIMEOUT", -6: "ADA_EUNSUPPORTED"}
 
@@ -28,6 +29,7 @@ EXPORTS = [
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
     "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_plan", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace", "ada_gemm_noalloc",
+    "ada_model_arena_bytes", "ada_model_set_arena", "ada_debug_set_wait_limit",
 ]
 
 
@@ -57,11 +59,13 @@ class Stats(C.Structure):
                 ("steps", "head_evals", "early_exits", "verify_steps", "accepted", "rejected", "discarded",
                  "row_layers", "truncated")] + \
                [("exits_at_layer", C.c_int64 * ADA_MAX_LAYERS), ("layer_passes", C.c_int64), ("host_syncs", C.c_int64),
-                ("kernel_launches", C.c_int64), ("decode_ms", C.c_double)]
+                ("kernel_launches", C.c_int64), ("decode_ms", C.c_double), ("emitted", C.c_int64 * ADA_MAX_BATCH),
+                ("finished", C.c_int64), ("path", C.c_int64)]
 
     def as_dict(self) -> dict:
-        d = {n: getattr(self, n) for n, _ in self._fields_ if n != "exits_at_layer"}
+        d = {n: getattr(self, n) for n, _ in self._fields_ if n not in ("exits_at_layer", "emitted")}
         d["exits_at_layer"] = {i: int(v) for i, v in enumerate(self.exits_at_layer) if v}
+        d["emitted"] = [int(v) for v in self.emitted if v]
         return d
 
 
@@ -82,6 +86,10 @@ def load() -> C.CDLL:
         L.ada_model_set_tensor.argtypes = [vp, C.c_char_p, vp, sz]
         L.ada_model_set_exit_head.argtypes = [vp, i32, vp, C.c_float]
         L.ada_model_finalize.argtypes = [vp]
+        L.ada_model_arena_bytes.restype = sz
+        L.ada_model_arena_bytes.argtypes = [vp]
+        L.ada_model_set_arena.argtypes = [vp, vp, sz]
+        L.ada_debug_set_wait_limit.argtypes = [vp, C.c_uint64]
         L.ada_model_destroy.argtypes = [vp]
         L.ada_model_destroy.restype = None
         L.ada_session_scratch_bytes.restype = sz
@@ -93,8 +101,8 @@ def load() -> C.CDLL:
         L.ada_session_destroy.restype = None
         L.ada_session_reset.argtypes = [vp, i32]
         L.ada_prefill.argtypes = [vp, i32, vp, i32]
-        L.ada_plain_decode.argtypes = [vp, i32, vp, C.POINTER(Stats)]
-        L.ada_adaptive_decode.argtypes = [vp, i32, C.c_float, vp, i32, i32, vp, C.POINTER(Stats)]
+        L.ada_plain_decode.argtypes = [vp, i32, i32, vp, C.POINTER(Stats)]
+        L.ada_adaptive_decode.argtypes = [vp, i32, C.c_float, vp, i32, i32, i32, vp, C.POINTER(Stats)]
         L.ada_debug_capture_logits.argtypes = [vp, vp, i32]
         L.ada_debug_logits_captured.argtypes = [vp, C.POINTER(i32)]
         L.ada_debug_capture_heads.argtypes = [vp, vp, i32, C.POINTER(i32)]
@@ -161,7 +169,9 @@ def gemm_noalloc(W, X, Y, mode: int = 0):
 
 
 class Model:
-    """ada_model over borrowed torch CUDA tensors (fused layout of `synth.make_weights`)."""
+    """ada_model over borrowed torch CUDA tensors: the fused layout of `synth.make_weights` (wqkv,
+    w_gate_up) or the separate matrices (wq, wk, wv, w_gate, w_up), as the caller holds them.  The
+    arena the library repacks into is allocated here through torch and handed over."""
 
     def __init__(self, cfg, weights: Dict[str, "torch.Tensor"], tied: Optional[bool] = None):
         import torch
@@ -180,6 +190,7 @@ class Model:
             _ck(lib.ada_model_set_tensor(h, name.encode(), t.data_ptr(), t.numel() * t.element_size()),
                 f"ada_model_set_tensor({name})")
         self._finalized = False
+        self.arena = None
 
     def set_exit_head(self, layer: int, T=None, logit_scale: float = 1.0):
         ptr = None
@@ -191,7 +202,14 @@ class Model:
 
     def finalize(self):
         if not self._finalized:
-            _ck(load().ada_model_finalize(self.h), "ada_model_finalize")
+            import torch
+            lib = load()
+            need = lib.ada_model_arena_bytes(self.h)
+            if need:
+                self.arena = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
+                off = (-self.arena.data_ptr()) % 256
+                _ck(lib.ada_model_set_arena(self.h, self.arena.data_ptr() + off, need), "ada_model_set_arena")
+            _ck(lib.ada_model_finalize(self.h), "ada_model_finalize")
             self._finalized = True
 
     def __del__(self):
@@ -240,18 +258,19 @@ class Session:
         p = np.ascontiguousarray(np.asarray(prompt, dtype=np.int32))
         _ck(load().ada_prefill(self.h, seq, p.ctypes.data, len(p)), "ada_prefill")
 
-    def plain_decode(self, n_tokens: int, stats: Optional[Stats] = None, out: Optional[np.ndarray] = None) -> np.ndarray:
+    def plain_decode(self, n_tokens: int, stats: Optional[Stats] = None, out: Optional[np.ndarray] = None,
+                     eos_id: int = -1) -> np.ndarray:
         out = np.empty((self.batch, n_tokens), dtype=np.int32) if out is None else out
-        _ck(load().ada_plain_decode(self.h, n_tokens, out.ctypes.data, C.byref(stats) if stats is not None else None),
+        _ck(load().ada_plain_decode(self.h, n_tokens, eos_id, out.ctypes.data, C.byref(stats) if stats is not None else None),
             "ada_plain_decode")
         return out
 
     def adaptive_decode(self, n_tokens: int, threshold: float, exit_layers: Sequence[int], max_early: int = 5,
-                        stats: Optional[Stats] = None, out: Optional[np.ndarray] = None) -> np.ndarray:
+                        stats: Optional[Stats] = None, out: Optional[np.ndarray] = None, eos_id: int = -1) -> np.ndarray:
         out = np.empty((self.batch, n_tokens), dtype=np.int32) if out is None else out
         ex = np.ascontiguousarray(np.asarray(exit_layers, dtype=np.int32))
         _ck(load().ada_adaptive_decode(self.h, n_tokens, threshold, ex.ctypes.data if len(ex) else None, len(ex),
-                                       max_early, out.ctypes.data, C.byref(stats) if stats is not None else None),
+                                       max_early, eos_id, out.ctypes.data, C.byref(stats) if stats is not None else None),
             "ada_adaptive_decode")
         return out
 
@@ -316,6 +335,9 @@ class Session:
 
     def set_launch_steps(self, steps: int):
         _ck(load().ada_debug_set_launch_steps(self.h, steps), "ada_debug_set_launch_steps")
+
+    def set_wait_limit(self, ns: int):
+        _ck(load().ada_debug_set_wait_limit(self.h, ns), "ada_debug_set_wait_limit")
 
     def trace(self, cap_events: int, step0: int, step1: int):
         """Record the persistent kernel's events of steps [step0, step1) of every following launch

@@ -29,8 +29,11 @@ thread_local std::string g_cuda_err;
     } while (0)
 
 struct LayerW {
-    const void *attn_norm = nullptr, *wqkv = nullptr, *wo = nullptr, *ffn_norm = nullptr, *w_gate_up = nullptr,
-               *w_down = nullptr;
+    // q, k, v and gate, up are held as separate matrices: lent fused (wqkv, w_gate_up) they point into
+    // the one tensor.  wqkv_perm is the library's own copy of q | k | v in the caller's arena, with the
+    // rows of every q and k head reordered for the persistent kernel's QKV epilogue.
+    const void *attn_norm = nullptr, *wq = nullptr, *wk = nullptr, *wv = nullptr, *wo = nullptr, *ffn_norm = nullptr,
+               *w_gate = nullptr, *w_up = nullptr, *w_down = nullptr, *wqkv_perm = nullptr;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -78,6 +81,8 @@ struct ada_model {
     std::vector<int> has_head;
     std::vector<const void *> head_T;
     std::vector<float> head_scale;
+    void *arena = nullptr;
+    size_t arena_bytes = 0;
     bool finalized = false;
 };
 
@@ -92,7 +97,8 @@ struct ada_session {
     std::vector<int> free_pages;
     std::vector<std::vector<int>> seq_pages;
     std::vector<int> h_len, h_prompt, h_reported;
-    std::vector<char> prefilled;
+    std::vector<char> prefilled, finished;   // finished: the sequence ended on an end-of-sequence token (eos_tok)
+    std::vector<int> eos_tok;
     int32_t *pinned = nullptr; // small read-back area
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     int path = 0;
@@ -100,10 +106,11 @@ struct ada_session {
     bool mega = false;
     int grid = 0;
     mg::MegaArgs margs;
-    CUtensorMap *maps_dev = nullptr;      // [5 L + 2]: wqkv, wo, wgu, wdown per layer, lm_head, then T per 1-based layer
+    CUtensorMap *maps_dev = nullptr;      // [6 L + 2]: wqkv, wo, wgu, wup, wdown per layer, lm_head, then T per 1-based layer
     mg::MegaModel *mm_dev = nullptr;
     int *exit_at_dev = nullptr;
     int steps_per_launch = 256;
+    unsigned long long wait_ns = st::WAIT_NS_DEFAULT;
     int64_t launches = 0, syncs = 0, layer_passes = 0;
     // per-class profiling
     bool prof = false;
@@ -127,7 +134,7 @@ namespace {
 // Scratch layout (all offsets 256-byte aligned).
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
-        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qkvraw, attn_cnt, rope_freq, part,
+        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qfrag, attn_cnt, rope_freq, part,
         grid_ctr, pub, err, total;
 };
 
@@ -166,7 +173,7 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
     L.t_out = take(sizeof(float) * (size_t)R * g.d_model);
     // persistent-kernel buffers (bf16 models)
     if (g.dtype == ADA_DTYPE_BF16) {
-        L.maps = take(sizeof(CUtensorMap) * (5 * (size_t)g.n_layers + 2));
+        L.maps = take(sizeof(CUtensorMap) * (6 * (size_t)g.n_layers + 2));
         L.mm = take(sizeof(mg::MegaModel));
         L.exit_at = take(sizeof(int) * (g.n_layers + 1));
         L.xa = take(st::xfrag_bytes(g.d_model));
@@ -177,7 +184,7 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
         L.xh = take(st::xfrag_bytes(g.d_ff));
         L.ssq_a = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
         L.ssq_b = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
-        L.qkvraw = take(sizeof(float) * (size_t)st::MAX_COLS * qkv_rows);
+        L.qfrag = take((size_t)g.n_kv_heads * 2 * (g.head_dim / 16) * 1024);
         L.attn_cnt = take(sizeof(unsigned) * g.n_kv_heads);
         L.rope_freq = take(sizeof(double) * (g.head_dim / 2));
         L.part = take(kPartBytesPerCta * kPartMaxGrid);
@@ -289,7 +296,17 @@ int run_layer_t(ada_session *S, int layer, int rows) {
     }
     CK(cudaGetLastError());
     S->launches++;
-    if ((rc = launch_gemv<T>(S, 2, 0, w.wqkv, qkv_rows, d, S->c.xn, ldx, S->c.qkv, qkv_rows, layer))) return rc;
+    {
+        const int kvd = g.n_kv_heads * g.head_dim;
+        const bool fused = (const T *)w.wk == (const T *)w.wq + (size_t)qd * d && (const T *)w.wv == (const T *)w.wk + (size_t)kvd * d;
+        if (fused) {
+            if ((rc = launch_gemv<T>(S, 2, 0, w.wq, qkv_rows, d, S->c.xn, ldx, S->c.qkv, qkv_rows, layer))) return rc;
+        } else {
+            if ((rc = launch_gemv<T>(S, 2, 0, w.wq, qd, d, S->c.xn, ldx, S->c.qkv, qkv_rows, layer))) return rc;
+            if ((rc = launch_gemv<T>(S, 2, 0, w.wk, kvd, d, S->c.xn, ldx, S->c.qkv + qd, qkv_rows, layer))) return rc;
+            if ((rc = launch_gemv<T>(S, 2, 0, w.wv, kvd, d, S->c.xn, ldx, S->c.qkv + qd + kvd, qkv_rows, layer))) return rc;
+        }
+    }
     {
         Prof pf(S, 3, 0.0);
         k_rope_kv<T><<<rows, 128, 0, S->stream>>>(S->c, layer);
@@ -304,7 +321,12 @@ int run_layer_t(ada_session *S, int layer, int rows) {
     }
     CK(cudaGetLastError());
     S->launches++;
-    if ((rc = launch_gemv<T>(S, 6, 0, w.w_gate_up, 2 * g.d_ff, d, S->c.xn, ldx, S->c.gu, 2 * g.d_ff, layer))) return rc;
+    if ((const T *)w.w_up == (const T *)w.w_gate + (size_t)g.d_ff * d) {
+        if ((rc = launch_gemv<T>(S, 6, 0, w.w_gate, 2 * g.d_ff, d, S->c.xn, ldx, S->c.gu, 2 * g.d_ff, layer))) return rc;
+    } else {
+        if ((rc = launch_gemv<T>(S, 6, 0, w.w_gate, g.d_ff, d, S->c.xn, ldx, S->c.gu, 2 * g.d_ff, layer))) return rc;
+        if ((rc = launch_gemv<T>(S, 6, 0, w.w_up, g.d_ff, d, S->c.xn, ldx, S->c.gu + g.d_ff, 2 * g.d_ff, layer))) return rc;
+    }
     {
         Prof pf(S, 7, 0.0);
         k_swiglu<<<dim3((g.d_ff + 255) / 256, rows), 256, 0, S->stream>>>(S->c, layer);
@@ -414,6 +436,7 @@ void add_stats(ada_session *S, const DevStats &d, ada_stats *out, float ms, int6
     out->host_syncs += S->syncs - s0;
     out->kernel_launches += S->launches - l0;
     out->decode_ms += ms;
+    out->path = (S->mega && S->path == 1) ? 1 : 0;
 }
 
 // ---- persistent-kernel path --------------------------------------------------------------------
@@ -421,27 +444,42 @@ void add_stats(ada_session *S, const DevStats &d, ada_stats *out, float ms, int6
 template <int HD> const void *persistent_kernel() { return (const void *)mg::k_decode_persistent<HD>; }
 const void *persistent_kernel_for(int hd) { return hd == 64 ? persistent_kernel<64>() : persistent_kernel<128>(); }
 
+// Whether a model's shape and dtype are ones the persistent kernel is built for (the session adds its
+// own conditions: one sequence, at most eight token columns, 64-token pages).
+bool model_fits_persistent(const ada_config &g) {
+    const int qd = g.n_q_heads * g.head_dim, group = g.n_q_heads / g.n_kv_heads;
+    if (g.dtype != ADA_DTYPE_BF16) return false;
+    if ((g.head_dim != 64 && g.head_dim != 128) || group > 4) return false;
+    if (g.d_model % 64 || qd % 64 || g.d_ff % 64) return false;
+    return true;
+}
+
 // Decide whether this session can run the persistent kernel and build what it needs: tensor maps
-// of every weight matrix, the device-side model description, the argument block.
+// of every weight matrix, the device-side model description, the argument block.  A session that
+// does not qualify runs one kernel per operation (path 0) and says so through ada_debug_get_path and
+// ada_stats.path; a session that qualifies but cannot be set up (no cooperative launch, a tensor map
+// the driver refuses) fails with that error instead of quietly taking the slow path.
 int setup_persistent(ada_session *S, const Layout &lay) {
     const ada_model *m = S->m;
     const ada_config &g = m->cfg;
     S->mega = false;
     S->path = 0;
-    const int qd = g.n_q_heads * g.head_dim, group = g.n_q_heads / g.n_kv_heads;
-    if (g.dtype != ADA_DTYPE_BF16 || S->batch != 1 || S->slots > st::MAX_COLS || S->page_tokens != mg::ATT_PAGE) return ADA_OK;
-    if ((g.head_dim != 64 && g.head_dim != 128) || group > 4) return ADA_OK;
-    if (g.d_model % 64 || qd % 64 || g.d_ff % 64) return ADA_OK;
+    const int qd = g.n_q_heads * g.head_dim;
+    if (!model_fits_persistent(g) || S->batch != 1 || S->slots > st::MAX_COLS || S->page_tokens != mg::ATT_PAGE) return ADA_OK;
     int dev = 0, sms = 0, coop = 0, nb = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return ADA_OK; }
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    CK(cudaGetDevice(&dev));
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CK(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     const void *kern = persistent_kernel_for(g.head_dim);
-    if (!coop || sms < 1 ||
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st::SMEM_BYTES) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, st::THREADS, st::SMEM_BYTES) != cudaSuccess || nb < 1) {
-        cudaGetLastError();
-        return ADA_OK;
+    if (!coop || sms < 1) {
+        g_cuda_err = "the device does not support cooperative launches, which the persistent decode kernel needs";
+        return ADA_EUNSUPPORTED;
+    }
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st::SMEM_BYTES));
+    CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, st::THREADS, st::SMEM_BYTES));
+    if (nb < 1) {
+        g_cuda_err = "the persistent decode kernel does not fit on one multiprocessor of this device";
+        return ADA_EUNSUPPORTED;
     }
     S->grid = std::min(sms, S->head_blocks);
     const int L = g.n_layers;
@@ -449,26 +487,30 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     S->maps_dev = (CUtensorMap *)(b + lay.maps);
     S->mm_dev = (mg::MegaModel *)(b + lay.mm);
     S->exit_at_dev = (int *)(b + lay.exit_at);
-    S->maps_host.assign(5 * (size_t)L + 2, CUtensorMap());
+    S->maps_host.assign(6 * (size_t)L + 2, CUtensorMap());
     S->mm_host.reset(new mg::MegaModel());
     mg::MegaModel &M = *S->mm_host;
     memset(&M, 0, sizeof(M));
+    int rc;
     for (int l = 0; l < L; ++l) {
         const LayerW &w = m->layers[l];
-        if (make_weight_map(&S->maps_host[4 * l + 0], w.wqkv, S->c.qkv_rows, g.d_model) ||
-            make_weight_map(&S->maps_host[4 * l + 1], w.wo, g.d_model, qd) ||
-            make_weight_map(&S->maps_host[4 * l + 2], w.w_gate_up, 2 * g.d_ff, g.d_model) ||
-            make_weight_map(&S->maps_host[4 * l + 3], w.w_down, g.d_model, g.d_ff))
-            return ADA_OK;
-        M.layer[l].wqkv = S->maps_dev + 4 * l + 0;
-        M.layer[l].wo = S->maps_dev + 4 * l + 1;
-        M.layer[l].wgu = S->maps_dev + 4 * l + 2;
-        M.layer[l].wdown = S->maps_dev + 4 * l + 3;
+        const bool gu_fused = (const __nv_bfloat16 *)w.w_up == (const __nv_bfloat16 *)w.w_gate + (size_t)g.d_ff * g.d_model;
+        if (!w.wqkv_perm) return ADA_ESTATE;
+        if ((rc = make_weight_map(&S->maps_host[5 * l + 0], w.wqkv_perm, S->c.qkv_rows, g.d_model))) return rc;
+        if ((rc = make_weight_map(&S->maps_host[5 * l + 1], w.wo, g.d_model, qd))) return rc;
+        if ((rc = make_weight_map(&S->maps_host[5 * l + 2], w.w_gate, gu_fused ? 2 * g.d_ff : g.d_ff, g.d_model))) return rc;
+        if (!gu_fused && (rc = make_weight_map(&S->maps_host[5 * l + 3], w.w_up, g.d_ff, g.d_model))) return rc;
+        if ((rc = make_weight_map(&S->maps_host[5 * l + 4], w.w_down, g.d_model, g.d_ff))) return rc;
+        M.layer[l].wqkv = S->maps_dev + 5 * l + 0;
+        M.layer[l].wo = S->maps_dev + 5 * l + 1;
+        M.layer[l].wgu = S->maps_dev + 5 * l + 2;
+        M.layer[l].wup = gu_fused ? nullptr : S->maps_dev + 5 * l + 3;
+        M.layer[l].wdown = S->maps_dev + 5 * l + 4;
         M.layer[l].attn_norm = (const __nv_bfloat16 *)w.attn_norm;
         M.layer[l].ffn_norm = (const __nv_bfloat16 *)w.ffn_norm;
     }
-    if (make_weight_map(&S->maps_host[4 * L], m->lm_head, g.vocab, g.d_model)) return ADA_OK;
-    M.lm_head = S->maps_dev + 4 * L;
+    if ((rc = make_weight_map(&S->maps_host[5 * L], m->lm_head, g.vocab, g.d_model))) return rc;
+    M.lm_head = S->maps_dev + 5 * L;
     M.tok_embed = (const __nv_bfloat16 *)m->tok_embed;
     M.final_norm = (const __nv_bfloat16 *)m->final_norm;
     M.rope_base = g.rope_base;
@@ -485,7 +527,7 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.XA = (__nv_bfloat16 *)(b + lay.xa); a.XB = (__nv_bfloat16 *)(b + lay.xb); a.XO = (__nv_bfloat16 *)(b + lay.xo);
     a.XH = (__nv_bfloat16 *)(b + lay.xh); a.XF = (__nv_bfloat16 *)(b + lay.xf); a.XT = (__nv_bfloat16 *)(b + lay.xt);
     a.ssq_a = (float *)(b + lay.ssq_a); a.ssq_b = (float *)(b + lay.ssq_b);
-    a.qkvraw = (float *)(b + lay.qkvraw);
+    a.qfrag = (uint32_t *)(b + lay.qfrag);
     a.attn_part = S->c.attn_part;
     a.head_part = S->c.head_part;
     a.attn_cnt = (unsigned *)(b + lay.attn_cnt);
@@ -495,6 +537,7 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.pub = (mg::Pub *)(b + lay.pub);
     a.err = (int *)(b + lay.err);
     a.step_budget = S->steps_per_launch;
+    a.wait_ns = S->wait_ns;
     a.store_logits = 0;
     a.trace = st::Trace{nullptr, nullptr, 0};
     a.trace_step0 = a.trace_step1 = 0;
@@ -518,21 +561,25 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
             M.layer[e].head_scale = m->head_scale[e];
             M.layer[e].wT = nullptr;
             if (m->head_T[e]) {
-                CUtensorMap &tm = S->maps_host[4 * (size_t)L + 1 + e];
+                CUtensorMap &tm = S->maps_host[5 * (size_t)L + 1 + e];
                 int rc = make_weight_map(&tm, m->head_T[e], g.d_model, g.d_model);
                 if (rc) return rc;
-                CK(cudaMemcpyAsync(S->maps_dev + 4 * L + 1 + e, &tm, sizeof(tm), cudaMemcpyHostToDevice, S->stream));
-                M.layer[e].wT = S->maps_dev + 4 * L + 1 + e;
+                CK(cudaMemcpyAsync(S->maps_dev + 5 * L + 1 + e, &tm, sizeof(tm), cudaMemcpyHostToDevice, S->stream));
+                M.layer[e].wT = S->maps_dev + 5 * L + 1 + e;
             }
             CK(cudaMemcpyAsync(&S->mm_dev->layer[e], &M.layer[e], sizeof(mg::MegaLayer), cudaMemcpyHostToDevice, S->stream));
         }
     }
     CK(cudaMemcpyAsync(S->exit_at_dev, ex.data(), sizeof(int) * (L + 1), cudaMemcpyHostToDevice, S->stream));
+    // a call that ended on a device-side error may have left the error word and the attention counters set
+    CK(cudaMemsetAsync(S->margs.err, 0, sizeof(int), S->stream));
+    CK(cudaMemsetAsync(S->margs.attn_cnt, 0, sizeof(unsigned) * g.n_kv_heads, S->stream));
     CK(cudaStreamSynchronize(S->stream));   // ex and the maps live on the host until copied
     S->syncs++;
     mg::MegaArgs a = S->margs;
     a.c = S->c;   // capture pointers may have changed
     a.step_budget = S->steps_per_launch;
+    a.wait_ns = S->wait_ns;
     a.store_logits = S->capture_dev ? 1 : 0;
     const void *kern = persistent_kernel_for(g.head_dim);
     for (long long guard = 0;; ++guard) {
@@ -557,12 +604,18 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
 }
 
 // Shared body of both decode calls.
-int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers, int n_exit, int max_early,
+int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers, int n_exit, int max_early, int eos_id,
            int32_t *out_host, ada_stats *stats) {
     const ada_model *m = S->m;
     const int L = m->cfg.n_layers;
-    if (!out_host || n_tokens < 1) return ADA_EINVAL;
-    for (int s = 0; s < S->batch; ++s) if (!S->prefilled[s]) return ADA_ESTATE;
+    if (!out_host || n_tokens < 1 || eos_id >= m->cfg.vocab) return ADA_EINVAL;
+    if (eos_id < 0) eos_id = -1;
+    int n_live = 0;
+    for (int s = 0; s < S->batch; ++s) {
+        if (!S->prefilled[s]) return ADA_ESTATE;
+        n_live += !S->finished[s];
+    }
+    if (n_live == 0) return ADA_ESTATE;   // every sequence has already ended on its end-of-sequence token
     if (max_early < 0 || max_early > S->max_early) return ADA_ECAPACITY;
     for (int e = 0; e < n_exit; ++e) {
         if (exit_layers[e] < 1 || exit_layers[e] >= L || !m->has_head[exit_layers[e]]) return ADA_EINVAL;
@@ -572,7 +625,7 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
     memset(&tg, 0, sizeof(tg));
     int max_steps_plain = 0;
     for (int s = 0; s < S->batch; ++s) {
-        int target = S->h_prompt[s] + S->h_reported[s] + n_tokens;
+        int target = S->h_prompt[s] + S->h_reported[s] + (S->finished[s] ? 0 : n_tokens);
         if (target + 1 > S->max_seq) return ADA_ECAPACITY;
         int rc = ensure_pages(S, s, target + 1);
         if (rc) return rc;
@@ -587,7 +640,7 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
     int tape_n = (int)std::min<size_t>(S->tape.size(), kMaxTape);
     if (tape_n) CK(cudaMemcpyAsync(S->c.st->tape, S->tape.data(), tape_n, cudaMemcpyHostToDevice, S->stream));
     CK(cudaEventRecord(S->ev0, S->stream));
-    k_call_begin<<<1, 32, 0, S->stream>>>(S->c, tg, gamma, max_early, tape_n);
+    k_call_begin<<<1, 32, 0, S->stream>>>(S->c, tg, gamma, max_early, tape_n, eos_id);
     CK(cudaGetLastError());
     S->launches++;
 
@@ -647,20 +700,45 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
         }
     }
     CK(cudaEventRecord(S->ev1, S->stream));
-    // results
-    for (int s = 0; s < S->batch; ++s) {
-        CK(cudaMemcpyAsync(out_host + (size_t)s * n_tokens,
-                           S->c.tokens + (size_t)s * S->max_seq + S->h_prompt[s] + S->h_reported[s],
-                           sizeof(int32_t) * n_tokens, cudaMemcpyDeviceToHost, S->stream));
-    }
+    // results: how far every sequence got (a verified end-of-sequence token ends it before the requested
+    // count), then its tokens
+    int32_t len_host[ADA_MAX_BATCH], eos_host[ADA_MAX_BATCH];
+    CK(cudaMemcpyAsync(len_host, S->c.st->len, sizeof(int32_t) * S->batch, cudaMemcpyDeviceToHost, S->stream));
+    CK(cudaMemcpyAsync(eos_host, S->c.st->eos_hit, sizeof(int32_t) * S->batch, cudaMemcpyDeviceToHost, S->stream));
     DevStats ds;
     CK(cudaMemcpyAsync(&ds, &S->c.st->st, sizeof(DevStats), cudaMemcpyDeviceToHost, S->stream));
     int32_t hl_n = 0;
     if (S->head_log_host) {
         CK(cudaMemcpyAsync(&hl_n, &S->c.st->head_log_n, sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
     }
+    if (eos_id < 0) {   // no end-of-sequence token: every sequence still running delivers the requested count
+        for (int s = 0; s < S->batch; ++s) {
+            if (S->finished[s]) {
+                for (int i = 0; i < n_tokens; ++i) out_host[(size_t)s * n_tokens + i] = S->eos_tok[s];
+                continue;
+            }
+            CK(cudaMemcpyAsync(out_host + (size_t)s * n_tokens, S->c.tokens + (size_t)s * S->max_seq + S->h_prompt[s] + S->h_reported[s],
+                               sizeof(int32_t) * n_tokens, cudaMemcpyDeviceToHost, S->stream));
+        }
+    }
     CK(cudaStreamSynchronize(S->stream));
     S->syncs++;
+    int emitted[ADA_MAX_BATCH];
+    for (int s = 0; s < S->batch; ++s) {
+        emitted[s] = eos_id < 0 ? n_tokens : std::min(n_tokens, std::max(0, len_host[s] - (S->h_prompt[s] + S->h_reported[s])));
+        if (S->finished[s]) emitted[s] = 0;
+    }
+    if (eos_id >= 0) {
+        for (int s = 0; s < S->batch; ++s) {
+            int32_t *row = out_host + (size_t)s * n_tokens;
+            if (emitted[s] > 0)
+                CK(cudaMemcpyAsync(row, S->c.tokens + (size_t)s * S->max_seq + S->h_prompt[s] + S->h_reported[s],
+                                   sizeof(int32_t) * emitted[s], cudaMemcpyDeviceToHost, S->stream));
+            for (int i = emitted[s]; i < n_tokens; ++i) row[i] = S->finished[s] ? S->eos_tok[s] : eos_id;
+        }
+        CK(cudaStreamSynchronize(S->stream));
+        S->syncs++;
+    }
     if (S->head_log_host) {
         int n = std::min(hl_n, S->head_log_cap);
         if (n > 0) CK(cudaMemcpy(S->head_log_host, S->c.head_log, sizeof(float) * 4 * n, cudaMemcpyDeviceToHost));
@@ -669,8 +747,14 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
     float ms = 0.f;
     CK(cudaEventElapsedTime(&ms, S->ev0, S->ev1));
     for (int s = 0; s < S->batch; ++s) {
-        S->h_reported[s] += n_tokens;
-        S->h_len[s] = tg.target_len[s];
+        S->h_reported[s] += emitted[s];
+        S->h_len[s] = S->h_prompt[s] + S->h_reported[s];
+        if (eos_id >= 0 && eos_host[s] && !S->finished[s]) {
+            S->finished[s] = 1;
+            S->eos_tok[s] = eos_id;
+            if (stats) stats->finished += 1;
+        }
+        if (stats) stats->emitted[s] += emitted[s];
     }
     S->tape.clear();
     if (S->prof) {
@@ -746,16 +830,48 @@ int ada_model_set_tensor(ada_model *m, const char *name, const void *dev_ptr, si
         if (l < 0 || l >= g.n_layers) return ADA_EINVAL;
         std::string f = n.substr(dot + 1);
         LayerW &w = m->layers[l];
+        const size_t kvd = (size_t)g.n_kv_heads * g.head_dim;
+        const char *base = (const char *)dev_ptr;
         if (f == "attn_norm") { want = d; slot = &w.attn_norm; }
         else if (f == "ffn_norm") { want = d; slot = &w.ffn_norm; }
-        else if (f == "wqkv") { want = qkv_rows * d; slot = &w.wqkv; }
+        else if (f == "wq") { want = qd * d; slot = &w.wq; }
+        else if (f == "wk") { want = kvd * d; slot = &w.wk; }
+        else if (f == "wv") { want = kvd * d; slot = &w.wv; }
+        else if (f == "wqkv") {   // the three matrices stacked in one tensor: q rows, k rows, v rows
+            if (bytes != qkv_rows * d * m->esz) return ADA_EINVAL;
+            w.wq = base; w.wk = base + qd * d * m->esz; w.wv = base + (qd + kvd) * d * m->esz;
+            return ADA_OK;
+        }
         else if (f == "wo") { want = d * qd; slot = &w.wo; }
-        else if (f == "w_gate_up") { want = 2 * (size_t)g.d_ff * d; slot = &w.w_gate_up; }
+        else if (f == "w_gate") { want = (size_t)g.d_ff * d; slot = &w.w_gate; }
+        else if (f == "w_up") { want = (size_t)g.d_ff * d; slot = &w.w_up; }
+        else if (f == "w_gate_up") {   // gate rows stacked over up rows
+            if (bytes != 2 * (size_t)g.d_ff * d * m->esz) return ADA_EINVAL;
+            w.w_gate = base; w.w_up = base + (size_t)g.d_ff * d * m->esz;
+            return ADA_OK;
+        }
         else if (f == "w_down") { want = d * (size_t)g.d_ff; slot = &w.w_down; }
         else return ADA_EINVAL;
     } else return ADA_EINVAL;
     if (bytes != want * m->esz) return ADA_EINVAL;
     *slot = dev_ptr;
+    return ADA_OK;
+}
+
+size_t ada_model_arena_bytes(const ada_model *m) {
+    if (!m || !model_fits_persistent(m->cfg)) return 0;
+    const ada_config &g = m->cfg;
+    const size_t per_layer = align_up((size_t)(g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim * g.d_model * 2, 256);
+    return per_layer * g.n_layers;
+}
+
+int ada_model_set_arena(ada_model *m, void *arena_dev, size_t bytes) {
+    if (!m || !arena_dev) return ADA_EINVAL;
+    if (m->finalized) return ADA_ESTATE;
+    if ((uintptr_t)arena_dev % 256) return ADA_EINVAL;
+    if (bytes < ada_model_arena_bytes(m)) return ADA_ECAPACITY;
+    m->arena = arena_dev;
+    m->arena_bytes = bytes;
     return ADA_OK;
 }
 
@@ -772,11 +888,33 @@ int ada_model_set_exit_head(ada_model *m, int32_t layer, const void *T_dev, floa
 
 int ada_model_finalize(ada_model *m) {
     if (!m) return ADA_EINVAL;
+    if (m->finalized) return ADA_OK;
     if (!m->tok_embed || !m->final_norm) return ADA_ESTATE;
     if (m->cfg.tied_lm_head) m->lm_head = m->tok_embed;
     if (!m->lm_head) return ADA_ESTATE;
     for (const LayerW &w : m->layers)
-        if (!w.attn_norm || !w.wqkv || !w.wo || !w.ffn_norm || !w.w_gate_up || !w.w_down) return ADA_ESTATE;
+        if (!w.attn_norm || !w.wq || !w.wk || !w.wv || !w.wo || !w.ffn_norm || !w.w_gate || !w.w_up || !w.w_down) return ADA_ESTATE;
+    const size_t need = ada_model_arena_bytes(m);
+    if (need) {
+        // Repack on load: q | k | v of every layer, copied into the caller's arena with the rows of each q and
+        // k head reordered (see k_repack_qkv).  The tensors the caller lent stay as they are.
+        if (!m->arena || m->arena_bytes < need) {
+            g_cuda_err = "ada_model_finalize: this model needs an arena of ada_model_arena_bytes() bytes (ada_model_set_arena)";
+            return ADA_ESTATE;
+        }
+        const ada_config &g = m->cfg;
+        const size_t per_layer = need / g.n_layers;
+        const int rows = (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim;
+        for (int l = 0; l < g.n_layers; ++l) {
+            LayerW &w = m->layers[l];
+            __nv_bfloat16 *dst = (__nv_bfloat16 *)((char *)m->arena + per_layer * l);
+            mg::k_repack_qkv<<<rows, 128>>>((const __nv_bfloat16 *)w.wq, (const __nv_bfloat16 *)w.wk, (const __nv_bfloat16 *)w.wv, dst,
+                                            g.n_q_heads, g.n_kv_heads, g.head_dim, g.d_model);
+            CK(cudaGetLastError());
+            w.wqkv_perm = dst;
+        }
+        CK(cudaDeviceSynchronize());
+    }
     m->finalized = true;
     return ADA_OK;
 }
@@ -880,6 +1018,8 @@ int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, i
     S->seq_pages.resize(batch);
     S->h_len.assign(batch, 0); S->h_prompt.assign(batch, 0); S->h_reported.assign(batch, 0);
     S->prefilled.assign(batch, 0);
+    S->finished.assign(batch, 0);
+    S->eos_tok.assign(batch, -1);
     *out = S;
     return ADA_OK;
 }
@@ -900,6 +1040,7 @@ int ada_session_reset(ada_session *S, int32_t seq) {
         for (int p : S->seq_pages[s]) S->free_pages.push_back(p);
         S->seq_pages[s].clear();
         S->prefilled[s] = 0;
+        S->finished[s] = 0;
         S->h_len[s] = S->h_prompt[s] = S->h_reported[s] = 0;
     }
     return ADA_OK;
@@ -954,15 +1095,21 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
     return ADA_OK;
 }
 
-int ada_plain_decode(ada_session *S, int32_t n_tokens, int32_t *out_host, ada_stats *stats) {
+int ada_plain_decode(ada_session *S, int32_t n_tokens, int32_t eos_id, int32_t *out_host, ada_stats *stats) {
     if (!S) return ADA_EINVAL;
-    return decode(S, n_tokens, 2.0f, nullptr, 0, 0, out_host, stats);
+    return decode(S, n_tokens, 2.0f, nullptr, 0, 0, eos_id, out_host, stats);
 }
 
 int ada_adaptive_decode(ada_session *S, int32_t n_tokens, float threshold, const int32_t *exit_layers,
-                        int32_t n_exit_layers, int32_t max_early, int32_t *out_host, ada_stats *stats) {
+                        int32_t n_exit_layers, int32_t max_early, int32_t eos_id, int32_t *out_host, ada_stats *stats) {
     if (!S || n_exit_layers < 0 || (n_exit_layers > 0 && !exit_layers)) return ADA_EINVAL;
-    return decode(S, n_tokens, threshold, exit_layers, n_exit_layers, max_early, out_host, stats);
+    return decode(S, n_tokens, threshold, exit_layers, n_exit_layers, max_early, eos_id, out_host, stats);
+}
+
+int ada_debug_set_wait_limit(ada_session *S, uint64_t ns) {
+    if (!S || ns < 1) return ADA_EINVAL;
+    S->wait_ns = ns;
+    return ADA_OK;
 }
 
 int ada_debug_capture_logits(ada_session *S, float *dev_buf, int32_t max_tokens) {

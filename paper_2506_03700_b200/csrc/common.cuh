@@ -45,6 +45,8 @@ struct DevState {
     // parameters of the current adaptive call
     float gamma;
     int32_t max_early;
+    int32_t eos_id;                     // end-of-sequence token of the current call (-1: none)
+    int32_t eos_hit[ADA_MAX_BATCH];     // the call ended this sequence on a verified end-of-sequence token
     // debug: forced decisions (sequence 0), head log, logits capture
     int32_t tape_n, tape_i;
     uint8_t tape[kMaxTape];

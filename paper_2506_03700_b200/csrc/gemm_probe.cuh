@@ -22,7 +22,7 @@ k_gemm_probe(const CUtensorMap *__restrict__ W, int N, int K, int mode, const ui
     st::Smem *sm = st::smem_base(smem_raw);
     st::smem_init(sm);
     __syncthreads();
-    st::Shared S{sm, err, st::Trace{nullptr, nullptr, 0}, 0};
+    st::Shared S{sm, err, st::Trace{nullptr, nullptr, 0}, 0, st::WAIT_NS_DEFAULT};
     st::Gemm g;
     g.W = W; g.X = X; g.N = N; g.K = K; g.pair = mode == 1 ? 2 : 1; g.half = mode == 1 ? N / 2 : 0;
     g.ctas = st::balanced_ctas(g.tiles(), gridDim.x);

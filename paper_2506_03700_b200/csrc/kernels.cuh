@@ -599,19 +599,29 @@ __global__ void k_verify(Ctx c) {
                 tok[new_base] = c.head_res[s * c.slots + bad].token;
                 keep = bad + 1;
             }
+            // "while t_i != [EOS]" (Algorithm 1): the first verified end-of-sequence token ends the sequence
+            int target = st->target_len[s];
+            if (st->eos_id >= 0) {
+                for (int j = 0; j < keep; ++j)
+                    if (c.head_res[s * c.slots + j].token == st->eos_id) {
+                        if (base + j + 2 <= target) { target = base + j + 2; st->eos_hit[s] = 1; }
+                        break;
+                    }
+            }
             int new_len = new_base + 1;
-            if (new_len > st->target_len[s]) {
-                st->st.truncated += new_len - st->target_len[s];
-                new_len = st->target_len[s];
+            if (new_len > target) {
+                st->st.truncated += new_len - target;
+                new_len = target;
                 new_base = new_len - 1;
             }
+            keep = new_len - 1 - base;   // verified tokens that stay
             for (int l = 0; l < c.L; ++l) c.fill[s * c.L + l] = new_base;
             st->len[s] = new_len;
             st->base[s] = new_base;
             st->st.verify_steps++;
             st->st.steps++;
             st->climbing[s] = 0;
-            if (new_len >= st->target_len[s]) st->done[s] = 1;
+            if (new_len >= target) st->done[s] = 1;
             if (s == 0) st->keep_rows = keep;
         } else if (s == 0) {
             st->keep_rows = 0;
@@ -639,13 +649,21 @@ __global__ void k_capture_advance(Ctx c) {
 
 // Start of a decode call: set targets and parameters.
 struct CallTargets { int32_t target_len[ADA_MAX_BATCH]; };
-__global__ void k_call_begin(Ctx c, CallTargets tg, float gamma, int max_early, int tape_n) {
+__global__ void k_call_begin(Ctx c, CallTargets tg, float gamma, int max_early, int tape_n, int eos_id) {
     DevState *st = c.st;
     if (threadIdx.x != 0) return;
     int ndone = 0;
+    st->eos_id = eos_id;
     for (int s = 0; s < st->batch; ++s) {
         st->target_len[s] = tg.target_len[s];
-        st->done[s] = st->len[s] >= tg.target_len[s];
+        st->eos_hit[s] = 0;
+        // the pending token (verified, not yet returned) may itself be the end-of-sequence token
+        if (eos_id >= 0 && st->len[s] >= 1 && st->len[s] <= tg.target_len[s] &&
+            c.tokens[(size_t)s * c.max_seq + st->len[s] - 1] == eos_id) {
+            st->target_len[s] = st->len[s];
+            st->eos_hit[s] = 1;
+        }
+        st->done[s] = st->len[s] >= st->target_len[s];
         st->climbing[s] = 0;
         ndone += st->done[s];
     }

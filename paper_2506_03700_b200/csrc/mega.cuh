@@ -52,7 +52,9 @@ struct Pub {                   // what CTA 0 publishes at a control point
 };
 
 struct MegaLayer {
-    const CUtensorMap *wqkv, *wo, *wgu, *wdown, *wT;
+    // wqkv: the fused q | k | v matrix with the rows of every q and k head reordered for the rotation (see the QKV phase);
+    // wgu: gate stacked over up, or the gate matrix alone when wup is set (the two lent as separate tensors)
+    const CUtensorMap *wqkv, *wo, *wgu, *wup, *wdown, *wT;
     const __nv_bfloat16 *attn_norm, *ffn_norm;
     float head_scale;
     int has_head;
@@ -72,7 +74,7 @@ struct MegaArgs {
     const int *exit_at;        // [L + 1]: 1 if this call consults the head after 1-based layer e
     __nv_bfloat16 *XA, *XB, *XO, *XH, *XF, *XT;   // GEMM inputs in fragment layout (see stream.cuh)
     float *ssq_a, *ssq_b;      // [d/16][8] partial sums of squares of the residual (per 16-feature tile, per column)
-    float *qkvraw;             // [8][qkv_rows]
+    uint32_t *qfrag;           // [nkv][2][hd/16][32][8]: rotated, scaled queries as tensor-core A fragments (bf16 high parts, then low parts)
     float *attn_part;          // [8 * nq][n_chunks][hd + 4]
     float *head_part;          // [grid][8][4]
     const double *rope_freq;   // [hd/2]: base^(-2i/hd), computed once on the host
@@ -82,6 +84,7 @@ struct MegaArgs {
     Pub *pub;                  // [2]
     int *err;
     int step_budget;           // steps this launch may start
+    unsigned long long wait_ns;   // a single device-side wait gives up after this long
     int store_logits;
     Trace trace;               // test hook: event trace of the steps [trace_step0, trace_step1) of this launch
     int trace_step0, trace_step1;
@@ -214,6 +217,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
         const int pf_end0 = st->pf_end, pf_pos0 = st->pf_pos, max_early0 = st->max_early;
         const int tape_n0 = st->tape_n, tape_i0 = st->tape_i, hl_n0 = st->head_log_n;
         const float gamma0 = st->gamma;
+        const int eos0 = st->eos_id;
         const long long steps0 = __ldcg(&st->st.steps);   // past the L1: the counters are bumped by reductions
         int action = ACT_NEWSTEP, verified = 0;
         int len = len0, base = base0, done = done0, pf_end = pf_end0, pf_pos = pf_pos0;
@@ -295,12 +299,24 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
                 tok[new_base] = min(max(hr_s[bad].token, 0), c.vocab - 1);
                 keep = bad + 1;
             }
+            // Algorithm 1 runs "while t_i != [EOS]": the verified tokens of this step (positions base + 1 .. new_base,
+            // each equal to the full-depth argmax of the row before it) end the sequence at the first end-of-sequence
+            // token among them.  An early-predicted end-of-sequence token stops nothing until it is verified here.
+            int target = target0;
+            if (eos0 >= 0) {
+                for (int j = 0; j < keep; ++j)
+                    if (min(max(hr_s[j].token, 0), c.vocab - 1) == eos0) {
+                        if (base + j + 2 <= target) { target = base + j + 2; st->eos_hit[0] = 1; }
+                        break;
+                    }
+            }
             int new_len = new_base + 1;
-            if (new_len > target0) {
-                bump(&st->st.truncated, new_len - target0);
-                new_len = target0;
+            if (new_len > target) {
+                bump(&st->st.truncated, new_len - target);
+                new_len = target;
                 new_base = new_len - 1;
             }
+            keep = new_len - 1 - base;   // verified tokens that stay: their logit rows are the ones a capture keeps
             for (int l = 0; l < c.L; ++l) { fill_s[l] = new_base; c.fill[l] = new_base; }
             len = new_len; base = new_base;
             st->len[0] = len;
@@ -308,7 +324,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
             bump(&st->st.verify_steps, 1);
             bump(&st->st.steps, 1);
             bump(&st->st.layer_passes, c.L);
-            if (new_len >= target0) { done = 1; st->done[0] = 1; }
+            if (new_len >= target) { done = 1; st->done[0] = 1; }
             st->keep_rows = keep;
             st->keep_row0 = 0;
             verified = 1;
@@ -450,6 +466,13 @@ __device__ __forceinline__ int control_point(const MegaArgs &A, const Shared &S,
             if (d.n_cols < 1 || d.n_cols > MAX_COLS || d.newest < 0 || d.newest >= MAX_COLS || d.pmax < 0 || d.pmax >= A.c.max_seq)
                 act = ACT_STOP;   // cannot happen unless memory was corrupted; never index with it
         }
+        // The two record slots alternate.  A role that fell two control points behind would find its slot
+        // already rewritten for a later one: a record is used only if its number is still the expected one
+        // after it has been copied.
+        if (!aborted(S) && ld_acquire(&pub->seq) != pub_no) {
+            raise_error(S, ERR_BAD_STATE);
+            act = ACT_STOP;
+        }
         return act;
     };
     if (ROLE == 2) {
@@ -489,18 +512,33 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// K/V producer: for every work item of this CTA, the K and V page blocks of its sub-blocks.
-__device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, Rings &r, uint64_t pol) {
+// K/V producer: for every work item of this CTA, the K and V page blocks of its sub-blocks.  The K and V
+// rows of the tokens of this pass were written into the cache by the QKV epilogues of other CTAs; a
+// work item whose positions include such a row is fetched only once the grid has passed the barrier
+// that ends the QKV phase (`bar_target`).  Every other item reads rows of earlier passes only and is
+// fetched as soon as ring slots are free, i.e. while the QKV product is still streaming.
+__device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, unsigned mask, unsigned bar_target,
+                                             Rings &r, uint64_t pol) {
     const Ctx &c = A.c;
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31, cta = blockIdx.x, G = gridDim.x;
     const int nchunk = d.pmax / ATT_CHUNK + 1, n_items = c.nkv * nchunk;
     const uint32_t bytes = (uint32_t)(ATT_PAGE * c.hd * 2);
     const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
+    bool synced = false;
     for (int item = cta; item < n_items; item += G) {
         const int kvh = item / nchunk, j = item - kvh * nchunk;
         const int p_base = j * ATT_CHUNK;
         const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.pmax - p_base) / ATT_PAGE + 1);
+        bool has_new = false;
+#pragma unroll
+        for (int cc = 0; cc < MAX_COLS; ++cc)
+            has_new = has_new || (((mask >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK);
+        if (has_new && !synced) {
+            grid_wait(S, A.grid_ctr, bar_target);
+            fence_proxy_async();
+            synced = true;
+        }
         for (int sb = 0; sb < nsb; ++sb) {
             const int page = c.page_table[(p_base + sb * ATT_PAGE) >> c.page_shift];
             for (int which = 0; which < 2; ++which) {
@@ -557,12 +595,11 @@ __device__ __forceinline__ void attn_merge_to(const float (&o)[NT][4], const flo
     }
 }
 
-// Consumers: causal attention of every active column over the cache plus the in-flight rows.
-// Work item = (kv head, 128-position chunk).  Within a 64-position sub-block warp (mt, qr) handles
-// query tile mt (16 of the up to 32 (column, q head) pairs of the kv head) and positions
-// [16 qr, 16 qr + 16).  K and V rows of the columns processed in this pass are not in the cache
-// yet: they are rotated / rounded here from the QKV output, patched into the shared-memory copy
-// and written to the cache by the item that owns their position.
+// Consumers: causal attention of every active column over the cache, which by now holds the rows
+// of this pass too (the QKV epilogue wrote them).  Work item = (kv head, 128-position chunk).
+// Within a 64-position sub-block warp (mt, qr) handles query tile mt (16 of the up to 32 (column,
+// q head) pairs of the kv head) and positions [16 qr, 16 qr + 16).  The queries arrive rotated,
+// scaled and split into bf16 high / low parts, laid out as the tensor-core A fragments.
 // x / group for the q heads per kv head the persistent path admits (1..4) and x < 128, without the
 // general integer division (some thirty of those sat on the critical path of every attention item)
 __device__ __forceinline__ int div_group(int x, int group) {
@@ -574,17 +611,14 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     const Ctx &c = A.c;
     Smem *sm = S.sm;
     AttnSmem<HD> *as = reinterpret_cast<AttnSmem<HD> *>(sm->scratch);
-    constexpr int KSQ = HD / 16, NT = HD / 8, HALF = HD / 2;
+    constexpr int KSQ = HD / 16, NT = HD / 8;
     constexpr int ATT_STRIDE = HD + 4;                     // floats per chunk partial: output, max, sum, padding (16-byte rows)
-    constexpr int QPT = 32 * HALF / CONS_THREADS;          // (query, rotation pair) items per thread
-    constexpr int KPT = MAX_COLS * HALF / CONS_THREADS;    // new-row K rotation pairs per thread
-    constexpr int VPT = MAX_COLS * HD / CONS_THREADS;      // new-row V elements per thread
+    constexpr int QV = 2 * KSQ * 64 / CONS_THREADS;        // 16-byte pieces of a kv head's query fragments per thread
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x, G = gridDim.x;
-    const int group = c.group, qd = c.nq * HD;
+    const int group = c.group;
     const int nchunk = d.pmax / ATT_CHUNK + 1, n_items = c.nkv * nchunk;
     const int mt = warp >> 2, qr = warp & 3;
-    const float scale = rsqrtf((float)HD);
-    __nv_bfloat16 *pool = reinterpret_cast<__nv_bfloat16 *>(c.kv_pool);
+    (void)layer;
     // Merge of the chunk partials of one kv head into the O-projection's input (by a whole CTA).
     auto merge_chunks = [&](int kvh) {
         // Four features of one (column, q head) per thread and pass; the chunk partials are folded in
@@ -637,71 +671,15 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
         const int kvh = item / nchunk, j = item - kvh * nchunk;
         const int p_base = j * ATT_CHUNK;
         const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.pmax - p_base) / ATT_PAGE + 1);
-        // columns of this pass whose (new) K/V row lies in this chunk
-        unsigned item_new = 0;
+        // ---- the kv head's query fragments: one round trip to L2, then shared memory
+        {
+            const uint4 *src = reinterpret_cast<const uint4 *>(A.qfrag) + (size_t)kvh * (2 * KSQ * 64);
+            uint4 v[QV];
 #pragma unroll
-        for (int cc = 0; cc < MAX_COLS; ++cc)
-            if (((mask >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK) item_new |= 1u << cc;
-        // ---- all global reads of the item are issued up front: queries, and the new rows' k / v
-        float qx0[QPT], qx1[QPT], qco[QPT], qsi[QPT];
+            for (int u = 0; u < QV; ++u) v[u] = __ldcg(src + tid + u * CONS_THREADS);
+            bar_consumers();   // the previous item is done with the shared buffers
 #pragma unroll
-        for (int u = 0; u < QPT; ++u) {
-            const int idx = tid + u * CONS_THREADS;
-            const int qcol = idx / HALF, jj = idx - qcol * HALF;
-            const int cc = div_group(qcol, group), g = qcol - cc * group;
-            qx0[u] = 0.f; qx1[u] = 0.f; qco[u] = 1.f; qsi[u] = 0.f;
-            if (cc < MAX_COLS && ((mask >> cc) & 1u)) {
-                const float *q = A.qkvraw + (size_t)cc * c.qkv_rows + (size_t)(kvh * group + g) * HD;
-                const float *cs = c.rope_cs + (size_t)cc * HALF * 2;
-                qx0[u] = __ldcg(q + jj); qx1[u] = __ldcg(q + jj + HALF); qco[u] = __ldcg(cs + 2 * jj); qsi[u] = __ldcg(cs + 2 * jj + 1);
-            }
-        }
-        __nv_bfloat16 nk0[KPT], nk1[KPT], nv[VPT];
-        if (item_new) {
-            float kx0[KPT], kx1[KPT], kco[KPT], ksi[KPT], vx[VPT];
-#pragma unroll
-            for (int u = 0; u < KPT; ++u) {
-                const int idx = tid + u * CONS_THREADS, cc = idx / HALF, jj = idx - cc * HALF;
-                kx0[u] = 0.f; kx1[u] = 0.f; kco[u] = 1.f; ksi[u] = 0.f;
-                if ((item_new >> cc) & 1u) {
-                    const float *k = A.qkvraw + (size_t)cc * c.qkv_rows + qd + (size_t)kvh * HD;
-                    const float *cs = c.rope_cs + (size_t)cc * HALF * 2;
-                    kx0[u] = __ldcg(k + jj); kx1[u] = __ldcg(k + jj + HALF); kco[u] = __ldcg(cs + 2 * jj); ksi[u] = __ldcg(cs + 2 * jj + 1);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < VPT; ++u) {
-                const int idx = tid + u * CONS_THREADS, cc = idx / HD, jj = idx - cc * HD;
-                vx[u] = ((item_new >> cc) & 1u) ? __ldcg(A.qkvraw + (size_t)cc * c.qkv_rows + qd + (size_t)(c.nkv + kvh) * HD + jj) : 0.f;
-            }
-#pragma unroll
-            for (int u = 0; u < KPT; ++u) {
-                nk0[u] = __float2bfloat16_rn(kx0[u] * kco[u] - kx1[u] * ksi[u]);
-                nk1[u] = __float2bfloat16_rn(kx1[u] * kco[u] + kx0[u] * ksi[u]);
-            }
-#pragma unroll
-            for (int u = 0; u < VPT; ++u) nv[u] = __float2bfloat16_rn(vx[u]);
-        }
-        bar_consumers();   // the previous item is done with the shared buffers
-        // ---- rotated, scaled queries -> A fragments (hi / lo)
-#pragma unroll
-        for (int u = 0; u < QPT; ++u) {
-            const int idx = tid + u * CONS_THREADS;
-            const int qcol = idx / HALF, jj = idx - qcol * HALF;
-            const float y0 = (qx0[u] * qco[u] - qx1[u] * qsi[u]) * scale, y1 = (qx1[u] * qco[u] + qx0[u] * qsi[u]) * scale;
-            const int row = qcol & 15, m = qcol >> 4;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int dim = jj + h * HALF;
-                const float y = h ? y1 : y0;
-                const int ks = dim >> 4, kk = dim & 15;
-                const int ln = (row & 7) * 4 + ((kk & 7) >> 1), reg = (row >> 3) + 2 * (kk >> 3);
-                const __nv_bfloat16 hi = __float2bfloat16_rn(y);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(y - __bfloat162float(hi));
-                __nv_bfloat16 *f = reinterpret_cast<__nv_bfloat16 *>(&as->qfrag[m][ks][ln][0]);
-                f[reg * 2 + (kk & 1)] = hi;
-                f[8 + reg * 2 + (kk & 1)] = lo;
-            }
+            for (int u = 0; u < QV; ++u) reinterpret_cast<uint4 *>(&as->qfrag[0][0][0][0])[tid + u * CONS_THREADS] = v[u];
         }
         bar_consumers();
         if (tid == 0) trace(S, EV_ATT, 2);   // queries ready
@@ -727,33 +705,11 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             for (int i = 0; i < 4; ++i) o[nt][i] = 0.f;
         for (int sb = 0; sb < nsb; ++sb) {
             const int p0 = p_base + sb * ATT_PAGE;
-            unsigned newm = 0;   // new rows inside this sub-block (uniform over the block)
-#pragma unroll
-            for (int cc = 0; cc < MAX_COLS; ++cc)
-                if (((item_new >> cc) & 1u) && d.pos[cc] >= p0 && d.pos[cc] < p0 + ATT_PAGE) newm |= 1u << cc;
-            const int page = c.page_table[p0 >> c.page_shift];
             float s[2][4];
             {   // ---- K block
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
-                unsigned char *kb = sm->x[slot];
-                if (newm) {
-                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + 0) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
-#pragma unroll
-                    for (int u = 0; u < KPT; ++u) {
-                        const int idx = tid + u * CONS_THREADS, cc = idx / HALF, jj = idx - cc * HALF;
-                        if ((newm >> cc) & 1u) {
-                            const int pos = d.pos[cc], t = pos - p0;
-                            const int e0 = t * HD + ((((jj >> 3) ^ (pos & 7)) << 3) | (jj & 7));
-                            const int e1 = t * HD + (((((jj + HALF) >> 3) ^ (pos & 7)) << 3) | (jj & 7));
-                            reinterpret_cast<__nv_bfloat16 *>(kb)[e0] = nk0[u];
-                            reinterpret_cast<__nv_bfloat16 *>(kb)[e1] = nk1[u];
-                            pool[blk + e0] = nk0[u];
-                            pool[blk + e1] = nk1[u];
-                        }
-                    }
-                    bar_consumers();
-                }
+                const unsigned char *kb = sm->x[slot];
                 float sh[2][4], sl[2][4];
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt)
@@ -822,21 +778,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             {   // ---- V block
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
-                unsigned char *vb = sm->x[slot];
-                if (newm) {
-                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + 1) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD);
-#pragma unroll
-                    for (int u = 0; u < VPT; ++u) {
-                        const int idx = tid + u * CONS_THREADS, cc = idx / HD, jj = idx - cc * HD;
-                        if ((newm >> cc) & 1u) {
-                            const int pos = d.pos[cc], t = pos - p0;
-                            const int e0 = t * HD + ((((jj >> 3) ^ (pos & 7)) << 3) | (jj & 7));
-                            reinterpret_cast<__nv_bfloat16 *>(vb)[e0] = nv[u];
-                            pool[blk + e0] = nv[u];
-                        }
-                    }
-                    bar_consumers();
-                }
+                const unsigned char *vb = sm->x[slot];
                 const int id = lane >> 3;
                 const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
                 const unsigned char *vrow = vb + pl * (HD * 2);
@@ -1072,29 +1014,90 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
         for (int l = 0; l < L; ++l) {
             const MegaLayer &ly = M.layer[l];
             const unsigned mask = active_mask(d, l);
-            // ---- QKV
+            // ---- QKV, finished in the epilogue: q rotated, scaled and stored as tensor-core fragments for the
+            // attention phase; k rotated, v as it is, both rounded to bf16 and written straight into their cache
+            // rows (Algorithm 1: "update KV cache at layer l by processing all tokens in P[l] in parallel").
+            // The rows of every q and k head come reordered so that a 16-row tile holds the features
+            // [8 t, 8 t + 8) and [hd/2 + 8 t, hd/2 + 8 t + 8): the two partners (i, i + hd/2) of a rotation
+            // are then rows r and r + 8 of one tile, which one thread holds for its two columns.
             {
                 Gemm g; g.W = ly.wqkv; g.X = reinterpret_cast<const uint4 *>(A.XA); g.N = c.qkv_rows; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_qkv; g.part = nullptr; g.phase_id = bar_no + 1; g.columns(mask);
                 x_ready();
                 const unsigned vseq = bar_no + 1;
                 if (ROLE == 2) {
-                    const int c0 = 2 * (lane & 3);
+                    constexpr int HALF = HD / 2, KSQ = HD / 16;
+                    const int c0 = 2 * (lane & 3), rq = lane >> 2;
+                    const int kvd = c.nkv * HD, group = c.group;
+                    const float qscale = rsqrtf((float)HD);
                     float r0 = 0.f, r1 = 0.f;
                     bool have_r = false;
-                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
-                        if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0]; r1 = sm->vec[c0 + 1]; have_r = true; }
+                    uint32_t *stash = stash_of(sm);
+                    __nv_bfloat16 *pool = reinterpret_cast<__nv_bfloat16 *>(c.kv_pool);
+                    gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile) {
+                        // rotary factors and cache pages of this lane's two columns, fetched while the weights stream
+                        const int n0 = tile * 16;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8, cc = c0 + (i & 1);
-                            if (n < c.qkv_rows && ((mask >> cc) & 1u)) A.qkvraw[(size_t)cc * c.qkv_rows + n] = acc[0][i] * ((i & 1) ? r1 : r0);
+                        for (int q = 0; q < 2; ++q) {
+                            const int cc = c0 + q;
+                            if (!((mask >> cc) & 1u)) continue;
+                            if (n0 < qd + kvd) {
+                                const float *cs = c.rope_cs + ((size_t)cc * HALF + ((n0 & (HD - 1)) >> 1) + rq) * 2;
+                                cp_async4(stash + (2 * q) * 32, cs);
+                                cp_async4(stash + (2 * q + 1) * 32, cs + 1);
+                            }
+                            if (n0 >= qd) cp_async4(stash + (4 + q) * 32, c.page_table + (d.pos[cc] >> c.page_shift));
+                        }
+                    }, [&](int tile, float (&acc)[1][4]) {
+                        if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0]; r1 = sm->vec[c0 + 1]; have_r = true; }
+                        cp_async_wait_all();
+                        const int n0 = tile * 16;
+                        if (n0 >= c.qkv_rows) return;
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const int cc = c0 + q;
+                            if (!((mask >> cc) & 1u)) continue;
+                            const float rs = q ? r1 : r0;
+                            const float x0 = acc[0][q] * rs, x1 = acc[0][2 + q] * rs;   // rows rq and rq + 8 of the tile
+                            if (n0 < qd + kvd) {
+                                const float co = __uint_as_float(stash[(2 * q) * 32]), si = __uint_as_float(stash[(2 * q + 1) * 32]);
+                                const int j = ((n0 & (HD - 1)) >> 1) + rq;   // feature j pairs with j + hd/2
+                                float y0 = x0 * co - x1 * si, y1 = x1 * co + x0 * si;
+                                if (n0 < qd) {
+                                    const int h = n0 / HD, kvh = div_group(h, group), qcol = cc * group + (h - kvh * group);
+                                    const int row = qcol & 15, m = qcol >> 4;
+                                    __nv_bfloat16 *f0 = reinterpret_cast<__nv_bfloat16 *>(A.qfrag + (((size_t)kvh * 2 + m) * KSQ) * 256);
+#pragma unroll
+                                    for (int hh = 0; hh < 2; ++hh) {
+                                        const int dim = j + hh * HALF;
+                                        const float y = (hh ? y1 : y0) * qscale;
+                                        const int ks = dim >> 4, kk = dim & 15;
+                                        const int ln = (row & 7) * 4 + ((kk & 7) >> 1), reg = (row >> 3) + 2 * (kk >> 3);
+                                        const __nv_bfloat16 hi = __float2bfloat16_rn(y);
+                                        const __nv_bfloat16 lo = __float2bfloat16_rn(y - __bfloat162float(hi));
+                                        __nv_bfloat16 *f = f0 + ((size_t)ks * 32 + ln) * 16;
+                                        f[reg * 2 + (kk & 1)] = hi;
+                                        f[8 + reg * 2 + (kk & 1)] = lo;
+                                    }
+                                } else {
+                                    const int kvh = (n0 - qd) / HD, pos = d.pos[cc], t = pos & (ATT_PAGE - 1);
+                                    const size_t blk = ((((size_t)stash[(4 + q) * 32] * c.L + l) * 2 + 0) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD) + (size_t)t * HD;
+                                    pool[blk + ((((j >> 3) ^ (pos & 7)) << 3) | (j & 7))] = __float2bfloat16_rn(y0);
+                                    pool[blk + (((((j + HALF) >> 3) ^ (pos & 7)) << 3) | (j & 7))] = __float2bfloat16_rn(y1);
+                                }
+                            } else {
+                                const int nv = n0 - qd - kvd, kvh = nv / HD, j = (nv & (HD - 1)) + rq, pos = d.pos[cc], t = pos & (ATT_PAGE - 1);
+                                const size_t blk = ((((size_t)stash[(4 + q) * 32] * c.L + l) * 2 + 1) * c.nkv + kvh) * ((size_t)ATT_PAGE * HD) + (size_t)t * HD;
+                                pool[blk + ((((j >> 3) ^ (pos & 7)) << 3) | (j & 7))] = __float2bfloat16_rn(x0);
+                                pool[blk + (((((j + 8) >> 3) ^ (pos & 7)) << 3) | (j & 7))] = __float2bfloat16_rn(x1);
+                            }
                         }
                     });
                 } else if (ROLE == 1) gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { rstd_produce(sm, A.ssq_a, ntd, d_model, c.eps, vseq); });
                 else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
                 phase_barrier(2);
             }
-            // ---- attention (the KV producer may run ahead: rows of this pass are patched in by the consumers)
-            if (ROLE == 1) attn_produce(A, S, d, l, r, pol);
+            // ---- attention (work items that hold no row of this pass are fetched before the QKV phase has ended)
+            if (ROLE == 1) attn_produce(A, S, d, l, mask, bar_no * (unsigned)G, r, pol);
             if (ROLE == 2) attn_consume<HD>(A, S, d, l, mask, r);
             phase_barrier(4);
             // ---- O projection + residual; prepares the FFN input
@@ -1140,7 +1143,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             }
             // ---- gate / up + SwiGLU
             {
-                Gemm g; g.W = ly.wgu; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff; g.ctas = n_gu;
+                Gemm g; g.W = ly.wgu; g.W2 = ly.wup; g.X = reinterpret_cast<const uint4 *>(A.XB); g.N = 2 * c.dff; g.K = d_model; g.pair = 2; g.half = c.dff; g.ctas = n_gu;
                 // the one GEMM of the layer where the unit-balanced split pays (measured: it shortens gate-up by 1.4 us,
                 // but lengthens down, QKV and O, whose tile groups are k-split among the warps)
                 g.part = A.part; g.phase_id = bar_no + 1; g.columns(mask);
@@ -1254,6 +1257,28 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     }
 }
 
+// Repack on load.  Destination row `prow` of the fused q | k | v matrix: v rows are copied as they are; inside
+// every q and k head the rows are reordered so that the 16-row tile t of the head holds the features
+// [8 t, 8 t + 8) in its rows 0..7 and [hd/2 + 8 t, hd/2 + 8 t + 8) in its rows 8..15.  The two partners
+// (i, i + hd/2) of a rotation then sit in rows r and r + 8 of one tensor-core tile, i.e. in one thread of the
+// QKV epilogue.  d must be a multiple of 8 and every pointer 16-byte aligned.
+__global__ void k_repack_qkv(const __nv_bfloat16 *__restrict__ wq, const __nv_bfloat16 *__restrict__ wk, const __nv_bfloat16 *__restrict__ wv,
+                             __nv_bfloat16 *__restrict__ dst, int nq, int nkv, int hd, int d) {
+    const int prow = blockIdx.x, qd = nq * hd, kvd = nkv * hd;
+    const __nv_bfloat16 *src;
+    if (prow < qd + kvd) {
+        const __nv_bfloat16 *w = prow < qd ? wq : wk;
+        const int rr = prow < qd ? prow : prow - qd;
+        const int h = rr / hd, pr = rr - h * hd, t = pr >> 4, r = pr & 15;
+        src = w + (size_t)(h * hd + t * 8 + (r & 7) + (r >> 3) * (hd / 2)) * d;
+    } else {
+        src = wv + (size_t)(prow - qd - kvd) * d;
+    }
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+    uint4 *d4 = reinterpret_cast<uint4 *>(dst + (size_t)prow * d);
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) d4[i] = s4[i];
+}
+
 // Arms the prompt passes of the persistent kernel for sequence 0 (KV cache <- LM(x), first line of Algorithm 1).
 __global__ void k_prefill_arm(Ctx c, int n_prompt) {
     DevState *st = c.st;
@@ -1275,7 +1300,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_decode_persistent(const __grid_c
     Smem *sm = smem_base(smem_raw);
     smem_init(sm);
     __syncthreads();
-    Shared S{sm, A.err, A.trace, 0};
+    Shared S{sm, A.err, A.trace, 0, A.wait_ns};
     const int warp = threadIdx.x >> 5;
     if (warp == CONS_WARPS) run<0, HD>(A, S);
     else if (warp == CONS_WARPS + 1) run<1, HD>(A, S);

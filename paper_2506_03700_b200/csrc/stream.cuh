@@ -32,8 +32,14 @@ constexpr int TILE_N = 16;                       // weight rows per stage (mma M
 constexpr int KG = KC / 64;                      // 64-element (128-byte) k groups per stage
 constexpr int W_STAGE = TILE_N * KC * 2;         // 16384: [k group][row][128 B, 16-byte chunks xor-swizzled by row%8]
 constexpr int X_STAGE = KSTEPS * 32 * 16;        // 16384: [column pair][k-step][8 slots][b0.hi b1.hi b0.lo b1.lo]
-constexpr int NW = 9;                            // weight stages in flight per CTA
-constexpr int NX = 3;                            // activation stages
+#ifndef ADA_NW
+#define ADA_NW 9
+#endif
+#ifndef ADA_NX
+#define ADA_NX 3
+#endif
+constexpr int NW = ADA_NW;                       // weight stages in flight per CTA
+constexpr int NX = ADA_NX;                       // activation / KV stages
 constexpr int CONS_WARPS = 8;
 constexpr int CONS_THREADS = CONS_WARPS * 32;
 constexpr int THREADS = CONS_THREADS + 64;       // + weight producer warp + activation producer warp
@@ -42,7 +48,7 @@ constexpr int RED_BYTES = CONS_WARPS * 2 * 128 * 4;  // cross-warp reduction scr
 constexpr int SCRATCH_BYTES = 33 * 1024;         // consumers' scratch: GEMM reduction, or the attention phase's buffers
 
 constexpr int ERR_TIMEOUT_MBAR = 1, ERR_TIMEOUT_GRID = 2;
-constexpr unsigned long long WAIT_NS = 2000000000ull;   // a single wait gives up after two seconds
+constexpr unsigned long long WAIT_NS_DEFAULT = 2000000000ull;   // a single wait gives up after two seconds unless told otherwise
 
 struct Smem {                                    // must start on a 1024-byte boundary (swizzle pattern)
     alignas(1024) unsigned char w[NW][W_STAGE];
@@ -159,6 +165,7 @@ struct Shared {            // what every role needs to wait safely
     int *err;              // global error word (0 = fine)
     Trace tr;
     int tr_on;             // this block is currently tracing
+    unsigned long long wait_ns;   // a single wait gives up after this many nanoseconds
 };
 
 constexpr int EV_PHASE_BEGIN = 1, EV_X0 = 2, EV_W0 = 3, EV_MAIN_END = 4, EV_EPI_END = 5, EV_WP_BEGIN = 6, EV_WP_END = 7,
@@ -196,7 +203,7 @@ __device__ __forceinline__ void mbar_wait(const Shared &S, unsigned long long *b
             if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
             unsigned long long t = gtime();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > WAIT_NS) { raise_error(S, ERR_TIMEOUT_MBAR); return; }
+            else if (t - t0 > S.wait_ns) { raise_error(S, ERR_TIMEOUT_MBAR); return; }
         }
     }
 }
@@ -229,7 +236,7 @@ __device__ __forceinline__ void vec_wait(const Shared &S, unsigned seq) {
             if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
             unsigned long long t = gtime();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > WAIT_NS) { raise_error(S, ERR_TIMEOUT_MBAR); return; }
+            else if (t - t0 > S.wait_ns) { raise_error(S, ERR_TIMEOUT_MBAR); return; }
         }
     }
 }
@@ -250,7 +257,7 @@ __device__ __forceinline__ void grid_wait(const Shared &S, const unsigned *ctr, 
             if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
             unsigned long long t = gtime();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > WAIT_NS) { raise_error(S, ERR_TIMEOUT_GRID); return; }
+            else if (t - t0 > S.wait_ns) { raise_error(S, ERR_TIMEOUT_GRID); return; }
         }
         __nanosleep(32);
     }
@@ -291,6 +298,7 @@ __host__ __device__ inline size_t xfrag_bytes(int K) { return (size_t)((K + KC -
 // is a stage.  Rows past N and k groups past K read as zeros.  K must be a multiple of 64.
 struct Gemm {
     const CUtensorMap *W;
+    const CUtensorMap *W2 = nullptr;   // pair == 2 only: map of the second matrix when the two are separate tensors (null: stacked in W)
     const uint4 *X;
     int N, K, pair, half;
     int ctas;   // CTAs 0 .. ctas-1 share the tiles (see balanced_ctas); 0 = the whole grid
@@ -412,7 +420,7 @@ __device__ __forceinline__ void gemm_produce_w(const Shared &S, const Gemm &g, i
         mbar_wait(S, &sm->w_empty[slot], ((r.wi / NW) & 1) ^ 1);
         if (lane == 0 && !aborted(S)) {
             mbar_expect_tx(&sm->w_full[slot], (uint32_t)W_STAGE);
-            tma_load_3d(sm->w[slot], g.W, 0, tile * TILE_N + p * g.half, kc * KG, &sm->w_full[slot], pol);
+            tma_load_3d(sm->w[slot], (p && g.W2) ? g.W2 : g.W, 0, tile * TILE_N + ((p && !g.W2) ? g.half : 0), kc * KG, &sm->w_full[slot], pol);
         }
         ++r.wi;
     };
@@ -648,7 +656,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                     bool stop = aborted(S) || *(volatile int *)S.err != 0;
                     const unsigned long long t = gtime();
                     if (t0 == 0) t0 = t;
-                    else if (t - t0 > WAIT_NS) { if (lane == 0) raise_error(S, ERR_TIMEOUT_GRID); stop = true; }
+                    else if (t - t0 > S.wait_ns) { if (lane == 0) raise_error(S, ERR_TIMEOUT_GRID); stop = true; }
                     if (__any_sync(0xffffffffu, stop)) { *(volatile int *)&S.sm->abort = 1; break; }
                 }
                 __nanosleep(64);
