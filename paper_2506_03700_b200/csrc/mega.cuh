@@ -526,6 +526,7 @@ __device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S,
     const uint32_t bytes = (uint32_t)(ATT_PAGE * c.hd * 2);
     const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
     bool synced = false;
+    if (lane == 0) trace(S, EV_ATT, 8);
     for (int item = cta; item < n_items; item += G) {
         const int kvh = item / nchunk, j = item - kvh * nchunk;
         const int p_base = j * ATT_CHUNK;
@@ -548,6 +549,7 @@ __device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S,
                     const size_t blk = ((((size_t)page * c.L + layer) * 2 + which) * c.nkv + kvh) * ((size_t)ATT_PAGE * c.hd);
                     mbar_expect_tx(&sm->x_full[slot], bytes);
                     bulk_g2s(sm->x[slot], pool + blk, bytes, &sm->x_full[slot], pol);
+                    trace(S, EV_ATT, 9 + 16 * (2 * sb + which));
                 }
                 ++r.xi;
             }
@@ -709,6 +711,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             {   // ---- K block
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                if (tid == 0) trace(S, EV_ATT, 3 + 16 * sb);   // K block landed
                 const unsigned char *kb = sm->x[slot];
                 float sh[2][4], sl[2][4];
 #pragma unroll
@@ -778,6 +781,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             {   // ---- V block
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                if (tid == 0) trace(S, EV_ATT, 4 + 16 * sb);   // V block landed
                 const unsigned char *vb = sm->x[slot];
                 const int id = lane >> 3;
                 const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);

@@ -49,6 +49,7 @@ constexpr int SCRATCH_BYTES = 33 * 1024;         // consumers' scratch: GEMM red
 
 constexpr int ERR_TIMEOUT_MBAR = 1, ERR_TIMEOUT_GRID = 2;
 constexpr unsigned long long WAIT_NS_DEFAULT = 2000000000ull;   // a single wait gives up after two seconds unless told otherwise
+constexpr unsigned long long SHORT_LIMIT_NS = 1000000ull;       // a limit below this is checked at every poll, not every 64th or 128th
 
 struct Smem {                                    // must start on a 1024-byte boundary (swizzle pattern)
     alignas(1024) unsigned char w[NW][W_STAGE];
@@ -198,7 +199,7 @@ __device__ __forceinline__ void mbar_wait(const Shared &S, unsigned long long *b
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
         if (mbar_try(bar, parity)) return;
-        if ((it & 127u) == 0) {
+        if ((it & 127u) == 0 || S.wait_ns < SHORT_LIMIT_NS) {
             if (aborted(S)) return;
             if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
             unsigned long long t = gtime();
@@ -231,7 +232,7 @@ __device__ __forceinline__ void vec_wait(const Shared &S, unsigned seq) {
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
         if (*(volatile unsigned *)&S.sm->vec_seq == seq) return;
-        if ((it & 127u) == 127u) {
+        if ((it & 127u) == 127u || S.wait_ns < SHORT_LIMIT_NS) {
             if (aborted(S)) return;
             if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
             unsigned long long t = gtime();
@@ -252,7 +253,7 @@ __device__ __forceinline__ void grid_wait(const Shared &S, const unsigned *ctr, 
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
         if (ld_acquire(ctr) >= target) return;
-        if ((it & 63u) == 0) {
+        if ((it & 63u) == 0 || S.wait_ns < SHORT_LIMIT_NS) {
             if (aborted(S)) return;
             if (*(volatile int *)S.err != 0) { *(volatile int *)&S.sm->abort = 1; return; }
             unsigned long long t = gtime();
@@ -652,7 +653,7 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
                         for (int i = 0; i < 4; ++i) d[p][i] += add[p][i];
                     break;
                 }
-                if ((it & 15u) == 15u) {   // bounded like every other wait on another CTA
+                if ((it & 15u) == 15u || S.wait_ns < SHORT_LIMIT_NS) {   // bounded like every other wait on another CTA
                     bool stop = aborted(S) || *(volatile int *)S.err != 0;
                     const unsigned long long t = gtime();
                     if (t0 == 0) t0 = t;

@@ -30,16 +30,11 @@ def medium(dtype, **kw):
 
 
 def tol(cfg, std):
-    """Logit tolerance: 1e-4 (fp32 models); 2e-2 x the logit std (bf16 models up to the 32 layers of the
-    8B shape).  With a bf16 cache the two sides round K and V from slightly different fp values, a few
-    elements per thousand land on the other side of a rounding boundary, and each such flip feeds a
-    5e-3 relative change into the next layer: the difference grows like sqrt(depth) (measured on the
-    13B shape: 7e-3, 9e-3, 1.4e-2, 1.7e-2, 2.2e-2 x std at 5, 10, 20, 30, 40 layers), whichever way the
-    GPU computes.  Deeper models therefore get 2e-2 x sqrt(L / 32) x 1.3."""
+    """The stated logit tolerance: 1e-4 (absolute and x std) for fp32 models, 2e-2 x the logit std for
+    bf16 models, whatever their depth."""
     if cfg.dtype == "fp32":
         return 1e-4 * min(1.0, std)
-    depth = max(1.0, (cfg.n_layers / 32.0) ** 0.5)
-    return 2e-2 * std * (depth * 1.3 if cfg.n_layers > 32 else 1.0)
+    return 2e-2 * std
 
 
 class Pair:
@@ -64,10 +59,12 @@ class Pair:
         return oracle.Session(self.om, max_seq)
 
 
-def check_against_oracle(pair, prompt, gpu_tokens, gpu_logits):
+def check_against_oracle(pair, prompt, gpu_tokens, gpu_logits, assert_logit_bound=True):
     """Teacher-forced comparison: the oracle recomputes, from scratch, the logits of the sequence
     the GPU produced; logits must agree within tolerance at every step and each GPU token must be
-    the oracle's argmax wherever the oracle's top-2 gap exceeds the tolerance."""
+    the oracle's argmax wherever the oracle's top-2 gap exceeds the tolerance.  Returns the worst
+    max|d| / tolerance over the steps (with assert_logit_bound=False the logit bound is measured
+    and returned, not asserted; the token rule is always asserted)."""
     cfg = pair.cfg
     seq = np.concatenate([prompt, gpu_tokens[:-1]])
     full = pair.om.full_logits(seq)
@@ -76,14 +73,65 @@ def check_against_oracle(pair, prompt, gpu_tokens, gpu_logits):
         ref = full[len(prompt) - 1 + i]
         t = tol(cfg, ref.std())
         err = np.abs(ref - gpu_logits[i].astype(np.float64)).max()
-        assert err <= t, (i, err, t)
+        if assert_logit_bound:
+            assert err <= t, (i, err, t)
         worst = max(worst, err / t)
+        slack = t if assert_logit_bound else max(t, err)
         top2 = np.sort(ref)[-2:]
-        if top2[1] - top2[0] > t:
+        if top2[1] - top2[0] > slack:
             assert int(tok) == int(np.argmax(ref)), i
         else:   # near tie: the GPU token must be one of the tied candidates
-            assert ref[int(tok)] >= top2[1] - 2 * t
+            assert ref[int(tok)] >= top2[1] - 2 * slack
     return worst
+
+
+def schedule_parity(pair, make_session, n, ptol, n_prompt=17, seeds=(5678, 5679, 5680), min_rows=4):
+    """Algorithm 1's decisions against the oracle's, over several prompts.  Where the two greedy
+    token streams agree to the end, every head evaluation (step, layer, token, probability) and
+    every counter is compared.  Where they part (possible only at a near-tie of the final logits,
+    which is asserted), the head evaluations are compared row by row up to the first that differs,
+    and at least `min_rows` must have agreed.  At least one prompt must give the full comparison,
+    so a run that compares nothing fails."""
+    cfg = pair.cfg
+    full = 0
+    for seed in seeds:
+        prompt = synth.make_prompt(cfg, n=n_prompt, seed=seed).numpy()
+        gamma = clear_gamma(pair, prompt, n, cfg.exit_layers, 5, 0.45, 2 * ptol)
+        assert gamma is not None
+        S = make_session()
+        S.capture_heads()
+        S.prefill(prompt)
+        st = binding.Stats()
+        out = S.adaptive_decode(n, gamma, cfg.exit_layers, 5, st)[0]
+        O = pair.cpu()
+        O.record_heads()
+        O.prefill(prompt)
+        ost = oracle.Stats()
+        ref = O.adaptive_decode(n, gamma, cfg.exit_layers, 5, stats=ost)
+        gh, oh = S.captured_heads(), O.heads
+        if np.array_equal(ref, out):
+            assert len(gh) == len(oh) and len(gh) >= min_rows
+            assert np.array_equal(gh[:, :3].astype(np.int64), oh[:, :3].astype(np.int64))
+            assert np.abs(gh[:, 3] - oh[:, 3]).max() <= ptol
+            for k in ("steps", "head_evals", "early_exits", "verify_steps", "accepted", "rejected", "discarded",
+                      "row_layers", "truncated"):
+                assert getattr(st, k) == getattr(ost, k), k
+            assert st.early_exits > 0
+            full += 1
+        else:
+            O2 = pair.cpu()
+            O2.record_logits(n + 4)
+            O2.prefill(prompt)
+            r2 = O2.plain_decode(n)
+            k = int(np.argmax(r2 != out))
+            z = np.sort(O2.logits[k])
+            assert z[-1] - z[-2] <= tol(cfg, O2.logits[k].std()), "the streams part where the oracle has no near-tie"
+            m = min(len(gh), len(oh))
+            same = np.all(gh[:m, :3].astype(np.int64) == oh[:m, :3].astype(np.int64), axis=1) & \
+                (np.abs(gh[:m, 3] - oh[:m, 3]) <= ptol)
+            agreed = m if same.all() else int(np.argmin(same))
+            assert agreed >= min_rows, (agreed, m)
+    assert full >= 1, "no prompt gave a full schedule comparison"
 
 
 def clear_gamma(pair, prompt, n, exits, cap, gamma0, tol, max_seq=256):
@@ -163,42 +211,10 @@ def test_adaptive_is_bit_exact_with_plain(dtype):
 @pytest.mark.parametrize("dtype,T_noise", [("fp32", None), ("bf16", None), ("fp32", 0.3)])
 def test_adaptive_schedule_and_heads_match_oracle(dtype, T_noise):
     """Same decisions as the oracle's Algorithm 1: per head evaluation the same step, layer and
-    token and the same probability within tolerance; identical counters.  (Decisions can differ
-    only where |p - gamma| is within rounding; such a case is skipped, not compared.)"""
+    token and the same probability within tolerance; identical counters (see schedule_parity)."""
     cfg = medium(dtype)
     pair = Pair(cfg, T_noise=T_noise)
-    prompt = synth.make_prompt(cfg, n=17).numpy()
-    n = 40
-    ptol = 1e-4 if dtype == "fp32" else 3e-3
-    gamma = clear_gamma(pair, prompt, n, cfg.exit_layers, 5, 0.45, 2 * ptol)
-    assert gamma is not None
-    S = pair.gpu()
-    S.capture_heads()
-    S.prefill(prompt)
-    st = binding.Stats()
-    out = S.adaptive_decode(n, gamma, cfg.exit_layers, 5, st)[0]
-    O = pair.cpu()
-    O.record_heads()
-    O.prefill(prompt)
-    ost = oracle.Stats()
-    ref = O.adaptive_decode(n, gamma, cfg.exit_layers, 5, stats=ost)
-    gh, oh = S.captured_heads(), O.heads
-    if np.array_equal(ref, out):
-        assert len(gh) == len(oh)
-        assert np.array_equal(gh[:, :3].astype(np.int64), oh[:, :3].astype(np.int64))
-        assert np.abs(gh[:, 3] - oh[:, 3]).max() <= ptol
-        for k in ("steps", "head_evals", "early_exits", "verify_steps", "accepted", "rejected", "discarded",
-                  "row_layers", "truncated"):
-            assert getattr(st, k) == getattr(ost, k), k
-        assert st.early_exits > 0
-    else:   # the two greedy runs part at a near-tie of the final logits: nothing to compare beyond it
-        O2 = pair.cpu()
-        O2.record_logits(n + 4)
-        O2.prefill(prompt)
-        r2 = O2.plain_decode(n)
-        k = int(np.argmax(r2 != out))
-        z = np.sort(O2.logits[k])
-        assert z[-1] - z[-2] <= tol(cfg, O2.logits[k].std())
+    schedule_parity(pair, pair.gpu, 40, 1e-4 if dtype == "fp32" else 3e-3)
 
 
 def test_forced_tapes_never_change_the_output():
@@ -258,15 +274,21 @@ def test_chained_and_mixed_calls():
     pair = Pair(cfg)
     prompt = synth.make_prompt(cfg, n=8).numpy()
     P = pair.gpu()
+    P.capture_logits(40)
     P.prefill(prompt)
     ref = P.plain_decode(36)[0]
+    ref_lg = P.captured_logits()[:36].clone()
     S = pair.gpu()
+    S.capture_logits(40)
     S.prefill(prompt)
     a = S.adaptive_decode(1, 0.0, cfg.exit_layers, 5)[0]
     b = S.adaptive_decode(9, 0.0, cfg.exit_layers, 5)[0]
     c = S.plain_decode(6)[0]
     d = S.adaptive_decode(20, 0.3, cfg.exit_layers[:1], 2)[0]
     assert np.array_equal(np.concatenate([a, b, c, d]), ref)
+    # one captured logits row per returned token, also across calls that ended by dropping a verified token
+    lg = S.captured_logits()
+    assert len(lg) == 36 and torch.equal(lg, ref_lg)
     # a new prefill on the same session starts over
     S.prefill(prompt)
     assert np.array_equal(S.plain_decode(5)[0], ref[:5])
@@ -345,10 +367,10 @@ def test_errors_are_codes_not_faults():
     assert len(S.plain_decode(3)[0]) == 3
 
 
-@pytest.mark.parametrize("name,n_prompt,n_gen", [("tiny", 16, 128), ("1b", 24, 6)])
+@pytest.mark.parametrize("name,n_prompt,n_gen", [("tiny", 16, 128), ("1b", 512, 16)])
 def test_named_configurations_sampled(name, n_prompt, n_gen):
-    """The benchmark's own shapes: the tiny fp32 configuration in full, the 1B shape on a short
-    prompt (outputs the oracle can compute one by one)."""
+    """The benchmark's own shapes: the tiny fp32 configuration in full, the 1B shape on its own
+    512-token prompt and 16 tokens (outputs the oracle can compute one by one)."""
     cfg = synth.CONFIGS[name]
     pair = Pair(cfg, jitter=0.0)
     prompt = synth.make_prompt(cfg, n=n_prompt).numpy()
@@ -361,3 +383,96 @@ def test_named_configurations_sampled(name, n_prompt, n_gen):
     A.prefill(prompt)
     st = binding.Stats()
     assert np.array_equal(A.adaptive_decode(n_gen, cfg.threshold, cfg.exit_layers, 5, st)[0], out)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_end_of_sequence_token_stops_decoding(dtype):
+    """Algorithm 1 runs "while t_i != [EOS]": decoding ends at the first VERIFIED end-of-sequence token.
+    Plain and adaptive decoding (every forced tape, planted early exits included) return the same
+    tokens, the same count and leave the same state; the oracle with the same token agrees."""
+    cfg = small(dtype)
+    pair = Pair(cfg)
+    prompt = synth.make_prompt(cfg, n=9).numpy()
+    n = 30
+    P = pair.gpu()
+    P.prefill(prompt)
+    ref = P.plain_decode(n)[0]
+    i = next(k for k in range(4, n) if ref[k] not in ref[:k])
+    eos = int(ref[i])
+    Q = pair.gpu()
+    Q.prefill(prompt)
+    st = binding.Stats()
+    want = Q.plain_decode(n, st, eos_id=eos)[0]
+    assert st.emitted[0] == i + 1 and st.finished == 1
+    assert np.array_equal(want[:i + 1], ref[:i + 1]) and (want[i + 1:] == eos).all()
+    lq, fq = Q.state()
+    assert lq == len(prompt) + i + 1 and (fq == len(prompt) + i).all()
+    with pytest.raises(binding.AdaError) as e:      # the only sequence has ended
+        Q.plain_decode(4, eos_id=eos)
+    assert e.value.code == -2
+    O = pair.cpu()
+    O.prefill(prompt)
+    oref = O.plain_decode(n, eos_id=eos)
+    if dtype == "fp32":                             # at 1e-4 the two greedy streams are the same stream
+        assert O.emitted == i + 1 and np.array_equal(oref, want)
+    elif np.array_equal(oref[:O.emitted], ref[:O.emitted]):
+        assert O.emitted == i + 1
+    rng = np.random.default_rng(3)
+    for trial in range(8):
+        S = pair.gpu()
+        S.prefill(prompt)
+        S.set_exit_tape(rng.integers(0, 2, 64))
+        st = binding.Stats()
+        out = S.adaptive_decode(n, 0.5, cfg.exit_layers, int(rng.integers(1, 6)), st, eos_id=eos)[0]
+        assert np.array_equal(out, want), trial
+        assert st.emitted[0] == i + 1 and st.finished == 1
+        ls, fs = S.state()
+        assert ls == lq and np.array_equal(fs, fq)
+    # chained: the stop falls into the second call; a token that never occurs changes nothing
+    S = pair.gpu()
+    S.prefill(prompt)
+    st = binding.Stats()
+    a = S.adaptive_decode(3, 0.0, cfg.exit_layers, 5, st, eos_id=eos)[0]
+    b = S.adaptive_decode(n, 0.0, cfg.exit_layers, 5, st, eos_id=eos)[0]
+    assert st.emitted[0] == i + 1 and np.array_equal(np.concatenate([a, b[:i + 1 - 3]]), ref[:i + 1])
+    unused = next(t for t in range(cfg.vocab) if t not in ref)
+    S = pair.gpu()
+    S.prefill(prompt)
+    assert np.array_equal(S.adaptive_decode(n, 0.3, cfg.exit_layers, 5, eos_id=unused)[0], ref)
+
+
+def split_weights(cfg, w):
+    """The same model with q, k, v and gate, up as separately allocated tensors."""
+    nq, nkv, ff = cfg.n_q_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim, cfg.d_ff
+    out = {}
+    for k, v in w.items():
+        if k.endswith(".wqkv"):
+            p = k[:-4]
+            out[p + "wq"], out[p + "wk"], out[p + "wv"] = v[:nq].clone(), v[nq:nq + nkv].clone(), v[nq + nkv:].clone()
+        elif k.endswith(".w_gate_up"):
+            p = k[:-9]
+            out[p + "w_gate"], out[p + "w_up"] = v[:ff].clone(), v[ff:].clone()
+        else:
+            out[k] = v
+    return out
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_separate_q_k_v_gate_up_tensors_give_the_same_bits(dtype):
+    cfg = medium(dtype)
+    pair = Pair(cfg)
+    gm2 = binding.Model(cfg, split_weights(cfg, pair.w))
+    for l in cfg.exit_layers:
+        gm2.set_exit_head(l, None, cfg.logit_scale)
+    prompt = synth.make_prompt(cfg, n=19).numpy()
+    n = 24
+    outs = []
+    for gm in (pair.gm, gm2):
+        S = binding.Session(gm, 1, 256, 16, 5)
+        S.capture_logits(n + 4)
+        S.prefill(prompt)
+        st = binding.Stats()
+        t = S.adaptive_decode(n, 0.3, cfg.exit_layers, 5, st)[0]
+        assert st.path == 0
+        outs.append((t, S.captured_logits()[:n].clone()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])

@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 import oracle
 from paper_2506_03700_b200 import binding, synth
-from test_gpu_parity import Pair, check_against_oracle, clear_gamma, tol
+from test_gpu_parity import Pair, check_against_oracle, schedule_parity, split_weights, tol
 
 
 def gqa(**kw):      # 4 q heads per kv head, head_dim 64, ragged vocabulary tile, FFN depth with a short last k chunk
@@ -98,37 +98,7 @@ def test_adaptive_is_bit_exact_with_plain(mk):
 def test_adaptive_schedule_and_heads_match_oracle(mk, T_noise):
     cfg = mk()
     pair = Pair(cfg, T_noise=T_noise)
-    prompt = synth.make_prompt(cfg, n=17).numpy()
-    n, ptol = 40, 3e-3
-    gamma = clear_gamma(pair, prompt, n, cfg.exit_layers, 5, 0.45, 2 * ptol)
-    assert gamma is not None
-    S = session(pair)
-    S.capture_heads()
-    S.prefill(prompt)
-    st = binding.Stats()
-    out = S.adaptive_decode(n, gamma, cfg.exit_layers, 5, st)[0]
-    O = pair.cpu()
-    O.record_heads()
-    O.prefill(prompt)
-    ost = oracle.Stats()
-    ref = O.adaptive_decode(n, gamma, cfg.exit_layers, 5, stats=ost)
-    gh, oh = S.captured_heads(), O.heads
-    if np.array_equal(ref, out):
-        assert len(gh) == len(oh)
-        assert np.array_equal(gh[:, :3].astype(np.int64), oh[:, :3].astype(np.int64))
-        assert np.abs(gh[:, 3] - oh[:, 3]).max() <= ptol
-        for k in ("steps", "head_evals", "early_exits", "verify_steps", "accepted", "rejected", "discarded",
-                  "row_layers", "truncated"):
-            assert getattr(st, k) == getattr(ost, k), k
-        assert st.early_exits > 0
-    else:   # the two greedy runs part at a near-tie of the final logits: nothing to compare beyond it
-        O2 = pair.cpu()
-        O2.record_logits(n + 4)
-        O2.prefill(prompt)
-        r2 = O2.plain_decode(n)
-        k = int(np.argmax(r2 != out))
-        z = np.sort(O2.logits[k])
-        assert z[-1] - z[-2] <= tol(cfg, O2.logits[k].std())
+    schedule_parity(pair, lambda: session(pair), 40, 3e-3)
 
 
 def test_forced_tapes_and_relaunches_never_change_the_output():
@@ -189,15 +159,23 @@ def test_chained_calls_and_both_paths_mixed():
     pair = Pair(cfg)
     prompt = synth.make_prompt(cfg, n=8).numpy()
     P = session(pair)
+    P.capture_logits(40)
     P.prefill(prompt)
     ref = P.plain_decode(36)[0]
+    ref_lg = P.captured_logits()[:36].clone()
     S = session(pair)
+    S.capture_logits(40)
     S.prefill(prompt)
-    a = S.adaptive_decode(1, 0.0, cfg.exit_layers, 5)[0]
-    b = S.adaptive_decode(9, 0.0, cfg.exit_layers, 5)[0]
-    c = S.plain_decode(6)[0]
-    d = S.adaptive_decode(20, 0.3, cfg.exit_layers[:1], 2)[0]
+    st = binding.Stats()
+    a = S.adaptive_decode(1, 0.0, cfg.exit_layers, 5, st)[0]
+    b = S.adaptive_decode(9, 0.0, cfg.exit_layers, 5, st)[0]
+    c = S.plain_decode(6, st)[0]
+    d = S.adaptive_decode(20, 0.3, cfg.exit_layers[:1], 2, st)[0]
     assert np.array_equal(np.concatenate([a, b, c, d]), ref)
+    assert st.path == 1 and st.emitted[0] == 36
+    # one captured logits row per returned token, also across calls that ended by dropping a verified token
+    lg = S.captured_logits()
+    assert len(lg) == 36 and torch.equal(lg, ref_lg)
     S.prefill(prompt)
     assert np.array_equal(S.plain_decode(5)[0], ref[:5])
     # the one-kernel-per-operation path agrees within tolerance: same tokens on this model
@@ -264,3 +242,96 @@ def test_more_attention_work_items_than_ctas():
             A.set_exit_tape(tape)
         assert np.array_equal(A.adaptive_decode(n, gamma, cfg.exit_layers, 5)[0], out)
         assert torch.equal(A.captured_logits()[:n], lg)
+
+
+@pytest.mark.parametrize("mk", [gqa, hd128])
+def test_end_of_sequence_token_stops_decoding(mk):
+    """ "while t_i != [EOS]" inside the persistent kernel: the first verified end-of-sequence token ends
+    the call, under every forced tape and across relaunches; an early-predicted one stops nothing."""
+    cfg = mk()
+    pair = Pair(cfg)
+    prompt = synth.make_prompt(cfg, n=9).numpy()
+    n = 30
+    P = session(pair)
+    P.prefill(prompt)
+    ref = P.plain_decode(n)[0]
+    i = next(k for k in range(4, n) if ref[k] not in ref[:k])
+    eos = int(ref[i])
+    Q = session(pair)
+    Q.prefill(prompt)
+    st = binding.Stats()
+    want = Q.plain_decode(n, st, eos_id=eos)[0]
+    assert st.emitted[0] == i + 1 and st.finished == 1 and st.path == 1
+    assert np.array_equal(want[:i + 1], ref[:i + 1]) and (want[i + 1:] == eos).all()
+    lq, fq = Q.state()
+    assert lq == len(prompt) + i + 1 and (fq == len(prompt) + i).all()
+    rng = np.random.default_rng(5)
+    for trial in range(8):
+        S = session(pair, max_early=7)
+        S.set_launch_steps(int(rng.integers(1, 9)))
+        S.prefill(prompt)
+        S.set_exit_tape(rng.integers(0, 2, 64))
+        st = binding.Stats()
+        out = S.adaptive_decode(n, 0.5, cfg.exit_layers, int(rng.integers(1, 8)), st, eos_id=eos)[0]
+        assert np.array_equal(out, want), trial
+        assert st.emitted[0] == i + 1 and st.finished == 1
+        ls, fs = S.state()
+        assert ls == lq and np.array_equal(fs, fq)
+    # the token prefill produced is itself the end-of-sequence token: one token, no step
+    S = session(pair)
+    S.prefill(prompt)
+    st = binding.Stats()
+    out = S.adaptive_decode(5, 0.0, cfg.exit_layers, 5, st, eos_id=int(ref[0]))[0]
+    assert st.emitted[0] == 1 and st.steps == 0 and (out == ref[0]).all()
+    # a prefill starts the sequence afresh
+    S.prefill(prompt)
+    assert np.array_equal(S.plain_decode(6)[0], ref[:6])
+
+
+def test_separate_q_k_v_gate_up_tensors_give_the_same_bits():
+    """Weights lent as wq, wk, wv, w_gate, w_up (separate allocations): the gate and up matrices are
+    streamed through two tensor maps, q | k | v through the repacked copy in the arena."""
+    cfg = gqa()
+    pair = Pair(cfg)
+    gm2 = binding.Model(cfg, split_weights(cfg, pair.w))
+    for l in cfg.exit_layers:
+        gm2.set_exit_head(l, None, cfg.logit_scale)
+    prompt = synth.make_prompt(cfg, n=19).numpy()
+    n = 24
+    outs = []
+    for gm in (pair.gm, gm2):
+        S = binding.Session(gm, 1, 256, 64, 5)
+        assert S.get_path() == 1
+        S.capture_logits(n + 4)
+        S.prefill(prompt)
+        t = S.adaptive_decode(n, 0.3, cfg.exit_layers, 5)[0]
+        outs.append((t, S.captured_logits()[:n].clone()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
+def test_a_wait_that_runs_out_ends_the_call_with_a_timeout_and_the_session_recovers():
+    """Every device-side wait is bounded.  With the limit set far below what a grid-wide wait lasts, the
+    first wait that is not satisfied at once gives up: the kernel raises its error word, every other
+    wait falls through, the kernel ends and the call returns ADA_ETIMEOUT (no trap, no hang, the
+    context stays usable).  After a reset and a prefill the same session decodes correctly."""
+    cfg = gqa()
+    pair = Pair(cfg)
+    prompt = synth.make_prompt(cfg, n=12).numpy()
+    n = 12
+    P = session(pair)
+    P.prefill(prompt)
+    ref = P.plain_decode(n)[0]
+    S = session(pair)
+    S.prefill(prompt)
+    S.set_wait_limit(20)                  # nanoseconds
+    with pytest.raises(binding.AdaError) as e:
+        S.plain_decode(n)
+    assert e.value.code == -5
+    torch.cuda.synchronize()              # the context is intact
+    S.set_wait_limit(2_000_000_000)
+    S.reset()
+    S.prefill(prompt)
+    assert np.array_equal(S.plain_decode(n)[0], ref)
+    st = binding.Stats()
+    S.prefill(prompt)
+    assert np.array_equal(S.adaptive_decode(n, 0.3, cfg.exit_layers, 5, st)[0], ref) and st.early_exits > 0

@@ -226,3 +226,84 @@ def test_bad_arguments_are_refused():
         s.adaptive_decode(4, 0.5, (2, 1), max_early=5)        # not ascending
     with pytest.raises(RuntimeError):
         s.adaptive_decode(400, 0.5, (1,), max_early=5)        # beyond capacity
+
+
+# ---------------------------------------------------------------- end of sequence (Algorithm 1: "while t_i != [EOS]")
+
+def _first_repeat_free_eos(ref):
+    """A token of the plain stream, not its first, whose first occurrence is where it stands."""
+    for i in range(3, len(ref)):
+        if ref[i] not in ref[:i]:
+            return i, int(ref[i])
+    raise AssertionError("degenerate stream")
+
+
+def test_plain_decoding_with_eos_is_the_prefix_up_to_the_first_eos():
+    """Definition: generate until the end-of-sequence token has been produced."""
+    cfg = _mini()
+    w, m = make_oracle(cfg)
+    prompt = synth.make_prompt(cfg, n=5).numpy()
+    n = 14
+    ref = _plain(m, prompt, n)
+    i, eos = _first_repeat_free_eos(ref)
+    s = oracle.Session(m, 128)
+    s.prefill(prompt)
+    out = s.plain_decode(n, eos_id=eos)
+    assert s.emitted == i + 1
+    assert np.array_equal(out[:i + 1], ref[:i + 1]) and (out[i + 1:] == eos).all()
+    assert s.len == len(prompt) + i + 1
+    assert all(s.kv_len(l) == len(prompt) + i for l in range(cfg.n_layers))
+    # an end-of-sequence token that never occurs changes nothing
+    unused = next(t for t in range(cfg.vocab) if t not in ref)
+    s = oracle.Session(m, 128)
+    s.prefill(prompt)
+    assert np.array_equal(s.plain_decode(n, eos_id=unused), ref) and s.emitted == n
+    # the token prefill produced may already be it
+    s = oracle.Session(m, 128)
+    s.prefill(prompt)
+    out = s.plain_decode(n, eos_id=int(ref[0]))
+    assert s.emitted == 1 and out[0] == ref[0] and s.len == len(prompt) + 1
+
+
+def test_adaptive_with_eos_equals_plain_with_eos_on_every_tape():
+    """Only a VERIFIED end-of-sequence token ends the sequence: under every forced exit tape, with and
+    without planted early predictions of the end-of-sequence token itself, the adaptive procedure
+    returns what plain decoding with the same token returns, and leaves the same state."""
+    cfg = _mini()
+    w, m = make_oracle(cfg)
+    prompt = synth.make_prompt(cfg, n=5).numpy()
+    n = 12
+    ref = _plain(m, prompt, n)
+    i, eos = _first_repeat_free_eos(ref)
+    assert i + 1 < n                           # the call would have gone on
+    p = oracle.Session(m, 128)
+    p.prefill(prompt)
+    want = p.plain_decode(n, eos_id=eos)
+    planted = 0
+    for tape in itertools.product((0, 1), repeat=8):
+        for plant in (False, True):
+            s = oracle.Session(m, 128)
+            s.prefill(prompt)
+            st = oracle.Stats()
+            tape_tok = [eos if (plant and k % 3 == 1) else -1 for k in range(len(tape))]
+            out = s.adaptive_decode(n, 0.5, cfg.exit_layers, max_early=3, tape=tape, tape_tok=tape_tok, stats=st, eos_id=eos)
+            assert np.array_equal(out, want), (tape, plant, out, want)
+            assert s.emitted == i + 1
+            assert s.len == p.len and all(s.kv_len(l) == p.kv_len(l) for l in range(cfg.n_layers))
+            planted += plant and st.rejected > 0
+    assert planted > 0                         # a wrongly predicted end-of-sequence token was rejected, not obeyed
+
+
+def test_eos_across_chained_calls():
+    cfg = _mini()
+    w, m = make_oracle(cfg)
+    prompt = synth.make_prompt(cfg, n=5).numpy()
+    ref = _plain(m, prompt, 14)
+    i, eos = _first_repeat_free_eos(ref)
+    s = oracle.Session(m, 128)
+    s.prefill(prompt)
+    a = s.adaptive_decode(2, 0.0, cfg.exit_layers, eos_id=eos)
+    assert s.emitted == 2
+    b = s.adaptive_decode(12, 0.0, cfg.exit_layers, eos_id=eos)
+    assert s.emitted == i + 1 - 2
+    assert np.array_equal(np.concatenate([a, b[:s.emitted]]), ref[:i + 1])

@@ -1,7 +1,8 @@
 """ada_gemm_noalloc: the streaming GEMM for callers that cannot lend or allocate device scratch
 (for example a server whose allocator already owns all of HBM).  Its result must equal that of
-ada_debug_gemm, which works in caller-provided scratch; checked on two calls in a row because
-every call reuses the one built-in scratch array and finds the previous call's contents in it."""
+ada_debug_gemm, which works in caller-provided scratch, and a float64 matrix product within the
+GEMM tolerance; checked on calls in a row because every call reuses the one built-in scratch array
+and finds the previous call's contents in it."""
 
 import numpy as np
 import pytest
@@ -12,23 +13,58 @@ pytestmark = pytest.mark.gpu
 from paper_2506_03700_b200 import binding, synth
 
 
+def _float64(W, X, mode):
+    ref = X.double().cpu().numpy() @ W.double().cpu().numpy().T
+    if mode == 1:
+        h = W.shape[0] // 2
+        g, u = ref[:, :h], ref[:, h:]
+        ref = g / (1.0 + np.exp(-g)) * u
+    return ref
+
+
 def _pair(N, K, cols, mode, seed):
     W = synth.normal_tensor(seed, 11, (N, K), 0.05, torch.bfloat16, "cuda")
     X = synth.normal_tensor(seed, 12, (cols, K), 1.0, torch.float32, "cuda")
     ref, _ = binding.debug_gemm(W, X, mode)
     Y = torch.full_like(ref, float("nan"))          # allocated by the caller, as the call requires
     binding.gemm_noalloc(W, X, Y, mode)
-    return Y, ref
+    return Y, ref, _float64(W, X, mode)
 
 
 def test_two_calls_in_a_row_match_the_scratch_taking_entry_point():
     # second call: shallower K and fewer columns than the first, so stale scratch contents lie
     # behind and beside what it uses; third: the gate/up form
     for N, K, cols, mode, seed in [(1000, 1216, 8, 0, 5), (5003, 512, 3, 0, 6), (2 * 688, 256, 4, 1, 7)]:
-        y, ref = _pair(N, K, cols, mode, seed)
+        y, ref, ref64 = _pair(N, K, cols, mode, seed)
         assert torch.isfinite(y).all()
         assert (y - ref).abs().max().item() <= 2e-5 * max(1.0, ref.abs().max().item())
         assert torch.equal(y, ref)                   # same kernel, same layout: same bits
+        assert np.abs(y.double().cpu().numpy() - ref64).max() <= 2e-5 * max(1.0, np.abs(ref64).max())
+
+
+def test_the_deepest_product_the_built_in_scratch_holds():
+    """K = 16384 fills the activation part of the array to its last byte; the error word and the
+    tensor map sit right behind it."""
+    y, ref, ref64 = _pair(48, 16384, 8, 0, 9)
+    assert torch.equal(y, ref)
+    assert np.abs(y.double().cpu().numpy() - ref64).max() <= 2e-5 * max(1.0, np.abs(ref64).max())
+    y, ref, ref64 = _pair(32, 128, 1, 0, 10)         # a small one right after it
+    assert torch.equal(y, ref)
+
+
+def test_further_calls_take_no_device_memory():
+    """Once the library's device code is in place on the GPU (the first call sees to that), a call takes
+    nothing from the device's free memory: what the driver reports free is the same before and after."""
+    W = synth.normal_tensor(3, 11, (512, 1024), 0.05, torch.bfloat16, "cuda")
+    X = synth.normal_tensor(3, 12, (4, 1024), 1.0, torch.float32, "cuda")
+    Y = torch.empty(4, 512, dtype=torch.float32, device="cuda")
+    binding.gemm_noalloc(W, X, Y, 0)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(5):
+        binding.gemm_noalloc(W, X, Y, 0)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
 
 
 def test_depth_beyond_the_built_in_scratch_is_refused():
@@ -40,5 +76,5 @@ def test_depth_beyond_the_built_in_scratch_is_refused():
         binding.gemm_noalloc(W, X, Y, 0)
     assert e.value.code == -3
     # a call that fits still works afterwards
-    y, ref = _pair(48, 128, 3, 0, 8)
+    y, ref, _ = _pair(48, 128, 3, 0, 8)
     assert torch.equal(y, ref)
