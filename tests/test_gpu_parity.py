@@ -37,6 +37,13 @@ def tol(cfg, std):
     return 2e-2 * std
 
 
+# Tolerance on a head probability p = max softmax(z) of a bf16 model.  A logit error of e x std(z) moves p by at
+# most p (1 - p) * 2 e std(z) <= e std(z) / 2.  The intermediate heads of the test models scale their logits by 8
+# (std(z) about 5) and the logit error observed on them is about 3e-3 x std: 1e-2 on p.  (The stated logit bound
+# of 2e-2 x std would allow 5e-2.)
+PTOL_BF16 = 1e-2
+
+
 class Pair:
     """The same synthetic model on both sides."""
 
@@ -214,7 +221,7 @@ def test_adaptive_schedule_and_heads_match_oracle(dtype, T_noise):
     token and the same probability within tolerance; identical counters (see schedule_parity)."""
     cfg = medium(dtype)
     pair = Pair(cfg, T_noise=T_noise)
-    schedule_parity(pair, pair.gpu, 40, 1e-4 if dtype == "fp32" else 3e-3)
+    schedule_parity(pair, pair.gpu, 40, 1e-4 if dtype == "fp32" else PTOL_BF16)
 
 
 def test_forced_tapes_never_change_the_output():

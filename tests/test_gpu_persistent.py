@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 import oracle
 from paper_2506_03700_b200 import binding, synth
-from test_gpu_parity import Pair, check_against_oracle, schedule_parity, split_weights, tol
+from test_gpu_parity import PTOL_BF16, Pair, check_against_oracle, schedule_parity, split_weights, tol
 
 
 def gqa(**kw):      # 4 q heads per kv head, head_dim 64, ragged vocabulary tile, FFN depth with a short last k chunk
@@ -98,7 +98,7 @@ def test_adaptive_is_bit_exact_with_plain(mk):
 def test_adaptive_schedule_and_heads_match_oracle(mk, T_noise):
     cfg = mk()
     pair = Pair(cfg, T_noise=T_noise)
-    schedule_parity(pair, lambda: session(pair), 40, 3e-3)
+    schedule_parity(pair, lambda: session(pair), 40, PTOL_BF16)
 
 
 def test_forced_tapes_and_relaunches_never_change_the_output():
