@@ -140,7 +140,7 @@ void ada_session_destroy(ada_session *s);
 int ada_session_reset(ada_session *s, int32_t seq);
 
 /* KV cache <- LM(x) (first line of Algorithm 1): runs the n_prompt tokens of sequence `seq`
- * through all layers.  The first generated token (full-depth argmax at the last prompt token)
+ * through all layers (prompts of 32 tokens or more in dense blocks of 128 positions, see ada_debug_set_prefill).  The first generated token (full-depth argmax at the last prompt token)
  * becomes the sequence's pending token.  ADA_ECAPACITY if pages or max_seq_len do not suffice. */
 int ada_prefill(ada_session *s, int32_t seq, const int32_t *prompt_host, int32_t n_prompt);
 
@@ -196,6 +196,12 @@ int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out
  * ada_stats.path reports the path a decode call ran on. */
 int ada_debug_set_path(ada_session *s, int32_t path);
 int ada_debug_get_path(ada_session *s, int32_t *path_out);
+/* How ada_prefill runs prompts of 32 tokens or more.  1 (the default wherever it is available: bf16 models of
+ * the shapes the persistent kernel takes, on sm_100): the dense pass, blocks of 128 positions, every weight
+ * matrix streamed once per block through a tcgen05 GEMM with its accumulator in tensor memory.  0: through
+ * the decode path itself (passes of eight positions in the persistent kernel, or one kernel per operation).
+ * ADA_EUNSUPPORTED if the dense pass is asked of a session that cannot run it. */
+int ada_debug_set_prefill(ada_session *s, int32_t dense);
 /* Steps of Algorithm 1 one launch of the persistent kernel may start before it returns to the host
  * (default 256; the host relaunches until the call is complete). */
 int ada_debug_set_launch_steps(ada_session *s, int32_t steps);
@@ -239,6 +245,16 @@ size_t ada_debug_gemm_work_bytes(int32_t K);
 int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const float *X_dev, int32_t cols,
                    void *work_dev, size_t work_bytes, float *Y_dev, int32_t ldy, int32_t repeat, void *cuda_stream,
                    float *ms_out);
+
+/* Run the dense GEMM of the prompt pass by itself (Algorithm 1, first line: all prompt tokens go through the
+ * model at once): Y[m][n] = (or +=, if `accumulate`) sum_k X[m][k] W[n][k] for up to 128 rows m, on tcgen05
+ * tensor cores with the accumulator in tensor memory.  W_dev bf16 [N, K] row-major, X_dev fp32 [rows, K],
+ * Y_dev fp32 [rows, ldy] (16-byte aligned, ldy a multiple of 4), K a multiple of 64; work_dev: device scratch
+ * of ada_debug_dense_gemm_work_bytes(K) bytes, 256-byte aligned.  sm_100 only (ADA_EUNSUPPORTED elsewhere).
+ * Synchronises the stream; ADA_ETIMEOUT if a bounded device-side wait expired. */
+size_t ada_debug_dense_gemm_work_bytes(int32_t K);
+int ada_debug_dense_gemm(const void *W_dev, int32_t N, int32_t K, const float *X_dev, int32_t rows, float *Y_dev, int32_t ldy,
+                         int32_t accumulate, void *work_dev, size_t work_bytes, void *cuda_stream);
 
 /* The same streaming GEMM as ada_debug_gemm (modes, shapes and layouts as described there, one
  * product per call), for callers that have no device memory to lend and must not allocate any.

@@ -29,7 +29,8 @@ EXPORTS = [
     "ada_adaptive_decode", "ada_debug_capture_logits", "ada_debug_logits_captured", "ada_debug_capture_heads",
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
     "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_plan", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace", "ada_gemm_noalloc",
-    "ada_model_arena_bytes", "ada_model_set_arena", "ada_debug_set_wait_limit",
+    "ada_model_arena_bytes", "ada_model_set_arena", "ada_debug_set_wait_limit", "ada_debug_set_prefill",
+    "ada_debug_dense_gemm", "ada_debug_dense_gemm_work_bytes",
 ]
 
 
@@ -90,6 +91,10 @@ def load() -> C.CDLL:
         L.ada_model_arena_bytes.argtypes = [vp]
         L.ada_model_set_arena.argtypes = [vp, vp, sz]
         L.ada_debug_set_wait_limit.argtypes = [vp, C.c_uint64]
+        L.ada_debug_set_prefill.argtypes = [vp, i32]
+        L.ada_debug_dense_gemm_work_bytes.restype = sz
+        L.ada_debug_dense_gemm_work_bytes.argtypes = [i32]
+        L.ada_debug_dense_gemm.argtypes = [vp, i32, i32, vp, i32, vp, i32, i32, vp, sz, vp]
         L.ada_model_destroy.argtypes = [vp]
         L.ada_model_destroy.restype = None
         L.ada_session_scratch_bytes.restype = sz
@@ -155,6 +160,26 @@ def debug_gemm(W, X, mode: int = 0, repeat: int = 1):
     _ck(lib.ada_debug_gemm(W.data_ptr(), N, K, mode, X.data_ptr(), cols, work.data_ptr() + off, wb, Y.data_ptr(), n_out,
                            repeat, torch.cuda.current_stream().cuda_stream, C.byref(ms)), "ada_debug_gemm")
     return Y, ms.value
+
+
+def debug_dense_gemm(W, X, Y=None):
+    """The dense tcgen05 GEMM of the prompt pass by itself: W bf16 [N, K] (cuda), X fp32 [rows <= 128, K] (cuda).
+    Returns Y fp32 [rows, N]; with Y given, the product is added to it in place."""
+    import torch
+    lib = load()
+    N, K = W.shape
+    rows = X.shape[0]
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.is_contiguous()
+    assert X.is_cuda and X.dtype == torch.float32 and X.is_contiguous() and X.shape[1] == K
+    acc = Y is not None
+    if Y is None:
+        Y = torch.full((rows, N), float("nan"), dtype=torch.float32, device="cuda")
+    wb = lib.ada_debug_dense_gemm_work_bytes(K)
+    work = torch.empty(wb + 256, dtype=torch.uint8, device="cuda")
+    off = (-work.data_ptr()) % 256
+    _ck(lib.ada_debug_dense_gemm(W.data_ptr(), N, K, X.data_ptr(), rows, Y.data_ptr(), Y.shape[1], 1 if acc else 0,
+                                 work.data_ptr() + off, wb, torch.cuda.current_stream().cuda_stream), "ada_debug_dense_gemm")
+    return Y
 
 
 def gemm_noalloc(W, X, Y, mode: int = 0):
@@ -335,6 +360,9 @@ class Session:
 
     def set_launch_steps(self, steps: int):
         _ck(load().ada_debug_set_launch_steps(self.h, steps), "ada_debug_set_launch_steps")
+
+    def set_prefill(self, dense: bool):
+        _ck(load().ada_debug_set_prefill(self.h, 1 if dense else 0), "ada_debug_set_prefill")
 
     def set_wait_limit(self, ns: int):
         _ck(load().ada_debug_set_wait_limit(self.h, ns), "ada_debug_set_wait_limit")

@@ -12,6 +12,7 @@
 #include "kernels.cuh"
 #include "gemm_probe.cuh"
 #include "mega.cuh"
+#include "dense.cuh"
 
 using namespace ada;
 
@@ -71,6 +72,38 @@ int make_weight_map(CUtensorMap *out, const void *W, int N, int K) {
     return ADA_OK;
 }
 
+// Tensor map of a row-major bf16 matrix [rows][K] for the dense GEMM of the prompt pass: dimensions (K, rows),
+// box (64, box_rows), 128-byte swizzle, zero fill outside.
+int make_map_2d(CUtensorMap *out, const void *base, int rows, int K, int box_rows) {
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        cudaError_t e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qr);
+        if (e != cudaSuccess || qr != cudaDriverEntryPointSuccess || !fn) {
+            g_cuda_err = std::string("cuTensorMapEncodeTiled is not available: ") + cudaGetErrorString(e);
+            return ADA_ECUDA;
+        }
+        encode = (EncodeFn)fn;
+    }
+    if (K % 64 || rows < 1 || (uintptr_t)base % 16) return ADA_EUNSUPPORTED;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_cuda_err = "cuTensorMapEncodeTiled (2-D) failed with CUresult " + std::to_string((int)r);
+        return ADA_ECUDA;
+    }
+    return ADA_OK;
+}
+
 }  // namespace
 
 struct ada_model {
@@ -111,6 +144,12 @@ struct ada_session {
     int *exit_at_dev = nullptr;
     int steps_per_launch = 256;
     unsigned long long wait_ns = st::WAIT_NS_DEFAULT;
+    // dense prompt pass (tcgen05 GEMMs over blocks of up to 128 positions)
+    bool dense_ok = false, dense_on = false;   // available for this session / in use by the prefill that is running
+    int cur_rows = 0;                          // rows of the pass being issued
+    __nv_bfloat16 *pf_hi = nullptr, *pf_lo = nullptr;   // [128][max K]: high and low parts of a GEMM's input
+    int *pf_err = nullptr;
+    bool prefill_dense = true;                 // ada_debug_set_prefill
     int64_t launches = 0, syncs = 0, layer_passes = 0;
     // per-class profiling
     bool prof = false;
@@ -134,11 +173,15 @@ namespace {
 // Scratch layout (all offsets 256-byte aligned).
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
-        head_part, logit_stage, head_log, t_out, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qfrag, attn_cnt, rope_freq, part,
+        head_part, logit_stage, head_log, t_out, pf_hi, pf_lo, pf_err, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qfrag, attn_cnt, rope_freq, part,
         grid_ctr, pub, err, total;
 };
 
-int rows_alloc_for(int batch, int max_early) { return std::max(batch * (max_early + 1), 32); }
+bool model_fits_persistent(const ada_config &g);
+// rows a layer pass may carry: the decode rows of all sequences, or a 128-position block of a dense prompt pass
+int rows_alloc_for(const ada_config &g, int batch, int max_early) {
+    return std::max(batch * (max_early + 1), model_fits_persistent(g) ? dg::BM : 32);
+}
 
 // exchange area of weight tiles split between two CTAs: 8 k-splits x 256 tagged words per CTA
 constexpr size_t kPartBytesPerCta = (size_t)st::CONS_WARPS * 256 * sizeof(unsigned long long);
@@ -146,7 +189,7 @@ constexpr int kPartMaxGrid = 256;
 
 Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, int head_blocks) {
     Layout L{};
-    const int R = rows_alloc_for(batch, max_early);
+    const int R = rows_alloc_for(g, batch, max_early);
     const int qd = g.n_q_heads * g.head_dim, qkv_rows = (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim;
     const int n_chunks = (max_seq + kAttnChunk - 1) / kAttnChunk;
     const int max_pages = (max_seq + 15) / 16;  // upper bound for any page size >= 16
@@ -171,6 +214,12 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
     L.logit_stage = take(sizeof(float) * (size_t)R * g.vocab);
     L.head_log = take(sizeof(float) * 4 * kHeadLogCap);
     L.t_out = take(sizeof(float) * (size_t)R * g.d_model);
+    if (model_fits_persistent(g)) {   // dense prompt pass: a GEMM's input as two bf16 matrices [128][K]
+        const size_t kmax = (size_t)std::max(std::max(g.d_model, g.n_q_heads * g.head_dim), g.d_ff);
+        L.pf_hi = take(sizeof(__nv_bfloat16) * dg::BM * kmax);
+        L.pf_lo = take(sizeof(__nv_bfloat16) * dg::BM * kmax);
+        L.pf_err = take(256);
+    }
     // persistent-kernel buffers (bf16 models)
     if (g.dtype == ADA_DTYPE_BF16) {
         L.maps = take(sizeof(CUtensorMap) * (6 * (size_t)g.n_layers + 2));
@@ -245,8 +294,30 @@ void prof_collect(ada_session *S) {
 
 // ---- typed launch helpers --------------------------------------------------------------------
 
+// The same product for a block of a dense prompt pass (rows 0 .. cur_rows - 1, all of them active): the input
+// is split into bf16 high and low parts, then one tcgen05 GEMM kernel (dense.cuh).
+int launch_dense(ada_session *S, int cls, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy) {
+    Prof pf(S, cls, (double)N * K * 2);
+    CUtensorMap mhi, mlo, mw;
+    int rc;
+    if ((rc = make_map_2d(&mhi, S->pf_hi, dg::BM, K, dg::BM)) || (rc = make_map_2d(&mlo, S->pf_lo, dg::BM, K, dg::BM)) ||
+        (rc = make_map_2d(&mw, W, N, K, dg::BN)))
+        return rc;
+    dg::k_split_rows<<<dg::BM, 256, 0, S->stream>>>(X, ldx, S->cur_rows, K, S->pf_hi, S->pf_lo);
+    CK(cudaGetLastError());
+    const int grid = (N + dg::BN - 1) / dg::BN;
+    if (epi == 0)
+        dg::k_dense_gemm<0><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, Y, ldy, S->cur_rows, N, K, S->pf_err);
+    else
+        dg::k_dense_gemm<1><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, Y, ldy, S->cur_rows, N, K, S->pf_err);
+    CK(cudaGetLastError());
+    S->launches += 2;
+    return ADA_OK;
+}
+
 template <typename T>
 int launch_gemv(ada_session *S, int cls, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy, int sel) {
+    if (S->dense_on && sizeof(T) == 2 && sel >= 0) return launch_dense(S, cls, epi, W, N, K, X, ldx, Y, ldy);
     Prof pf(S, cls, (double)N * K * sizeof(T));
     int blocks = std::min((N + 7) / 8, 148 * 4);
     if (epi == 0)
@@ -952,7 +1023,7 @@ int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, i
     S->m = m;
     S->batch = batch; S->max_seq = max_seq_len; S->page_tokens = page_tokens; S->max_early = max_early;
     S->slots = max_early + 1;
-    S->rows_alloc = rows_alloc_for(batch, max_early);
+    S->rows_alloc = rows_alloc_for(g, batch, max_early);
     S->n_pages = n_pages;
     S->max_pages = (max_seq_len + 15) / 16;
     S->n_chunks = (max_seq_len + kAttnChunk - 1) / kAttnChunk;
@@ -1004,6 +1075,21 @@ int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, i
     {
         int rc = setup_persistent(S, lay);
         if (rc) return fail(rc);
+    }
+    // dense prompt pass: bf16 models of the shapes above on a device with fifth-generation tensor cores
+    S->dense_ok = false;
+    if (model_fits_persistent(g)) {
+        int dev = 0, major = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (major == 10 &&
+            cudaFuncSetAttribute(dg::k_dense_gemm<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dg::DSMEM_BYTES) == cudaSuccess &&
+            cudaFuncSetAttribute(dg::k_dense_gemm<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dg::DSMEM_BYTES) == cudaSuccess) {
+            S->dense_ok = true;
+            S->pf_hi = (__nv_bfloat16 *)(b + lay.pf_hi);
+            S->pf_lo = (__nv_bfloat16 *)(b + lay.pf_lo);
+            S->pf_err = (int *)(b + lay.pf_err);
+        } else cudaGetLastError();
     }
     // free list: pages are handed out from the back, in a scrambled order so that the page-table
     // indirection is always exercised
@@ -1061,7 +1147,10 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
         int32_t zero = 0;
         CK(cudaMemcpyAsync(&S->c.st->capture_n, &zero, sizeof(int32_t), cudaMemcpyHostToDevice, S->stream));
     }
-    if (S->mega && S->path == 1) {
+    // Prompts of some length take the dense pass: blocks of 128 positions, every weight matrix streamed once per block
+    // through the tcgen05 GEMM, the other operations by the per-operation kernels.
+    const bool dense = S->dense_ok && S->prefill_dense && n_prompt >= 32;
+    if (!dense && S->mega && S->path == 1) {
         // prompt passes of eight positions through the persistent kernel
         mg::k_prefill_arm<<<1, 32, 0, S->stream>>>(S->c, n_prompt);
         CK(cudaGetLastError());
@@ -1072,10 +1161,17 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
         S->h_reported[seq] = 0;
         return ADA_OK;
     }
-    const int chunk = std::min(S->rows_alloc, kMaxRows);
+    const int chunk = dense ? dg::BM : std::min(std::min(S->rows_alloc, kMaxRows), 64);
+    if (dense) CK(cudaMemsetAsync(S->pf_err, 0, sizeof(int), S->stream));
+    struct DenseScope {   // dense_on only while this prefill issues its passes
+        ada_session *S;
+        ~DenseScope() { S->dense_on = false; }
+    } scope{S};
+    S->dense_on = dense;
     for (int p0 = 0; p0 < n_prompt; p0 += chunk) {
         const int n = std::min(chunk, n_prompt - p0);
         const int last = p0 + n == n_prompt;
+        S->cur_rows = n;
         if (g.dtype == ADA_DTYPE_BF16)
             k_prefill_begin<__nv_bfloat16><<<1, 256, 0, S->stream>>>(S->c, (const __nv_bfloat16 *)m->tok_embed, g.rope_base, seq, p0, n);
         else
@@ -1086,6 +1182,14 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
         k_prefill_end<<<1, 32, 0, S->stream>>>(S->c, seq, p0 + n, last, n_prompt);
         CK(cudaGetLastError());
         if (last && seq == 0 && (rc = capture_rows(S, n - 1))) return rc;
+    }
+    if (dense) {
+        CK(cudaMemcpyAsync(S->pinned, S->pf_err, sizeof(int), cudaMemcpyDeviceToHost, S->stream));
+        CK(cudaStreamSynchronize(S->stream));
+        if (S->pinned[0] != 0) {
+            g_cuda_err = "dense prompt pass: a bounded device-side wait expired";
+            return ADA_ETIMEOUT;
+        }
     }
     CK(cudaStreamSynchronize(S->stream));
     S->prefilled[seq] = 1;
@@ -1216,6 +1320,13 @@ int ada_debug_get_path(ada_session *S, int32_t *path_out) {
     return ADA_OK;
 }
 
+int ada_debug_set_prefill(ada_session *S, int32_t dense) {
+    if (!S || dense < 0 || dense > 1) return ADA_EINVAL;
+    if (dense && !S->dense_ok) return ADA_EUNSUPPORTED;
+    S->prefill_dense = dense != 0;
+    return ADA_OK;
+}
+
 int ada_debug_set_launch_steps(ada_session *S, int32_t steps) {
     if (!S || steps < 1) return ADA_EINVAL;
     S->steps_per_launch = steps;
@@ -1291,6 +1402,42 @@ int ada_debug_gemm(const void *W_dev, int32_t N, int32_t K, int32_t mode, const 
     cudaEventDestroy(e1);
     CK(ce);
     if (ms_out) *ms_out = ms;
+    return herr ? ADA_ETIMEOUT : ADA_OK;
+}
+
+size_t ada_debug_dense_gemm_work_bytes(int32_t K) {
+    if (K < 64) return 0;
+    return 2 * (size_t)dg::BM * K * sizeof(__nv_bfloat16) + 256;
+}
+
+int ada_debug_dense_gemm(const void *W_dev, int32_t N, int32_t K, const float *X_dev, int32_t rows, float *Y_dev, int32_t ldy,
+                         int32_t accumulate, void *work_dev, size_t work_bytes, void *cuda_stream) {
+    if (!W_dev || !X_dev || !Y_dev || !work_dev || N < 1 || K < 64 || K % 64 || rows < 1 || rows > dg::BM || ldy < N) return ADA_EINVAL;
+    if ((uintptr_t)W_dev % 16 || (uintptr_t)work_dev % 256 || (uintptr_t)Y_dev % 16 || ldy % 4) return ADA_EINVAL;
+    if (work_bytes < ada_debug_dense_gemm_work_bytes(K)) return ADA_ECAPACITY;
+    int dev = 0, major = 0;
+    CK(cudaGetDevice(&dev));
+    CK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major != 10) return ADA_EUNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    __nv_bfloat16 *hi = (__nv_bfloat16 *)work_dev, *lo = hi + (size_t)dg::BM * K;
+    int *err = (int *)(lo + (size_t)dg::BM * K);
+    CUtensorMap mhi, mlo, mw;
+    int rc;
+    if ((rc = make_map_2d(&mhi, hi, dg::BM, K, dg::BM)) || (rc = make_map_2d(&mlo, lo, dg::BM, K, dg::BM)) || (rc = make_map_2d(&mw, W_dev, N, K, dg::BN)))
+        return rc;
+    CK(cudaFuncSetAttribute(dg::k_dense_gemm<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dg::DSMEM_BYTES));
+    CK(cudaFuncSetAttribute(dg::k_dense_gemm<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dg::DSMEM_BYTES));
+    CK(cudaMemsetAsync(err, 0, sizeof(int), stream));
+    dg::k_split_rows<<<dg::BM, 256, 0, stream>>>(X_dev, K, rows, K, hi, lo);
+    CK(cudaGetLastError());
+    const int grid = (N + dg::BN - 1) / dg::BN;
+    if (accumulate) dg::k_dense_gemm<1><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, stream>>>(mhi, mlo, mw, Y_dev, ldy, rows, N, K, err);
+    else dg::k_dense_gemm<0><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, stream>>>(mhi, mlo, mw, Y_dev, ldy, rows, N, K, err);
+    CK(cudaGetLastError());
+    int herr = 0;
+    CK(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    CK(cudaStreamSynchronize(stream));
     return herr ? ADA_ETIMEOUT : ADA_OK;
 }
 

@@ -9,7 +9,7 @@
 
 namespace ada {
 
-constexpr int kMaxRows = 64;        // rows (tokens) one layer pass can carry
+constexpr int kMaxRows = 128;       // rows (tokens) one layer pass can carry (a block of a dense prompt pass)
 constexpr int kAttnChunk = 128;     // attention split size; chunk c covers positions [128c, 128c+127]
 constexpr int kMaxTape = 4096;
 constexpr int kHeadLogCap = 1 << 16;

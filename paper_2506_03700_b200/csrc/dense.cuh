@@ -1,0 +1,232 @@
+// Dense GEMM for the prompt pass ("KV cache <- LM(x)", first line of Algorithm 1) on the fifth-generation
+// tensor cores of sm_100a: tcgen05.mma with the accumulator in tensor memory, operands staged in shared
+// memory by TMA.
+//
+// A prompt block of up to 128 positions goes through a weight matrix in one product
+//     Y[m][n] (+)= sum_k X[m][k] W[n][k],   m < 128 positions, n < N weight rows,
+// so a weight byte fetched from HBM is used for 128 tokens instead of the eight of a decode pass: here the
+// contraction really is dense, and the tensor cores are what it belongs on.  X arrives as two bf16
+// matrices, a high part and a low part (x = hi + lo, as everywhere in this library: fp32 activations
+// lose nothing), both multiplied into the same fp32 accumulator.
+//
+// One CTA computes a tile of 128 positions x 64 weight rows.  Warp 0 is the TMA producer (one k block of
+// 64 elements per stage: the 128-byte-swizzled tiles of X.hi, X.lo and W), warp 1 allocates the tensor
+// memory and issues the MMAs (one elected thread; UMMA shape M = 128, N = 64, K = 16, both operands
+// K-major), warps 2..5 read the accumulator back (tcgen05.ld, 32 lanes per warp) and write it out.
+// Every wait is bounded; on expiry an error word is set, the roles leave their loops, the tensor
+// memory is released and the kernel ends.
+#pragma once
+
+#include "stream.cuh"
+
+namespace ada {
+namespace dg {
+
+using namespace st;
+
+constexpr int BM = 128;     // positions per tile (UMMA M)
+constexpr int BN = 64;      // weight rows per tile (UMMA N)
+constexpr int BK = 64;      // k elements per stage: one 128-byte swizzle row
+constexpr int STAGES = 5;
+constexpr int DTHREADS = 192;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = 2 * A_BYTES + B_BYTES;
+// The tensor core adds into its fp32 accumulator with truncation, so the error of one accumulator grows in
+// proportion to the products added (1e-3 absolute at K = 14336 with sums of size 10).  The k blocks therefore
+// take NACC accumulators in turn, which the epilogue adds up in registers (round to nearest).
+constexpr int NACC = 4;
+constexpr int TMEM_COLS = NACC * BN;   // fp32 accumulator columns (a power of two >= 32)
+constexpr unsigned long long DENSE_WAIT_NS = 2000000000ull;
+
+struct DSmem {   // must start on a 1024-byte boundary (swizzle pattern)
+    alignas(1024) unsigned char stage[STAGES][STAGE_BYTES];   // [X.hi 128 x 64 | X.lo 128 x 64 | W 64 x 64], rows of 128 B
+    alignas(8) unsigned long long full[STAGES], empty[STAGES], acc_full;
+    uint32_t tmem_base;
+    int abort;
+};
+constexpr size_t DSMEM_BYTES = sizeof(DSmem) + 1024;
+static_assert(STAGE_BYTES % 1024 == 0 && A_BYTES % 1024 == 0, "operand tiles must start on 1024-byte boundaries");
+static_assert(DSMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a block may use");
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(s32(dst)),
+                 "l"(map), "r"(c0), "r"(c1), "r"(s32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled (the layout
+// a TMA box of 64 bf16 x rows leaves): start address / 16 in bits 0-13, leading byte offset / 16 in bits
+// 16-29 (1: not used by swizzled K-major tiles), stride byte offset / 16 in bits 32-45 (1024 bytes from one
+// group of eight rows to the next), descriptor version 1 in bits 46-47, swizzle mode 2 (128 bytes) in bits 61-63.
+__device__ __forceinline__ unsigned long long smem_desc(uint32_t saddr) {
+    return (unsigned long long)((saddr >> 4) & 0x3fffu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator (bits 4-5 = 1), bf16 A and B (bits 7-9 and 10-12 = 1),
+// both K-major (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void umma(uint32_t d_tmem, unsigned long long adesc, unsigned long long bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+        : "memory");
+}
+// the mbarrier is arrived on once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(unsigned long long *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s32(bar)) : "memory");
+}
+
+struct DWait {
+    DSmem *sm;
+    int *err;
+};
+__device__ __forceinline__ bool dwait(const DWait &w, unsigned long long *bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 255u) == 0) {
+            if (*(volatile int *)&w.sm->abort) return false;
+            const unsigned long long t = gtime();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > DENSE_WAIT_NS) {
+                atomicCAS(w.err, 0, ERR_TIMEOUT_MBAR);
+                *(volatile int *)&w.sm->abort = 1;
+                return false;
+            }
+        }
+    }
+}
+
+// EPI 0: Y[m][n] = acc.  EPI 1: Y[m][n] += acc (every element has one writer).  Rows m >= rows are not written.
+// mapXhi / mapXlo: 2-D maps over the bf16 matrices [128][K] (box 64 x 128); mapW: over W [N][K] (box 64 x 64);
+// all 128-byte swizzled, zero fill outside.  K a multiple of 64.
+template <int EPI>
+__global__ void __launch_bounds__(DTHREADS, 1)
+k_dense_gemm(const __grid_constant__ CUtensorMap mapXhi, const __grid_constant__ CUtensorMap mapXlo,
+             const __grid_constant__ CUtensorMap mapW, float *__restrict__ Y, int ldy, int rows, int N, int K, int *err) {
+    extern __shared__ unsigned char dsm_raw[];
+    DSmem *sm = reinterpret_cast<DSmem *>(dsm_raw + ((1024u - (s32(dsm_raw) & 1023u)) & 1023u));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN, nkb = K / BK;
+    const DWait W{sm, err};
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(&sm->full[i], 1); mbar_init(&sm->empty[i], 1); }
+        mbar_init(&sm->acc_full, 1);
+        sm->abort = 0;
+        fence_mbar_init();
+        fence_proxy_async();
+    }
+    __syncthreads();
+    if (warp == 1) {   // tensor memory for the accumulator: allocated, and later released, by this one warp
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *(volatile uint32_t *)&sm->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                if (!dwait(W, &sm->empty[s], ((kb / STAGES) & 1) ^ 1)) break;
+                mbar_expect_tx(&sm->full[s], (uint32_t)STAGE_BYTES);
+                tma_load_2d(sm->stage[s], &mapXhi, kb * BK, 0, &sm->full[s]);
+                tma_load_2d(sm->stage[s] + A_BYTES, &mapXlo, kb * BK, 0, &sm->full[s]);
+                tma_load_2d(sm->stage[s] + 2 * A_BYTES, &mapW, kb * BK, n0, &sm->full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                const int s = kb % STAGES;
+                ok = dwait(W, &sm->full[s], (kb / STAGES) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const unsigned long long ahi = smem_desc(s32(sm->stage[s])), alo = smem_desc(s32(sm->stage[s] + A_BYTES)),
+                                         b = smem_desc(s32(sm->stage[s] + 2 * A_BYTES));
+#pragma unroll
+                const uint32_t acc = tmem + (uint32_t)((kb % NACC) * BN);
+                for (int k = 0; k < BK / 16; ++k) {   // 32 bytes further along the swizzled row per K = 16 step
+                    umma(acc, ahi + 2 * k, b + 2 * k, (kb >= NACC || k != 0) ? 1u : 0u);
+                    umma(acc, alo + 2 * k, b + 2 * k, 1u);
+                }
+                umma_commit(&sm->empty[s]);   // the stage is free once these MMAs have read it
+            }
+            umma_commit(&sm->acc_full);
+        }
+    } else {
+        // epilogue: warp w may read the 32 lanes 32 (w % 4) .. of the tensor memory; lane = position within the block
+        const int q = warp & 3, m = q * 32 + lane;
+        const bool ok = dwait(W, &sm->acc_full, 0);
+        tc_fence_after();
+        if (ok) {
+            const int nacc = min(NACC, nkb);
+#pragma unroll
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t v[16];
+#pragma unroll
+                for (int a = 0; a < NACC; ++a) {
+                    if (a >= nacc) continue;
+                    uint32_t t[16];
+                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                                 : "=r"(t[0]), "=r"(t[1]), "=r"(t[2]), "=r"(t[3]), "=r"(t[4]), "=r"(t[5]), "=r"(t[6]), "=r"(t[7]), "=r"(t[8]),
+                                   "=r"(t[9]), "=r"(t[10]), "=r"(t[11]), "=r"(t[12]), "=r"(t[13]), "=r"(t[14]), "=r"(t[15])
+                                 : "r"(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * BN + c0)));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = a == 0 ? t[j] : __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(t[j]));
+                }
+                if (m < rows) {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        const int n = n0 + c0 + j;
+                        if (n + 3 < N) {
+                            float4 *p = reinterpret_cast<float4 *>(Y + (size_t)m * ldy + n);
+                            float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                            if (EPI == 1) { const float4 r = *p; o.x += r.x; o.y += r.y; o.z += r.z; o.w += r.w; }
+                            *p = o;
+                        } else {
+                            for (int e = 0; e < 4; ++e)
+                                if (n + e < N) {
+                                    float *p = Y + (size_t)m * ldy + n + e;
+                                    *p = (EPI == 1 ? *p : 0.f) + __uint_as_float(v[j + e]);
+                                }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*(volatile int *)&sm->abort) {   // copies already issued may still be landing: give them time before the block's memory goes
+        const unsigned long long t0 = gtime();
+        while (gtime() - t0 < 200000ull) __nanosleep(1000);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// fp32 rows X[r][ldx] (r < rows) -> the two bf16 matrices [128][K] the dense GEMM reads: high part and low part
+// (x = hi + lo); rows >= `rows` are zero.  One block per row.
+__global__ void k_split_rows(const float *__restrict__ X, int ldx, int rows, int K, __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo) {
+    const int r = blockIdx.x;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        const float v = r < rows ? X[(size_t)r * ldx + k] : 0.f;
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[(size_t)r * K + k] = h;
+        lo[(size_t)r * K + k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+}  // namespace dg
+}  // namespace ada

@@ -57,3 +57,19 @@ def test_bad_arguments_are_refused():
     with pytest.raises(binding.AdaError) as e:
         binding.debug_gemm(W, X, 0)
     assert e.value.code == -1
+
+
+# ---------------------------------------------------------------- dense GEMM of the prompt pass (tcgen05)
+
+@pytest.mark.parametrize("N,K,rows", [(64, 64, 128), (64, 256, 5), (200, 512, 128), (6144, 4096, 77), (4096, 14336, 128)])
+def test_dense_gemm_matches_float64(N, K, rows):
+    W = synth.normal_tensor(9, 11, (N, K), 0.05, torch.bfloat16, "cuda")
+    X = synth.normal_tensor(9, 12, (rows, K), 1.0, torch.float32, "cuda")
+    Y = binding.debug_dense_gemm(W, X)
+    ref = X.double().cpu().numpy() @ W.double().cpu().numpy().T
+    assert torch.isfinite(Y).all()
+    assert np.abs(Y.double().cpu().numpy() - ref).max() <= 2e-5 * max(1.0, np.abs(ref).max())
+    # accumulate form: the product is added to what the output holds
+    Y2 = torch.ones_like(Y)
+    binding.debug_dense_gemm(W, X, Y2)
+    assert np.abs(Y2.double().cpu().numpy() - (ref + 1.0)).max() <= 2e-5 * max(1.0, np.abs(ref).max())
