@@ -149,6 +149,8 @@ struct ada_session {
     int cur_rows = 0;                          // rows of the pass being issued
     __nv_bfloat16 *pf_hi = nullptr, *pf_lo = nullptr;   // [128][max K]: high and low parts of a GEMM's input
     int *pf_err = nullptr;
+    float *pf_part = nullptr;                  // shares of depth-split products: [splits][128][N]
+    size_t pf_part_bytes = 0;
     bool prefill_dense = true;                 // ada_debug_set_prefill
     int64_t launches = 0, syncs = 0, layer_passes = 0;
     // per-class profiling
@@ -173,11 +175,12 @@ namespace {
 // Scratch layout (all offsets 256-byte aligned).
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
-        head_part, logit_stage, head_log, t_out, pf_hi, pf_lo, pf_err, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qfrag, attn_cnt, rope_freq, part,
+        head_part, logit_stage, head_log, t_out, pf_hi, pf_lo, pf_err, pf_part, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qfrag, attn_cnt, rope_freq, part,
         grid_ctr, pub, err, total;
 };
 
 bool model_fits_persistent(const ada_config &g);
+constexpr size_t kDenseSplitMax = 4;   // shares of a depth-split dense product (O and down projections)
 // rows a layer pass may carry: the decode rows of all sequences, or a 128-position block of a dense prompt pass
 int rows_alloc_for(const ada_config &g, int batch, int max_early) {
     return std::max(batch * (max_early + 1), model_fits_persistent(g) ? dg::BM : 32);
@@ -219,6 +222,7 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
         L.pf_hi = take(sizeof(__nv_bfloat16) * dg::BM * kmax);
         L.pf_lo = take(sizeof(__nv_bfloat16) * dg::BM * kmax);
         L.pf_err = take(256);
+        L.pf_part = take(kDenseSplitMax * sizeof(float) * dg::BM * (size_t)g.d_model);
     }
     // persistent-kernel buffers (bf16 models)
     if (g.dtype == ADA_DTYPE_BF16) {
@@ -294,30 +298,109 @@ void prof_collect(ada_session *S) {
 
 // ---- typed launch helpers --------------------------------------------------------------------
 
-// The same product for a block of a dense prompt pass (rows 0 .. cur_rows - 1, all of them active): the input
-// is split into bf16 high and low parts, then one tcgen05 GEMM kernel (dense.cuh).
-int launch_dense(ada_session *S, int cls, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy) {
+// ---- dense prompt pass: one decoder layer over a block of up to 128 prompt rows (rows 0 .. cur_rows - 1) -------
+
+// One tcgen05 GEMM over the input last split into S->pf_hi / pf_lo (depth K): Y = or += X W^T.  Products with few
+// tiles are split in depth over several CTAs per tile (shares added in a fixed order by k_dense_reduce).
+int dense_gemm(ada_session *S, int cls, bool add, const void *W, int N, int K, float *Y, int ldy) {
     Prof pf(S, cls, (double)N * K * 2);
     CUtensorMap mhi, mlo, mw;
     int rc;
     if ((rc = make_map_2d(&mhi, S->pf_hi, dg::BM, K, dg::BM)) || (rc = make_map_2d(&mlo, S->pf_lo, dg::BM, K, dg::BM)) ||
         (rc = make_map_2d(&mw, W, N, K, dg::BN)))
         return rc;
-    dg::k_split_rows<<<dg::BM, 256, 0, S->stream>>>(X, ldx, S->cur_rows, K, S->pf_hi, S->pf_lo);
+    const int tiles = (N + dg::BN - 1) / dg::BN, nkb = K / dg::BK;
+    int splits = 1;
+    while (tiles * splits < 96 && splits * 2 <= nkb / 8 && (size_t)(splits * 2) * dg::BM * N * sizeof(float) <= S->pf_part_bytes && N % 4 == 0) splits *= 2;
+    if (splits == 1) {
+        if (add) dg::k_dense_gemm<1><<<tiles, dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, Y, ldy, S->cur_rows, N, K, 0, S->pf_err);
+        else dg::k_dense_gemm<0><<<tiles, dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, Y, ldy, S->cur_rows, N, K, 0, S->pf_err);
+        CK(cudaGetLastError());
+        S->launches++;
+    } else {
+        const size_t stride = (size_t)dg::BM * N;
+        dg::k_dense_gemm<0><<<dim3(tiles, splits), dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, S->pf_part, N, S->cur_rows, N, K, stride, S->pf_err);
+        CK(cudaGetLastError());
+        dg::k_dense_reduce<<<dim3((N / 4 + 255) / 256, S->cur_rows), 256, 0, S->stream>>>(S->pf_part, stride, splits, Y, ldy, S->cur_rows, N, add ? 1 : 0);
+        CK(cudaGetLastError());
+        S->launches += 2;
+    }
+    return ADA_OK;
+}
+
+int run_layer_dense(ada_session *S, int layer, int rows) {
+    const ada_model *m = S->m;
+    const ada_config &g = m->cfg;
+    const LayerW &w = m->layers[layer];
+    const int d = g.d_model, hd = g.head_dim, qd = g.n_q_heads * hd, kvd = g.n_kv_heads * hd, qkv_rows = S->c.qkv_rows;
+    typedef __nv_bfloat16 T;
+    int rc;
+    S->layer_passes++;
+    {
+        Prof pf(S, 1, 0.0);
+        dg::k_norm_split_rows<<<dg::BM, 256, 0, S->stream>>>(S->c.resid, rows, d, (const T *)w.attn_norm, g.rms_eps, S->pf_hi, S->pf_lo);
+    }
     CK(cudaGetLastError());
-    const int grid = (N + dg::BN - 1) / dg::BN;
-    if (epi == 0)
-        dg::k_dense_gemm<0><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, Y, ldy, S->cur_rows, N, K, S->pf_err);
-    else
-        dg::k_dense_gemm<1><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, S->stream>>>(mhi, mlo, mw, Y, ldy, S->cur_rows, N, K, S->pf_err);
+    S->launches++;
+    if ((const T *)w.wk == (const T *)w.wq + (size_t)qd * d && (const T *)w.wv == (const T *)w.wk + (size_t)kvd * d) {
+        if ((rc = dense_gemm(S, 2, false, w.wq, qkv_rows, d, S->c.qkv, qkv_rows))) return rc;
+    } else {
+        if ((rc = dense_gemm(S, 2, false, w.wq, qd, d, S->c.qkv, qkv_rows))) return rc;
+        if ((rc = dense_gemm(S, 2, false, w.wk, kvd, d, S->c.qkv + qd, qkv_rows))) return rc;
+        if ((rc = dense_gemm(S, 2, false, w.wv, kvd, d, S->c.qkv + qd + kvd, qkv_rows))) return rc;
+    }
+    {
+        Prof pf(S, 3, 0.0);
+        k_rope_kv<T><<<rows, 128, 0, S->stream>>>(S->c, layer);
+    }
     CK(cudaGetLastError());
-    S->launches += 2;
+    S->launches++;
+    {
+        Prof pf(S, 4, 0.0);
+        const dim3 grid((rows + PF_Q - 1) / PF_Q, g.n_kv_heads);
+        const int group = g.n_q_heads / g.n_kv_heads;
+#define PF_ATTN(E, G) k_pf_attn<E, G><<<grid, PF_Q * 32, 0, S->stream>>>(S->c, layer, rows)
+        if (hd == 128) { if (group == 4) PF_ATTN(4, 4); else if (group == 2) PF_ATTN(4, 2); else if (group == 1) PF_ATTN(4, 1); else return ADA_EUNSUPPORTED; }
+        else if (hd == 64) { if (group == 4) PF_ATTN(2, 4); else if (group == 2) PF_ATTN(2, 2); else if (group == 1) PF_ATTN(2, 1); else return ADA_EUNSUPPORTED; }
+        else return ADA_EUNSUPPORTED;
+#undef PF_ATTN
+    }
+    CK(cudaGetLastError());
+    S->launches++;
+    {
+        Prof pf(S, 11, 0.0);
+        dg::k_split_rows<<<dg::BM, 256, 0, S->stream>>>(S->c.attn_out, qd, rows, qd, S->pf_hi, S->pf_lo);
+    }
+    CK(cudaGetLastError());
+    if ((rc = dense_gemm(S, 5, true, w.wo, d, qd, S->c.resid, d))) return rc;
+    {
+        Prof pf(S, 1, 0.0);
+        dg::k_norm_split_rows<<<dg::BM, 256, 0, S->stream>>>(S->c.resid, rows, d, (const T *)w.ffn_norm, g.rms_eps, S->pf_hi, S->pf_lo);
+    }
+    CK(cudaGetLastError());
+    if ((const T *)w.w_up == (const T *)w.w_gate + (size_t)g.d_ff * d) {
+        if ((rc = dense_gemm(S, 6, false, w.w_gate, 2 * g.d_ff, d, S->c.gu, 2 * g.d_ff))) return rc;
+    } else {
+        if ((rc = dense_gemm(S, 6, false, w.w_gate, g.d_ff, d, S->c.gu, 2 * g.d_ff))) return rc;
+        if ((rc = dense_gemm(S, 6, false, w.w_up, g.d_ff, d, S->c.gu + g.d_ff, 2 * g.d_ff))) return rc;
+    }
+    {
+        Prof pf(S, 7, 0.0);
+        k_swiglu<<<dim3((g.d_ff + 255) / 256, rows), 256, 0, S->stream>>>(S->c, layer);
+    }
+    CK(cudaGetLastError());
+    {
+        Prof pf(S, 11, 0.0);
+        dg::k_split_rows<<<dg::BM, 256, 0, S->stream>>>(S->c.hact, g.d_ff, rows, g.d_ff, S->pf_hi, S->pf_lo);
+    }
+    CK(cudaGetLastError());
+    S->launches += 4;
+    if ((rc = dense_gemm(S, 8, true, w.w_down, d, g.d_ff, S->c.resid, d))) return rc;
     return ADA_OK;
 }
 
 template <typename T>
 int launch_gemv(ada_session *S, int cls, int epi, const void *W, int N, int K, const float *X, int ldx, float *Y, int ldy, int sel) {
-    if (S->dense_on && sizeof(T) == 2 && sel >= 0) return launch_dense(S, cls, epi, W, N, K, X, ldx, Y, ldy);
     Prof pf(S, cls, (double)N * K * sizeof(T));
     int blocks = std::min((N + 7) / 8, 148 * 4);
     if (epi == 0)
@@ -444,6 +527,7 @@ int run_head_t(ada_session *S, int layer1, int sel, int rows) {
 }
 
 int run_layer(ada_session *S, int layer, int rows) {
+    if (S->dense_on) return run_layer_dense(S, layer, rows);
     return S->m->cfg.dtype == ADA_DTYPE_BF16 ? run_layer_t<__nv_bfloat16>(S, layer, rows) : run_layer_t<float>(S, layer, rows);
 }
 int run_head(ada_session *S, int layer1, int sel, int rows) {
@@ -1089,6 +1173,8 @@ int ada_session_create(const ada_model *m, int32_t batch, int32_t max_seq_len, i
             S->pf_hi = (__nv_bfloat16 *)(b + lay.pf_hi);
             S->pf_lo = (__nv_bfloat16 *)(b + lay.pf_lo);
             S->pf_err = (int *)(b + lay.pf_err);
+            S->pf_part = (float *)(b + lay.pf_part);
+            S->pf_part_bytes = kDenseSplitMax * sizeof(float) * dg::BM * (size_t)g.d_model;
         } else cudaGetLastError();
     }
     // free list: pages are handed out from the back, in a scrambled order so that the page-table
@@ -1432,8 +1518,8 @@ int ada_debug_dense_gemm(const void *W_dev, int32_t N, int32_t K, const float *X
     dg::k_split_rows<<<dg::BM, 256, 0, stream>>>(X_dev, K, rows, K, hi, lo);
     CK(cudaGetLastError());
     const int grid = (N + dg::BN - 1) / dg::BN;
-    if (accumulate) dg::k_dense_gemm<1><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, stream>>>(mhi, mlo, mw, Y_dev, ldy, rows, N, K, err);
-    else dg::k_dense_gemm<0><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, stream>>>(mhi, mlo, mw, Y_dev, ldy, rows, N, K, err);
+    if (accumulate) dg::k_dense_gemm<1><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, stream>>>(mhi, mlo, mw, Y_dev, ldy, rows, N, K, 0, err);
+    else dg::k_dense_gemm<0><<<grid, dg::DTHREADS, dg::DSMEM_BYTES, stream>>>(mhi, mlo, mw, Y_dev, ldy, rows, N, K, 0, err);
     CK(cudaGetLastError());
     int herr = 0;
     CK(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, stream));

@@ -102,16 +102,21 @@ __device__ __forceinline__ bool dwait(const DWait &w, unsigned long long *bar, u
 }
 
 // EPI 0: Y[m][n] = acc.  EPI 1: Y[m][n] += acc (every element has one writer).  Rows m >= rows are not written.
+// gridDim.y > 1 splits the depth: block row y multiplies its share of the k blocks and writes (EPI 0) to
+// Y + y * split_stride; k_dense_reduce then adds the shares in a fixed order.
 // mapXhi / mapXlo: 2-D maps over the bf16 matrices [128][K] (box 64 x 128); mapW: over W [N][K] (box 64 x 64);
 // all 128-byte swizzled, zero fill outside.  K a multiple of 64.
 template <int EPI>
 __global__ void __launch_bounds__(DTHREADS, 1)
 k_dense_gemm(const __grid_constant__ CUtensorMap mapXhi, const __grid_constant__ CUtensorMap mapXlo,
-             const __grid_constant__ CUtensorMap mapW, float *__restrict__ Y, int ldy, int rows, int N, int K, int *err) {
+             const __grid_constant__ CUtensorMap mapW, float *__restrict__ Y, int ldy, int rows, int N, int K, size_t split_stride, int *err) {
     extern __shared__ unsigned char dsm_raw[];
     DSmem *sm = reinterpret_cast<DSmem *>(dsm_raw + ((1024u - (s32(dsm_raw) & 1023u)) & 1023u));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * BN, nkb = K / BK;
+    const int n0 = blockIdx.x * BN, nkb_all = K / BK;
+    const int kb_begin = (int)((long long)nkb_all * blockIdx.y / gridDim.y), kb_end = (int)((long long)nkb_all * (blockIdx.y + 1) / gridDim.y);
+    const int nkb = kb_end - kb_begin;
+    Y += (size_t)blockIdx.y * split_stride;
     const DWait W{sm, err};
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(&sm->full[i], 1); mbar_init(&sm->empty[i], 1); }
@@ -136,9 +141,9 @@ k_dense_gemm(const __grid_constant__ CUtensorMap mapXhi, const __grid_constant__
                 const int s = kb % STAGES;
                 if (!dwait(W, &sm->empty[s], ((kb / STAGES) & 1) ^ 1)) break;
                 mbar_expect_tx(&sm->full[s], (uint32_t)STAGE_BYTES);
-                tma_load_2d(sm->stage[s], &mapXhi, kb * BK, 0, &sm->full[s]);
-                tma_load_2d(sm->stage[s] + A_BYTES, &mapXlo, kb * BK, 0, &sm->full[s]);
-                tma_load_2d(sm->stage[s] + 2 * A_BYTES, &mapW, kb * BK, n0, &sm->full[s]);
+                tma_load_2d(sm->stage[s], &mapXhi, (kb_begin + kb) * BK, 0, &sm->full[s]);
+                tma_load_2d(sm->stage[s] + A_BYTES, &mapXlo, (kb_begin + kb) * BK, 0, &sm->full[s]);
+                tma_load_2d(sm->stage[s] + 2 * A_BYTES, &mapW, (kb_begin + kb) * BK, n0, &sm->full[s]);
             }
         }
     } else if (warp == 1) {
@@ -151,8 +156,8 @@ k_dense_gemm(const __grid_constant__ CUtensorMap mapXhi, const __grid_constant__
                 tc_fence_after();
                 const unsigned long long ahi = smem_desc(s32(sm->stage[s])), alo = smem_desc(s32(sm->stage[s] + A_BYTES)),
                                          b = smem_desc(s32(sm->stage[s] + 2 * A_BYTES));
-#pragma unroll
                 const uint32_t acc = tmem + (uint32_t)((kb % NACC) * BN);
+#pragma unroll
                 for (int k = 0; k < BK / 16; ++k) {   // 32 bytes further along the swizzled row per K = 16 step
                     umma(acc, ahi + 2 * k, b + 2 * k, (kb >= NACC || k != 0) ? 1u : 0u);
                     umma(acc, alo + 2 * k, b + 2 * k, 1u);
@@ -213,6 +218,50 @@ k_dense_gemm(const __grid_constant__ CUtensorMap mapXhi, const __grid_constant__
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// Y[m][n] = (or +=) sum over the `splits` shares of a depth-split product, added in index order.
+__global__ void k_dense_reduce(const float *__restrict__ part, size_t split_stride, int splits, float *__restrict__ Y, int ldy, int rows, int N, int add) {
+    const int m = blockIdx.y;
+    if (m >= rows) return;
+    for (int n = (blockIdx.x * blockDim.x + threadIdx.x) * 4; n < N; n += gridDim.x * blockDim.x * 4) {
+        float4 a = *reinterpret_cast<const float4 *>(part + (size_t)m * N + n);
+        for (int s = 1; s < splits; ++s) {
+            const float4 b = *reinterpret_cast<const float4 *>(part + s * split_stride + (size_t)m * N + n);
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        float4 *y = reinterpret_cast<float4 *>(Y + (size_t)m * ldy + n);
+        if (add) { const float4 r = *y; a.x += r.x; a.y += r.y; a.z += r.z; a.w += r.w; }
+        *y = a;
+    }
+}
+
+// RMSNorm and split in one pass: x = resid[r] / sqrt(mean(resid[r]^2) + eps) * g -> high and low parts.  One block
+// (256 threads) per row; rows >= `rows` are zero.
+__global__ void __launch_bounds__(256) k_norm_split_rows(const float *__restrict__ X, int rows, int K, const __nv_bfloat16 *__restrict__ gain,
+                                                         float eps, __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo) {
+    const int r = blockIdx.x;
+    __shared__ float red[8];
+    float rstd = 0.f;
+    if (r < rows) {
+        const float *x = X + (size_t)r * K;
+        float ss = 0.f;
+        for (int i = threadIdx.x; i < K; i += 256) ss = fmaf(x[i], x[i], ss);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot += red[w];
+        rstd = 1.0f / sqrtf(tot / K + eps);
+    }
+    for (int k = threadIdx.x; k < K; k += 256) {
+        const float v = r < rows ? X[(size_t)r * K + k] * rstd * __bfloat162float(gain[k]) : 0.f;
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[(size_t)r * K + k] = h;
+        lo[(size_t)r * K + k] = __float2bfloat16_rn(v - __bfloat162float(h));
     }
 }
 

@@ -408,6 +408,76 @@ __global__ void k_attn_combine(Ctx c, int layer) {
     }
 }
 
+// Causal attention of a block of prompt rows (a dense prompt pass), bf16 cache.  One block = one kv head x
+// PF_Q consecutive rows (one warp per row, serving all `group` q heads of the kv head); the K and V rows of 32
+// cache positions at a time are staged in shared memory once for the whole block, so a cached row is fetched
+// from L2 once per PF_Q x group (query, head) pairs instead of once per pair.  Online softmax in position
+// order per (row, head); the context is not split, so the result goes straight to attn_out.
+// EPL = head_dim / 32 elements per lane, GROUP = q heads per kv head (1, 2 or 4).
+constexpr int PF_Q = 4, PF_T = 32;
+template <int EPL, int GROUP>
+__global__ void __launch_bounds__(PF_Q * 32) k_pf_attn(Ctx c, int layer, int rows) {
+    constexpr int HD = EPL * 32;
+    __shared__ __align__(16) __nv_bfloat16 sK[PF_T][HD], sV[PF_T][HD];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, kvh = blockIdx.y;
+    const int r = blockIdx.x * PF_Q + warp;
+    const bool live = r < rows;
+    const int seq = c.rt->seq[min(r, rows - 1)], pos = live ? c.rt->pos[r] : -1;
+    const int r_last = min(blockIdx.x * PF_Q + PF_Q, rows) - 1, pos_max = c.rt->pos[r_last];   // rows of a block are consecutive positions
+    const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
+    const float scale = rsqrtf((float)HD);
+    float q[GROUP][EPL], acc[GROUP][EPL], m[GROUP], l[GROUP];
+#pragma unroll
+    for (int g = 0; g < GROUP; ++g) {
+        m[g] = -INFINITY; l[g] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            q[g][e] = live ? c.q[((size_t)r * c.nq + kvh * GROUP + g) * HD + lane * EPL + e] * scale : 0.f;
+            acc[g][e] = 0.f;
+        }
+    }
+    for (int t0 = 0; t0 <= pos_max; t0 += PF_T) {
+        __syncthreads();   // the previous tile has been used
+        for (int i = threadIdx.x; i < PF_T * (HD / 8); i += PF_Q * 32) {
+            const int t = i / (HD / 8), ch = i - t * (HD / 8), p = t0 + t;
+            uint4 kq = make_uint4(0, 0, 0, 0), vq = kq;
+            if (p <= pos_max) {
+                const int sc = ch ^ (p & c.kv_swz);   // stored chunk of logical chunk ch
+                kq = *reinterpret_cast<const uint4 *>(pool + kv_index(c, seq, layer, 0, kvh, p) + sc * 8);
+                vq = *reinterpret_cast<const uint4 *>(pool + kv_index(c, seq, layer, 1, kvh, p) + sc * 8);
+            }
+            *reinterpret_cast<uint4 *>(&sK[t][ch * 8]) = kq;
+            *reinterpret_cast<uint4 *>(&sV[t][ch * 8]) = vq;
+        }
+        __syncthreads();
+        const int tn = min(PF_T, pos - t0 + 1);   // keys of this tile the row may see (causal)
+        for (int t = 0; t < tn; ++t) {
+            float kf[EPL], vf[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) { kf[e] = __bfloat162float(sK[t][lane * EPL + e]); vf[e] = __bfloat162float(sV[t][lane * EPL + e]); }
+#pragma unroll
+            for (int g = 0; g < GROUP; ++g) {
+                float dot = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) dot = fmaf(q[g][e], kf[e], dot);
+                const float sc = warp_sum(dot);
+                const float mn = fmaxf(m[g], sc);
+                const float corr = expf(m[g] - mn), pr = expf(sc - mn);
+                l[g] = l[g] * corr + pr;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) acc[g][e] = acc[g][e] * corr + pr * vf[e];
+                m[g] = mn;
+            }
+        }
+    }
+    if (live) {
+#pragma unroll
+        for (int g = 0; g < GROUP; ++g)
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) c.attn_out[((size_t)r * c.nq + kvh * GROUP + g) * HD + lane * EPL + e] = acc[g][e] / l[g];
+    }
+}
+
 // ------------------------------------------------------------------ SwiGLU
 
 __global__ void k_swiglu(Ctx c, int layer) {

@@ -335,3 +335,40 @@ def test_a_wait_that_runs_out_ends_the_call_with_a_timeout_and_the_session_recov
     st = binding.Stats()
     S.prefill(prompt)
     assert np.array_equal(S.adaptive_decode(n, 0.3, cfg.exit_layers, 5, st)[0], ref) and st.early_exits > 0
+
+
+@pytest.mark.parametrize("mk,n_prompt", [(gqa, 200), (hd128, 131), (mha, 77)])
+def test_dense_prompt_pass_matches_the_pass_through_the_decode_path_and_the_oracle(mk, n_prompt):
+    """KV cache <- LM(x): prompts of 32 tokens or more run in blocks of 128 positions through the tcgen05
+    GEMMs.  The cache it leaves and the first token agree with the prompt pass through the decode kernel
+    (eight positions at a time) within the cache's bf16 rounding, and decoding on from it matches the oracle."""
+    cfg = mk()
+    pair = Pair(cfg)
+    prompt = synth.make_prompt(cfg, n=n_prompt).numpy()
+    n = 12
+    D = session(pair, max_seq=n_prompt + 64)
+    D.capture_logits(n + 4)
+    D.prefill(prompt)                     # dense (the default)
+    C = session(pair, max_seq=n_prompt + 64)
+    C.set_prefill(False)
+    C.prefill(prompt)
+    ld, fd = D.state()
+    lc, fc = C.state()
+    assert ld == lc == n_prompt + 1 and np.array_equal(fd, fc)
+    O = pair.cpu()
+    O.prefill(prompt)
+    for l in range(cfg.n_layers):
+        for pos in (0, 1, 63, 64, 127, 128, n_prompt - 1):
+            if pos >= n_prompt:
+                continue
+            for which in (0, 1):
+                a, b, ref = D.read_kv(which, l, pos), C.read_kv(which, l, pos), O.kv(which, l, pos)
+                scale = max(1.0, np.abs(ref).max())
+                assert np.abs(a - ref).max() <= 2e-2 * scale and np.abs(a - b).max() <= 2e-2 * scale
+    out = D.plain_decode(n)[0]
+    check_against_oracle(pair, prompt, out, D.captured_logits().cpu().numpy())
+    # adaptive decoding on top of a dense prompt pass equals plain decoding on top of one, bit for bit
+    A = session(pair, max_seq=n_prompt + 64)
+    A.prefill(prompt)
+    st = binding.Stats()
+    assert np.array_equal(A.adaptive_decode(n, 0.3, cfg.exit_layers, 5, st)[0], out) and st.early_exits > 0
