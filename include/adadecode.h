@@ -188,11 +188,13 @@ int ada_debug_read_kv(ada_session *s, int32_t seq, int32_t which, int32_t layer0
 int ada_debug_profile(ada_session *s, int32_t on);
 int ada_debug_profile_read(ada_session *s, double *ms_out, int64_t *launches_out, double *bytes_out);
 /* Select the decode path: 1 = the persistent kernel (one cooperative launch runs many steps of
- * Algorithm 1; bf16 models, one sequence, at most 8 tokens per pass, 64-token KV pages, head_dim 64
+ * Algorithm 1; bf16 models, at most 8 tokens per pass, 64-token KV pages, head_dim 64
  * or 128, at most 4 q heads per kv head, d_model / n_q_heads*head_dim / d_ff multiples of 64); it is
  * the default wherever a session qualifies; a session that qualifies but cannot be set up fails in
  * ada_session_create instead of taking the other path).  0 = one kernel per operation on CUDA cores
- * (any dtype, any batch).  ADA_EUNSUPPORTED if path 1 is asked of a session that does not qualify.
+ * (any dtype, any batch; sequences of a batch share every layer pass).  On path 1 the sequences of a batch are
+ * decoded one after another, each streaming the weights for itself.  ADA_EUNSUPPORTED if path 1 is asked of a
+ * session that does not qualify.
  * ada_stats.path reports the path a decode call ran on. */
 int ada_debug_set_path(ada_session *s, int32_t path);
 int ada_debug_get_path(ada_session *s, int32_t *path_out);

@@ -357,11 +357,12 @@ int run_layer_dense(ada_session *S, int layer, int rows) {
     S->launches++;
     {
         Prof pf(S, 4, 0.0);
-        const dim3 grid((rows + PF_Q - 1) / PF_Q, g.n_kv_heads);
         const int group = g.n_q_heads / g.n_kv_heads;
-#define PF_ATTN(E, G) k_pf_attn<E, G><<<grid, PF_Q * 32, 0, S->stream>>>(S->c, layer, rows)
-        if (hd == 128) { if (group == 4) PF_ATTN(4, 4); else if (group == 2) PF_ATTN(4, 2); else if (group == 1) PF_ATTN(4, 1); else return ADA_EUNSUPPORTED; }
-        else if (hd == 64) { if (group == 4) PF_ATTN(2, 4); else if (group == 2) PF_ATTN(2, 2); else if (group == 1) PF_ATTN(2, 1); else return ADA_EUNSUPPORTED; }
+        if (group != 1 && group != 2 && group != 4) return ADA_EUNSUPPORTED;
+        const dim3 grid((rows + 64 / group - 1) / (64 / group), g.n_kv_heads);   // four warps of 16 / group positions each
+#define PF_ATTN(H, G) dg::k_pf_attn_mma<H, G><<<grid, 128, 0, S->stream>>>(S->c, layer, rows)
+        if (hd == 128) { if (group == 4) PF_ATTN(128, 4); else if (group == 2) PF_ATTN(128, 2); else PF_ATTN(128, 1); }
+        else if (hd == 64) { if (group == 4) PF_ATTN(64, 4); else if (group == 2) PF_ATTN(64, 2); else PF_ATTN(64, 1); }
         else return ADA_EUNSUPPORTED;
 #undef PF_ATTN
     }
@@ -600,7 +601,7 @@ template <int HD> const void *persistent_kernel() { return (const void *)mg::k_d
 const void *persistent_kernel_for(int hd) { return hd == 64 ? persistent_kernel<64>() : persistent_kernel<128>(); }
 
 // Whether a model's shape and dtype are ones the persistent kernel is built for (the session adds its
-// own conditions: one sequence, at most eight token columns, 64-token pages).
+// own conditions: at most eight token columns per sequence, 64-token pages).
 bool model_fits_persistent(const ada_config &g) {
     const int qd = g.n_q_heads * g.head_dim, group = g.n_q_heads / g.n_kv_heads;
     if (g.dtype != ADA_DTYPE_BF16) return false;
@@ -620,7 +621,7 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     S->mega = false;
     S->path = 0;
     const int qd = g.n_q_heads * g.head_dim;
-    if (!model_fits_persistent(g) || S->batch != 1 || S->slots > st::MAX_COLS || S->page_tokens != mg::ATT_PAGE) return ADA_OK;
+    if (!model_fits_persistent(g) || S->slots > st::MAX_COLS || S->page_tokens != mg::ATT_PAGE) return ADA_OK;
     int dev = 0, sms = 0, coop = 0, nb = 0;
     CK(cudaGetDevice(&dev));
     CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
@@ -692,6 +693,7 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.pub = (mg::Pub *)(b + lay.pub);
     a.err = (int *)(b + lay.err);
     a.step_budget = S->steps_per_launch;
+    a.seq = 0;
     a.wait_ns = S->wait_ns;
     a.store_logits = 0;
     a.trace = st::Trace{nullptr, nullptr, 0};
@@ -702,7 +704,9 @@ int setup_persistent(ada_session *S, const Layout &lay) {
 }
 
 // Run the persistent kernel until the call's token targets are met.
-int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool plain) {
+// Sequences of a batch are decoded one after another, each by launches of its own (seq0 .. seq1 - 1): the kernel holds
+// one sequence's token columns at a time.
+int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool plain, int seq0, int seq1) {
     const ada_model *m = S->m;
     const ada_config &g = m->cfg;
     const int L = g.n_layers;
@@ -731,29 +735,36 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
     CK(cudaMemsetAsync(S->margs.attn_cnt, 0, sizeof(unsigned) * g.n_kv_heads, S->stream));
     CK(cudaStreamSynchronize(S->stream));   // ex and the maps live on the host until copied
     S->syncs++;
-    mg::MegaArgs a = S->margs;
-    a.c = S->c;   // capture pointers may have changed
-    a.step_budget = S->steps_per_launch;
-    a.wait_ns = S->wait_ns;
-    a.store_logits = S->capture_dev ? 1 : 0;
     const void *kern = persistent_kernel_for(g.head_dim);
-    for (long long guard = 0;; ++guard) {
-        if (guard > (1ll << 24)) return ADA_ETIMEOUT;
-        CK(cudaMemsetAsync(a.grid_ctr, 0, sizeof(unsigned), S->stream));
-        CK(cudaMemsetAsync(a.pub, 0, sizeof(mg::Pub) * 2, S->stream));
-        if (a.part) CK(cudaMemsetAsync(a.part, 0, kPartBytesPerCta * (size_t)S->grid, S->stream));
-        void *params[] = {(void *)&a};
-        CK(cudaLaunchCooperativeKernel(kern, dim3(S->grid), dim3(st::THREADS), params, st::SMEM_BYTES, S->stream));
-        S->launches++;
-        CK(cudaMemcpyAsync(S->pinned, &S->c.st->n_climbing, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
-        CK(cudaMemcpyAsync(S->pinned + 2, a.err, sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
-        CK(cudaStreamSynchronize(S->stream));
-        S->syncs++;
-        if (S->pinned[2] != 0) {
-            g_cuda_err = "persistent decode kernel: device-side error " + std::to_string(S->pinned[2]);
-            return S->pinned[2] == mg::ERR_BAD_STATE ? ADA_ESTATE : ADA_ETIMEOUT;
+    for (int sq = seq0; sq < seq1; ++sq) {
+        mg::MegaArgs a = S->margs;
+        a.c = S->c;   // capture pointers may have changed
+        a.c.tokens = S->c.tokens + (size_t)sq * S->max_seq;
+        a.c.fill = S->c.fill + (size_t)sq * L;
+        a.c.page_table = S->c.page_table + (size_t)sq * S->max_pages;
+        a.seq = sq;
+        a.step_budget = S->steps_per_launch;
+        a.wait_ns = S->wait_ns;
+        a.store_logits = (S->capture_dev && sq == 0) ? 1 : 0;
+        CK(cudaMemsetAsync(&S->c.st->n_done, 0, sizeof(int32_t), S->stream));
+        for (long long guard = 0;; ++guard) {
+            if (guard > (1ll << 24)) return ADA_ETIMEOUT;
+            CK(cudaMemsetAsync(a.grid_ctr, 0, sizeof(unsigned), S->stream));
+            CK(cudaMemsetAsync(a.pub, 0, sizeof(mg::Pub) * 2, S->stream));
+            if (a.part) CK(cudaMemsetAsync(a.part, 0, kPartBytesPerCta * (size_t)S->grid, S->stream));
+            void *params[] = {(void *)&a};
+            CK(cudaLaunchCooperativeKernel(kern, dim3(S->grid), dim3(st::THREADS), params, st::SMEM_BYTES, S->stream));
+            S->launches++;
+            CK(cudaMemcpyAsync(S->pinned, &S->c.st->n_climbing, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+            CK(cudaMemcpyAsync(S->pinned + 2, a.err, sizeof(int32_t), cudaMemcpyDeviceToHost, S->stream));
+            CK(cudaStreamSynchronize(S->stream));
+            S->syncs++;
+            if (S->pinned[2] != 0) {
+                g_cuda_err = "persistent decode kernel: device-side error " + std::to_string(S->pinned[2]);
+                return S->pinned[2] == mg::ERR_BAD_STATE ? ADA_ESTATE : ADA_ETIMEOUT;
+            }
+            if (S->pinned[1] >= 1) break;   // this sequence has reached its target
         }
-        if (S->pinned[1] >= S->batch) break;
     }
     return ADA_OK;
 }
@@ -801,7 +812,7 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
 
     const bool plain = (n_exit == 0 || max_early == 0);
     if (S->mega && S->path == 1) {
-        if ((rc = run_persistent(S, exit_layers, n_exit, plain))) return rc;
+        if ((rc = run_persistent(S, exit_layers, n_exit, plain, 0, S->batch))) return rc;
     } else if (plain) {
         // every step is one token through all layers; the step count is known, no read-back needed
         for (int it = 0; it < max_steps_plain; ++it) {
@@ -1238,9 +1249,11 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
     const bool dense = S->dense_ok && S->prefill_dense && n_prompt >= 32;
     if (!dense && S->mega && S->path == 1) {
         // prompt passes of eight positions through the persistent kernel
-        mg::k_prefill_arm<<<1, 32, 0, S->stream>>>(S->c, n_prompt);
+        Ctx cs = S->c;
+        cs.fill = S->c.fill + (size_t)seq * g.n_layers;
+        mg::k_prefill_arm<<<1, 32, 0, S->stream>>>(cs, seq, n_prompt);
         CK(cudaGetLastError());
-        if ((rc = run_persistent(S, nullptr, 0, true))) return rc;
+        if ((rc = run_persistent(S, nullptr, 0, true, seq, seq + 1))) return rc;
         S->prefilled[seq] = 1;
         S->h_prompt[seq] = n_prompt;
         S->h_len[seq] = n_prompt + 1;

@@ -9,14 +9,15 @@
 // matrices, a high part and a low part (x = hi + lo, as everywhere in this library: fp32 activations
 // lose nothing), both multiplied into the same fp32 accumulator.
 //
-// One CTA computes a tile of 128 positions x 64 weight rows.  Warp 0 is the TMA producer (one k block of
+// One CTA computes a tile of 128 positions x 128 weight rows.  Warp 0 is the TMA producer (one k block of
 // 64 elements per stage: the 128-byte-swizzled tiles of X.hi, X.lo and W), warp 1 allocates the tensor
-// memory and issues the MMAs (one elected thread; UMMA shape M = 128, N = 64, K = 16, both operands
+// memory and issues the MMAs (one elected thread; UMMA shape M = 128, N = 128, K = 16, both operands
 // K-major), warps 2..5 read the accumulator back (tcgen05.ld, 32 lanes per warp) and write it out.
 // Every wait is bounded; on expiry an error word is set, the roles leave their loops, the tensor
 // memory is released and the kernel ends.
 #pragma once
 
+#include "kernels.cuh"
 #include "stream.cuh"
 
 namespace ada {
@@ -25,9 +26,9 @@ namespace dg {
 using namespace st;
 
 constexpr int BM = 128;     // positions per tile (UMMA M)
-constexpr int BN = 64;      // weight rows per tile (UMMA N)
+constexpr int BN = 128;     // weight rows per tile (UMMA N)
 constexpr int BK = 64;      // k elements per stage: one 128-byte swizzle row
-constexpr int STAGES = 5;
+constexpr int STAGES = 4;
 constexpr int DTHREADS = 192;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = 2 * A_BYTES + B_BYTES;
 // The tensor core adds into its fp32 accumulator with truncation, so the error of one accumulator grows in
@@ -38,7 +39,7 @@ constexpr int TMEM_COLS = NACC * BN;   // fp32 accumulator columns (a power of t
 constexpr unsigned long long DENSE_WAIT_NS = 2000000000ull;
 
 struct DSmem {   // must start on a 1024-byte boundary (swizzle pattern)
-    alignas(1024) unsigned char stage[STAGES][STAGE_BYTES];   // [X.hi 128 x 64 | X.lo 128 x 64 | W 64 x 64], rows of 128 B
+    alignas(1024) unsigned char stage[STAGES][STAGE_BYTES];   // [X.hi 128 x 64 | X.lo 128 x 64 | W 128 x 64], rows of 128 B
     alignas(8) unsigned long long full[STAGES], empty[STAGES], acc_full;
     uint32_t tmem_base;
     int abort;
@@ -104,7 +105,7 @@ __device__ __forceinline__ bool dwait(const DWait &w, unsigned long long *bar, u
 // EPI 0: Y[m][n] = acc.  EPI 1: Y[m][n] += acc (every element has one writer).  Rows m >= rows are not written.
 // gridDim.y > 1 splits the depth: block row y multiplies its share of the k blocks and writes (EPI 0) to
 // Y + y * split_stride; k_dense_reduce then adds the shares in a fixed order.
-// mapXhi / mapXlo: 2-D maps over the bf16 matrices [128][K] (box 64 x 128); mapW: over W [N][K] (box 64 x 64);
+// mapXhi / mapXlo: 2-D maps over the bf16 matrices [128][K] (box 64 x 128); mapW: over W [N][K] (box 64 x 128);
 // all 128-byte swizzled, zero fill outside.  K a multiple of 64.
 template <int EPI>
 __global__ void __launch_bounds__(DTHREADS, 1)
@@ -274,6 +275,152 @@ __global__ void k_split_rows(const float *__restrict__ X, int ldx, int rows, int
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         hi[(size_t)r * K + k] = h;
         lo[(size_t)r * K + k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+// Causal attention of a block of prompt rows on the tensor cores (mma.sync m16n8k16, bf16 cache).  One warp owns
+// one 16-row query tile: 16 / GROUP consecutive prompt positions x the GROUP q heads of one kv head; a block of
+// four warps shares the K and V rows of 64 cache positions at a time, copied into shared memory exactly as the
+// cache stores them (16-byte chunks xor-swizzled by position: conflict-free for ldmatrix).  Queries are rotated
+// already (k_rope_kv); they are scaled and split into bf16 high / low parts in registers, the probabilities
+// likewise, so nothing but the cache itself is rounded to bf16.  Online softmax in position order; the context
+// is not split, the result goes straight to attn_out.
+template <int HD, int GROUP>
+__global__ void __launch_bounds__(128) k_pf_attn_mma(Ctx c, int layer, int rows) {
+    constexpr int KSQ = HD / 16, NT = HD / 8, PPW = 16 / GROUP, TILE = 64;
+    __shared__ __align__(128) unsigned char sK[TILE * HD * 2], sV[TILE * HD * 2];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, kvh = blockIdx.y;
+    const int r_blk = blockIdx.x * 4 * PPW, r_w = r_blk + warp * PPW;   // first row of the block / of this warp
+    const int seq = c.rt->seq[0], pos0 = c.rt->pos[0];                   // rows of a prompt block: consecutive positions of one sequence
+    const int pos_blk_max = pos0 + min(r_blk + 4 * PPW, rows) - 1;
+    const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
+    const float scale = rsqrtf((float)HD);
+    // ---- this lane's parts of the query fragments: rows lane/4 and lane/4 + 8 of the tile
+    int lim[2];
+    uint32_t ah[KSQ][4], al[KSQ][4];
+#pragma unroll
+    for (int rh = 0; rh < 2; ++rh) {
+        const int row = (lane >> 2) + 8 * rh, r = r_w + row / GROUP, g = row % GROUP;
+        const bool live = r < rows;
+        lim[rh] = live ? pos0 + r : -1;
+        const float *q = c.q + ((size_t)min(r, rows - 1) * c.nq + kvh * GROUP + g) * HD;
+#pragma unroll
+        for (int ks = 0; ks < KSQ; ++ks)
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                const float2 v = *reinterpret_cast<const float2 *>(q + ks * 16 + kh * 8 + 2 * (lane & 3));
+                const float y0 = live ? v.x * scale : 0.f, y1 = live ? v.y * scale : 0.f;
+                const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
+                const __nv_bfloat162 l = __floats2bfloat162_rn(y0 - __low2float(h), y1 - __high2float(h));
+                ah[ks][rh + 2 * kh] = *reinterpret_cast<const uint32_t *>(&h);
+                al[ks][rh + 2 * kh] = *reinterpret_cast<const uint32_t *>(&l);
+            }
+    }
+    const int lim_w = r_w < rows ? pos0 + min(r_w + PPW, rows) - 1 : -1;   // last position any row of this warp sees (the same in every lane)
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float o[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[nt][i] = 0.f;
+    for (int t0 = 0; t0 <= pos_blk_max; t0 += TILE) {
+        __syncthreads();   // the previous tile has been used
+        for (int i = threadIdx.x; i < TILE * (HD / 8); i += 128) {
+            const int t = i / (HD / 8), ch = i - t * (HD / 8), p = t0 + t;
+            uint4 kq = make_uint4(0, 0, 0, 0), vq = kq;
+            if (p <= pos_blk_max) {
+                kq = *reinterpret_cast<const uint4 *>(pool + kv_index(c, seq, layer, 0, kvh, p) + ch * 8);
+                vq = *reinterpret_cast<const uint4 *>(pool + kv_index(c, seq, layer, 1, kvh, p) + ch * 8);
+            }
+            *reinterpret_cast<uint4 *>(sK + (size_t)t * HD * 2 + ch * 16) = kq;
+            *reinterpret_cast<uint4 *>(sV + (size_t)t * HD * 2 + ch * 16) = vq;
+        }
+        __syncthreads();
+        for (int sl = 0; sl < TILE / 16; ++sl) {
+            const int p0 = t0 + 16 * sl;
+            if (p0 > lim_w) break;   // nothing further in this tile is visible to this warp (uniform per warp)
+            // ---- scores of the 16 positions p0 .. p0 + 15
+            float sh[2][4], sl_[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { sh[nt][i] = 0.f; sl_[nt][i] = 0.f; }
+            const int id = lane >> 3;
+            {
+                const int pl = 16 * sl + (lane & 7) + 8 * (id >> 1);
+                const unsigned char *krow = sK + pl * (HD * 2);
+#pragma unroll
+                for (int ks = 0; ks < KSQ; ++ks) {
+                    uint32_t kf[4];
+                    ldmatrix_x4(kf, krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
+                    mma16816(sh[0], ah[ks], kf[0], kf[1]);
+                    mma16816(sh[1], ah[ks], kf[2], kf[3]);
+                    mma16816(sl_[0], al[ks], kf[0], kf[1]);
+                    mma16816(sl_[1], al[ks], kf[2], kf[3]);
+                }
+            }
+            float s[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int pos = p0 + 8 * nt + 2 * (lane & 3) + (i & 1);
+                    s[nt][i] = pos <= lim[i >> 1] ? sh[nt][i] + sl_[nt][i] : -INFINITY;
+                }
+            // ---- online softmax
+            uint32_t ph[4], plo[4];
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                float mx = fmaxf(fmaxf(s[0][2 * rh], s[0][2 * rh + 1]), fmaxf(s[1][2 * rh], s[1][2 * rh + 1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float mn = fmaxf(m_run[rh], mx);
+                float corr = 1.f, p[4] = {0.f, 0.f, 0.f, 0.f};
+                if (mn != -INFINITY) {
+                    corr = __expf(m_run[rh] - mn);
+                    p[0] = __expf(s[0][2 * rh] - mn); p[1] = __expf(s[0][2 * rh + 1] - mn);
+                    p[2] = __expf(s[1][2 * rh] - mn); p[3] = __expf(s[1][2 * rh + 1] - mn);
+                }
+                m_run[rh] = mn;
+                l_run[rh] = l_run[rh] * corr + ((p[0] + p[1]) + (p[2] + p[3]));
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) { o[nt][2 * rh] *= corr; o[nt][2 * rh + 1] *= corr; }
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
+                const __nv_bfloat162 l0 = __floats2bfloat162_rn(p[0] - __low2float(h0), p[1] - __high2float(h0));
+                const __nv_bfloat162 l1 = __floats2bfloat162_rn(p[2] - __low2float(h1), p[3] - __high2float(h1));
+                ph[rh] = *reinterpret_cast<const uint32_t *>(&h0);
+                ph[2 + rh] = *reinterpret_cast<const uint32_t *>(&h1);
+                plo[rh] = *reinterpret_cast<const uint32_t *>(&l0);
+                plo[2 + rh] = *reinterpret_cast<const uint32_t *>(&l1);
+            }
+            // ---- o += P V
+            {
+                const int pl = 16 * sl + (lane & 7) + 8 * (id & 1);
+                const unsigned char *vrow = sV + pl * (HD * 2);
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) {
+                    uint32_t vf[4];
+                    ldmatrix_x4_trans(vf, vrow + ((((2 * np) | (id >> 1)) ^ (pl & 7)) << 4));
+                    mma16816(o[2 * np], ph, vf[0], vf[1]);
+                    mma16816(o[2 * np + 1], ph, vf[2], vf[3]);
+                    mma16816(o[2 * np], plo, vf[0], vf[1]);
+                    mma16816(o[2 * np + 1], plo, vf[2], vf[3]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int rh = 0; rh < 2; ++rh) {
+        l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 1);
+        l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 2);
+        const int row = (lane >> 2) + 8 * rh, r = r_w + row / GROUP, g = row % GROUP;
+        if (r < rows) {
+            float *out = c.attn_out + ((size_t)r * c.nq + kvh * GROUP + g) * HD;
+            const float inv = 1.0f / l_run[rh];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+                *reinterpret_cast<float2 *>(out + nt * 8 + 2 * (lane & 3)) = make_float2(o[nt][2 * rh] * inv, o[nt][2 * rh + 1] * inv);
+        }
     }
 }
 

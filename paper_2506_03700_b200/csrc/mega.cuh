@@ -84,6 +84,7 @@ struct MegaArgs {
     Pub *pub;                  // [2]
     int *err;
     int step_budget;           // steps this launch may start
+    int seq;                   // the sequence of the session this launch decodes (c.tokens, c.fill and c.page_table point at its rows)
     unsigned long long wait_ns;   // a single device-side wait gives up after this long
     int store_logits;
     Trace trace;               // test hook: event trace of the steps [trace_step0, trace_step1) of this launch
@@ -184,7 +185,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     const Ctx &c = A.c;
     DevState *st = c.st;
     const MegaModel &M = *A.mm;
-    const int tid = threadIdx.x, G = gridDim.x;
+    const int tid = threadIdx.x, G = gridDim.x, sq = A.seq;
     Pub *pub = A.pub + (pub_no & 1);
     // Shared-memory copies for the bookkeeping thread (fetched by many threads at once: a single
     // thread reading them from global memory one after the other spent 30 us here on round trips to L2):
@@ -194,7 +195,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     int *tok_s = reinterpret_cast<int *>(sm->scratch + 1024 + sizeof(HeadResult) * MAX_COLS);   // [MAX_COLS]: tokens base+1 ..
     for (int l = tid; l < c.L; l += CONS_THREADS) fill_s[l] = c.fill[l];
     if (tid >= CONS_THREADS - MAX_COLS) {
-        const int j = tid - (CONS_THREADS - MAX_COLS), at = st->base[0] + j + 1;
+        const int j = tid - (CONS_THREADS - MAX_COLS), at = st->base[sq] + j + 1;
         tok_s[j] = at < c.max_seq ? c.tokens[at] : -1;
     }
     // (a) head results of the columns that matter: warp w merges column w
@@ -213,7 +214,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     if (tid == 0) {
         auto bump = [](long long *p, long long v) { atomicAdd(reinterpret_cast<unsigned long long *>(p), (unsigned long long)v); };
         const int err0 = *(volatile int *)A.err;
-        const int len0 = st->len[0], base0 = st->base[0], target0 = st->target_len[0], done0 = st->done[0];
+        const int len0 = st->len[sq], base0 = st->base[sq], target0 = st->target_len[sq], done0 = st->done[sq];
         const int pf_end0 = st->pf_end, pf_pos0 = st->pf_pos, max_early0 = st->max_early;
         const int tape_n0 = st->tape_n, tape_i0 = st->tape_i, hl_n0 = st->head_log_n;
         const float gamma0 = st->gamma;
@@ -226,14 +227,14 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
         if (action != ACT_STOP && kind == CTRL_HEAD) {
             const HeadResult hr = hr_s[dprev.newest];
             bool decide = hr.p > gamma0;
-            if (tape_i0 < tape_n0) {
+            if (sq == 0 && tape_i0 < tape_n0) {
                 const uint8_t t = st->tape[tape_i0];
                 st->tape_i = tape_i0 + 1;
                 if (t == 0) decide = false;
                 if (t == 1) decide = true;
             }
             bump(&st->st.head_evals, 1);
-            if (c.head_log && hl_n0 < kHeadLogCap) {
+            if (sq == 0 && c.head_log && hl_n0 < kHeadLogCap) {
                 float *hl = c.head_log + 4 * (size_t)hl_n0;
                 hl[0] = (float)steps0; hl[1] = (float)e; hl[2] = (float)hr.token; hl[3] = hr.p;
                 st->head_log_n = hl_n0 + 1;
@@ -249,7 +250,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
                 bump(&st->st.row_layers, rl);
                 tok[len] = min(max(hr.token, 0), c.vocab - 1);
                 len = len + 1;
-                st->len[0] = len;
+                st->len[sq] = len;
                 bump(&st->st.early_exits, 1);
                 bump(&st->st.exits_at_layer[e], 1);
                 bump(&st->st.steps, 1);
@@ -267,10 +268,10 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
                 const int np = pf_end;
                 tok[np] = min(max(hr_s[n - 1].token, 0), c.vocab - 1);
                 len = np + 1; base = np; done = 1; pf_end = 0;
-                st->len[0] = len;
-                st->base[0] = base;
-                st->n_prompt[0] = np;
-                st->done[0] = 1;
+                st->len[sq] = len;
+                st->base[sq] = base;
+                st->n_prompt[sq] = np;
+                st->done[sq] = 1;
                 st->pf_end = 0;
                 st->keep_rows = 1;
                 st->keep_row0 = n - 1;
@@ -306,7 +307,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
             if (eos0 >= 0) {
                 for (int j = 0; j < keep; ++j)
                     if (min(max(hr_s[j].token, 0), c.vocab - 1) == eos0) {
-                        if (base + j + 2 <= target) { target = base + j + 2; st->eos_hit[0] = 1; }
+                        if (base + j + 2 <= target) { target = base + j + 2; st->eos_hit[sq] = 1; }
                         break;
                     }
             }
@@ -319,12 +320,12 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
             keep = new_len - 1 - base;   // verified tokens that stay: their logit rows are the ones a capture keeps
             for (int l = 0; l < c.L; ++l) { fill_s[l] = new_base; c.fill[l] = new_base; }
             len = new_len; base = new_base;
-            st->len[0] = len;
-            st->base[0] = base;
+            st->len[sq] = len;
+            st->base[sq] = base;
             bump(&st->st.verify_steps, 1);
             bump(&st->st.steps, 1);
             bump(&st->st.layer_passes, c.L);
-            if (new_len >= target) { done = 1; st->done[0] = 1; }
+            if (new_len >= target) { done = 1; st->done[sq] = 1; }
             st->keep_rows = keep;
             st->keep_row0 = 0;
             verified = 1;
@@ -383,7 +384,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     bar_consumers();
     const int action = sm->bcast[0];
     // (c) logits of the verified rows (test hook), then the embedding of the next newest token
-    if (kind == CTRL_TOP && c.capture && sm->bcast[3]) {
+    if (sq == 0 && kind == CTRL_TOP && c.capture && sm->bcast[3]) {
         const int keep = st->keep_rows, at = st->capture_n;
         for (int j = 0; j < keep && at + j < st->capture_cap; ++j) {
             const float *src = c.logit_stage + (size_t)(st->keep_row0 + j) * c.vocab;
@@ -1283,16 +1284,17 @@ __global__ void k_repack_qkv(const __nv_bfloat16 *__restrict__ wq, const __nv_bf
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) d4[i] = s4[i];
 }
 
-// Arms the prompt passes of the persistent kernel for sequence 0 (KV cache <- LM(x), first line of Algorithm 1).
-__global__ void k_prefill_arm(Ctx c, int n_prompt) {
+// Arms the prompt passes of the persistent kernel for one sequence (KV cache <- LM(x), first line of Algorithm 1);
+// c.fill points at that sequence's fill levels.
+__global__ void k_prefill_arm(Ctx c, int seq, int n_prompt) {
     DevState *st = c.st;
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     st->pf_pos = 0;
     st->pf_end = n_prompt;
-    st->done[0] = 0;
+    st->done[seq] = 0;
     st->n_done = 0;
-    st->len[0] = 0;
-    st->base[0] = 0;
+    st->len[seq] = 0;
+    st->base[seq] = 0;
     st->tape_n = 0;
     st->tape_i = 0;
     for (int l = 0; l < c.L; ++l) c.fill[l] = 0;

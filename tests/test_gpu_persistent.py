@@ -372,3 +372,49 @@ def test_dense_prompt_pass_matches_the_pass_through_the_decode_path_and_the_orac
     A.prefill(prompt)
     st = binding.Stats()
     assert np.array_equal(A.adaptive_decode(n, 0.3, cfg.exit_layers, 5, st)[0], out) and st.early_exits > 0
+
+
+def test_batch_of_ragged_sequences_on_the_persistent_path():
+    """Independent sequences in one session (ragged prompt lengths, one of them long enough for the dense prompt
+    pass): each equals its own single-sequence run bit for bit, plain and adaptive, with and without an
+    end-of-sequence token."""
+    cfg = gqa()
+    pair = Pair(cfg)
+    lens = [5, 19, 70]
+    prompts = [synth.make_prompt(cfg, n=n, seq=i).numpy() for i, n in enumerate(lens)]
+    n = 24
+    singles = []
+    for p in prompts:
+        S = session(pair)
+        S.prefill(p)
+        singles.append(S.plain_decode(n)[0])
+    B = binding.Session(pair.gm, 3, 256, 64, 5)
+    assert B.get_path() == 1
+    for i, p in enumerate(prompts):
+        B.prefill(p, seq=i)
+    st = binding.Stats()
+    out = B.plain_decode(n, st)
+    for i in range(3):
+        assert np.array_equal(out[i], singles[i]), i
+    assert st.path == 1 and list(st.emitted[:3]) == [n, n, n]
+    A = binding.Session(pair.gm, 3, 256, 64, 5)
+    for i, p in enumerate(prompts):
+        A.prefill(p, seq=i)
+    st = binding.Stats()
+    a1 = A.adaptive_decode(10, 0.3, cfg.exit_layers, 5, st)
+    a2 = A.adaptive_decode(n - 10, 0.0, cfg.exit_layers, 3, st)
+    assert np.array_equal(np.concatenate([a1, a2], axis=1), out) and st.early_exits > 0
+    for i in range(3):
+        ln, fill = A.state(i)
+        assert ln == lens[i] + n and (fill == lens[i] + n - 1).all()
+    # an end-of-sequence token that only the second sequence meets: the others run on
+    k = next(j for j in range(3, n) if singles[1][j] not in singles[1][:j] and singles[1][j] not in singles[0] and singles[1][j] not in singles[2])
+    eos = int(singles[1][k])
+    E = binding.Session(pair.gm, 3, 256, 64, 5)
+    for i, p in enumerate(prompts):
+        E.prefill(p, seq=i)
+    st = binding.Stats()
+    e = E.adaptive_decode(n, 0.3, cfg.exit_layers, 5, st, eos_id=eos)
+    assert list(st.emitted[:3]) == [n, k + 1, n] and st.finished == 1
+    assert np.array_equal(e[0], singles[0]) and np.array_equal(e[2], singles[2])
+    assert np.array_equal(e[1][:k + 1], singles[1][:k + 1]) and (e[1][k + 1:] == eos).all()
