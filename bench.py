@@ -333,7 +333,8 @@ def run_ours(args):
                                f"{gen_len} greedy tokens each, exits {list(cfg.exit_layers)}, gamma {cfg.threshold}, "
                                f"tied head logit scale {cfg.logit_scale}, max_early 5, o/down scale {cfg.resid_scale}",
                    "tokens_per_step": sizes[0], "last_step_tokens": sizes[-1], "l2": "inputs_larger_than_l2 (weights stream >> 126 MB)",
-                   "decode_path": "persistent kernel" if path == 1 else "one kernel per operation",
+                   "decode_path": ("persistent kernel" + (", sequences decoded one after another (each streams the weights for itself)"
+                                                           if cfg.batch > 1 else "")) if path == 1 else "one kernel per operation",
                    "parallelism": "replicas" if world > 1 else "single"},
         "e2e": {"value": whole_job_tokens_per_s(n_tok, world, a_wall), "unit": UNIT,
                 "h2d_bytes_per_step": int(64 + 4 * 16 + 4 * len(cfg.exit_layers)),
