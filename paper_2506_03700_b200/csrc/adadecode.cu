@@ -238,7 +238,7 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
         L.ssq_a = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
         L.ssq_b = take(sizeof(float) * (size_t)((g.d_model + 15) / 16) * st::MAX_COLS);
         L.qfrag = take((size_t)g.n_kv_heads * 2 * (g.head_dim / 16) * 1024);
-        L.attn_cnt = take(sizeof(unsigned) * g.n_kv_heads);
+        L.attn_cnt = take(sizeof(unsigned) * g.n_kv_heads * st::MAX_COLS);   // per (sequence of a launch, kv head)
         L.rope_freq = take(sizeof(double) * (g.head_dim / 2));
         L.part = take(kPartBytesPerCta * kPartMaxGrid);
         L.grid_ctr = take(256);
@@ -693,7 +693,8 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.pub = (mg::Pub *)(b + lay.pub);
     a.err = (int *)(b + lay.err);
     a.step_budget = S->steps_per_launch;
-    a.seq = 0;
+    a.seq0 = 0;
+    a.nseq = 1;
     a.wait_ns = S->wait_ns;
     a.store_logits = 0;
     a.trace = st::Trace{nullptr, nullptr, 0};
@@ -704,9 +705,11 @@ int setup_persistent(ada_session *S, const Layout &lay) {
 }
 
 // Run the persistent kernel until the call's token targets are met.
-// Sequences of a batch are decoded one after another, each by launches of its own (seq0 .. seq1 - 1): the kernel holds
-// one sequence's token columns at a time.
-int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool plain, int seq0, int seq1) {
+// The kernel holds eight token columns.  A sequence needs max_early + 1 of them, so a launch decodes
+// min(8 / (max_early + 1), batch) sequences together (one weight stream for all of them, lock-step: every step runs
+// up to the highest layer any of them reaches); the sequences seq_begin .. seq_end - 1 go in such groups, one group
+// after another.  `together` false: one sequence per launch (prompt passes, which use all eight columns).
+int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool plain, int seq_begin, int seq_end, bool together) {
     const ada_model *m = S->m;
     const ada_config &g = m->cfg;
     const int L = g.n_layers;
@@ -732,17 +735,16 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
     CK(cudaMemcpyAsync(S->exit_at_dev, ex.data(), sizeof(int) * (L + 1), cudaMemcpyHostToDevice, S->stream));
     // a call that ended on a device-side error may have left the error word and the attention counters set
     CK(cudaMemsetAsync(S->margs.err, 0, sizeof(int), S->stream));
-    CK(cudaMemsetAsync(S->margs.attn_cnt, 0, sizeof(unsigned) * g.n_kv_heads, S->stream));
+    CK(cudaMemsetAsync(S->margs.attn_cnt, 0, sizeof(unsigned) * g.n_kv_heads * st::MAX_COLS, S->stream));
     CK(cudaStreamSynchronize(S->stream));   // ex and the maps live on the host until copied
     S->syncs++;
     const void *kern = persistent_kernel_for(g.head_dim);
-    for (int sq = seq0; sq < seq1; ++sq) {
+    const int per_launch = together ? std::max(1, st::MAX_COLS / S->slots) : 1;
+    for (int sq = seq_begin; sq < seq_end; sq += per_launch) {
         mg::MegaArgs a = S->margs;
         a.c = S->c;   // capture pointers may have changed
-        a.c.tokens = S->c.tokens + (size_t)sq * S->max_seq;
-        a.c.fill = S->c.fill + (size_t)sq * L;
-        a.c.page_table = S->c.page_table + (size_t)sq * S->max_pages;
-        a.seq = sq;
+        a.seq0 = sq;
+        a.nseq = std::min(per_launch, seq_end - sq);
         a.step_budget = S->steps_per_launch;
         a.wait_ns = S->wait_ns;
         a.store_logits = (S->capture_dev && sq == 0) ? 1 : 0;
@@ -763,7 +765,7 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
                 g_cuda_err = "persistent decode kernel: device-side error " + std::to_string(S->pinned[2]);
                 return S->pinned[2] == mg::ERR_BAD_STATE ? ADA_ESTATE : ADA_ETIMEOUT;
             }
-            if (S->pinned[1] >= 1) break;   // this sequence has reached its target
+            if (S->pinned[1] >= 1) break;   // the sequences of this launch have reached their targets
         }
     }
     return ADA_OK;
@@ -812,7 +814,7 @@ int decode(ada_session *S, int n_tokens, float gamma, const int32_t *exit_layers
 
     const bool plain = (n_exit == 0 || max_early == 0);
     if (S->mega && S->path == 1) {
-        if ((rc = run_persistent(S, exit_layers, n_exit, plain, 0, S->batch))) return rc;
+        if ((rc = run_persistent(S, exit_layers, n_exit, plain, 0, S->batch, true))) return rc;
     } else if (plain) {
         // every step is one token through all layers; the step count is known, no read-back needed
         for (int it = 0; it < max_steps_plain; ++it) {
@@ -1249,11 +1251,9 @@ int ada_prefill(ada_session *S, int32_t seq, const int32_t *prompt_host, int32_t
     const bool dense = S->dense_ok && S->prefill_dense && n_prompt >= 32;
     if (!dense && S->mega && S->path == 1) {
         // prompt passes of eight positions through the persistent kernel
-        Ctx cs = S->c;
-        cs.fill = S->c.fill + (size_t)seq * g.n_layers;
-        mg::k_prefill_arm<<<1, 32, 0, S->stream>>>(cs, seq, n_prompt);
+        mg::k_prefill_arm<<<1, 32, 0, S->stream>>>(S->c, seq, n_prompt);
         CK(cudaGetLastError());
-        if ((rc = run_persistent(S, nullptr, 0, true, seq, seq + 1))) return rc;
+        if ((rc = run_persistent(S, nullptr, 0, true, seq, seq + 1, false))) return rc;
         S->prefilled[seq] = 1;
         S->h_prompt[seq] = n_prompt;
         S->h_len[seq] = n_prompt + 1;

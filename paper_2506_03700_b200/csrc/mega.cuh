@@ -34,15 +34,17 @@ constexpr int ATT_CHUNK = kAttnChunk; // positions per attention work item (fixe
 constexpr int ERR_BAD_STATE = 3;
 
 struct StepDesc {
-    int n_cols;                // columns with a token (in flight + newest)
-    int newest;                // column of the newest token
-    int head_ok;               // the newest token may consult intermediate heads in this step
-    int pmax;                  // position of the newest token
+    int n_cols;                // columns with a token (in flight + newest, over all sequences of the launch)
+    int newest_mask;           // columns holding the newest token of their sequence
+    int head_mask;             // newest columns that may consult intermediate heads in this step
+    int pmax;                  // highest position of the step
     int fresh;                 // columns whose token enters at layer 1 in this step (their embedding is set up by the control point)
     int run_final;             // the step ends with the final head (0: a prompt pass that is not the last)
-    int first_layer[MAX_COLS]; // 0-based layer at which the column resumes (INT_MAX: no token)
+    int first_layer[MAX_COLS]; // 0-based layer at which the column resumes (INT_MAX: no token, or its sequence has left the step)
     int pos[MAX_COLS];
+    int seq_pmax[MAX_COLS];    // per sequence of the launch: position of its newest token (-1: the sequence is not in this step)
 };
+static_assert(sizeof(StepDesc) <= 32 * sizeof(int), "the step descriptor must fit its shared-memory slot");
 
 struct Pub {                   // what CTA 0 publishes at a control point
     unsigned seq;
@@ -84,7 +86,8 @@ struct MegaArgs {
     Pub *pub;                  // [2]
     int *err;
     int step_budget;           // steps this launch may start
-    int seq;                   // the sequence of the session this launch decodes (c.tokens, c.fill and c.page_table point at its rows)
+    int seq0, nseq;            // the launch decodes sequences seq0 .. seq0 + nseq - 1 of the session together: sequence k of them owns the
+                               // token columns [k slots, (k + 1) slots), slots = max_early + 1, nseq slots <= 8; they share every weight stream
     unsigned long long wait_ns;   // a single device-side wait gives up after this long
     int store_logits;
     Trace trace;               // test hook: event trace of the steps [trace_step0, trace_step1) of this launch
@@ -185,24 +188,32 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     const Ctx &c = A.c;
     DevState *st = c.st;
     const MegaModel &M = *A.mm;
-    const int tid = threadIdx.x, G = gridDim.x, sq = A.seq;
+    const int tid = threadIdx.x, G = gridDim.x;
+    const int nseq = A.nseq, seq0 = A.seq0, cps = c.slots, L = c.L;   // cps: token columns per sequence
     Pub *pub = A.pub + (pub_no & 1);
     // Shared-memory copies for the bookkeeping thread (fetched by many threads at once: a single
     // thread reading them from global memory one after the other spent 30 us here on round trips to L2):
     // the fill levels, the head results, and the tokens the verification compares with.
-    int *fill_s = reinterpret_cast<int *>(sm->scratch);                                // [L]
-    HeadResult *hr_s = reinterpret_cast<HeadResult *>(sm->scratch + 1024);             // [MAX_COLS]
-    int *tok_s = reinterpret_cast<int *>(sm->scratch + 1024 + sizeof(HeadResult) * MAX_COLS);   // [MAX_COLS]: tokens base+1 ..
-    for (int l = tid; l < c.L; l += CONS_THREADS) fill_s[l] = c.fill[l];
+    int *fill_s = reinterpret_cast<int *>(sm->scratch);                                          // [nseq][L]
+    HeadResult *hr_s = reinterpret_cast<HeadResult *>(sm->scratch + 8192);                       // [MAX_COLS]
+    int *tok_s = reinterpret_cast<int *>(sm->scratch + 8192 + sizeof(HeadResult) * MAX_COLS);    // [MAX_COLS]: the token after the column's own
+    static_assert(ADA_MAX_LAYERS * MAX_COLS * sizeof(int) <= 8192, "fill levels of a launch's sequences must fit the scratch corner");
+    for (int i = tid; i < nseq * L; i += CONS_THREADS) fill_s[i] = c.fill[(size_t)seq0 * L + i];
     if (tid >= CONS_THREADS - MAX_COLS) {
-        const int j = tid - (CONS_THREADS - MAX_COLS), at = st->base[sq] + j + 1;
-        tok_s[j] = at < c.max_seq ? c.tokens[at] : -1;
+        const int j = tid - (CONS_THREADS - MAX_COLS), k = j / cps;
+        int v = -1;
+        if (k < nseq) {
+            const int at = st->base[seq0 + k] + (j - k * cps) + 1;
+            if (at < c.max_seq) v = c.tokens[(size_t)(seq0 + k) * c.max_seq + at];
+        }
+        tok_s[j] = v;
     }
     // (a) head results of the columns that matter: warp w merges column w
+    const unsigned head_cols = kind == CTRL_HEAD ? ((unsigned)dprev.head_mask & active_mask(dprev, e - 1))
+                                                 : (kind == CTRL_TOP ? active_mask(dprev, L - 1) : 0u);
     if (kind != CTRL_START) {
         const int w = tid >> 5;
-        const bool want = kind == CTRL_HEAD ? w == dprev.newest : w < dprev.n_cols;
-        if (want) {
+        if ((head_cols >> w) & 1u) {
             const HeadResult hr = merge_head(A.head_part, G, w);
             if ((tid & 31) == 0) { c.head_res[w] = hr; hr_s[w] = hr; }
         }
@@ -214,169 +225,197 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     if (tid == 0) {
         auto bump = [](long long *p, long long v) { atomicAdd(reinterpret_cast<unsigned long long *>(p), (unsigned long long)v); };
         const int err0 = *(volatile int *)A.err;
-        const int len0 = st->len[sq], base0 = st->base[sq], target0 = st->target_len[sq], done0 = st->done[sq];
         const int pf_end0 = st->pf_end, pf_pos0 = st->pf_pos, max_early0 = st->max_early;
-        const int tape_n0 = st->tape_n, tape_i0 = st->tape_i, hl_n0 = st->head_log_n;
+        const int tape_n0 = st->tape_n, hl_n0 = st->head_log_n;
+        int tape_i = st->tape_i, hl_n = hl_n0;
         const float gamma0 = st->gamma;
         const int eos0 = st->eos_id;
         const long long steps0 = __ldcg(&st->st.steps);   // past the L1: the counters are bumped by reductions
+        int len[MAX_COLS], base[MAX_COLS], target[MAX_COLS], done[MAX_COLS];
+#pragma unroll
+        for (int k = 0; k < MAX_COLS; ++k) {
+            const bool in = k < nseq;
+            len[k] = in ? st->len[seq0 + k] : 0; base[k] = in ? st->base[seq0 + k] : 0;
+            target[k] = in ? st->target_len[seq0 + k] : 0; done[k] = in ? st->done[seq0 + k] : 1;
+        }
         int action = ACT_NEWSTEP, verified = 0;
-        int len = len0, base = base0, done = done0, pf_end = pf_end0, pf_pos = pf_pos0;
-        int32_t *tok = c.tokens;
+        int pf_end = pf_end0, pf_pos = pf_pos0;
+        StepDesc nd = dprev;
         if (err0 != 0) action = ACT_STOP;
+        // ---- Eq. 1 after an intermediate head: every sequence whose newest token consulted it decides for itself
         if (action != ACT_STOP && kind == CTRL_HEAD) {
-            const HeadResult hr = hr_s[dprev.newest];
-            bool decide = hr.p > gamma0;
-            if (sq == 0 && tape_i0 < tape_n0) {
-                const uint8_t t = st->tape[tape_i0];
-                st->tape_i = tape_i0 + 1;
-                if (t == 0) decide = false;
-                if (t == 1) decide = true;
-            }
-            bump(&st->st.head_evals, 1);
-            if (sq == 0 && c.head_log && hl_n0 < kHeadLogCap) {
-                float *hl = c.head_log + 4 * (size_t)hl_n0;
-                hl[0] = (float)steps0; hl[1] = (float)e; hl[2] = (float)hr.token; hl[3] = hr.p;
-                st->head_log_n = hl_n0 + 1;
-            }
-            if (!decide) action = ACT_CONTINUE;
-            else {
+            unsigned still = 0;   // sequences that go on climbing in this step
+            int n_steps_seen = 0;
+            for (int k = 0; k < nseq; ++k) {
+                const int s = seq0 + k, col = k * cps + (len[k] - 1 - base[k]);
+                if (col < 0 || col >= MAX_COLS || dprev.first_layer[col] > e - 1) continue;   // not in this step any more
+                if (!((head_cols >> col) & 1u)) { still |= 1u << k; continue; }                // climbing, but may not exit early
+                const HeadResult hr = hr_s[col];
+                bool decide = hr.p > gamma0;
+                if (s == 0 && tape_i < tape_n0) {
+                    const uint8_t t = st->tape[tape_i++];
+                    if (t == 0) decide = false;
+                    if (t == 1) decide = true;
+                }
+                bump(&st->st.head_evals, 1);
+                if (s == 0 && c.head_log && hl_n < kHeadLogCap) {
+                    float *hl = c.head_log + 4 * (size_t)hl_n;
+                    hl[0] = (float)(steps0 + n_steps_seen); hl[1] = (float)e; hl[2] = (float)hr.token; hl[3] = hr.p;
+                    ++hl_n;
+                }
+                if (!decide) { still |= 1u << k; continue; }
                 long long rl = 0;
                 for (int l = 0; l < e; ++l) {
-                    rl += len - fill_s[l];
-                    fill_s[l] = len;
-                    c.fill[l] = len;
+                    rl += len[k] - fill_s[k * L + l];
+                    fill_s[k * L + l] = len[k];
+                    c.fill[(size_t)s * L + l] = len[k];
                 }
                 bump(&st->st.row_layers, rl);
-                tok[len] = min(max(hr.token, 0), c.vocab - 1);
-                len = len + 1;
-                st->len[sq] = len;
+                c.tokens[(size_t)s * c.max_seq + len[k]] = min(max(hr.token, 0), c.vocab - 1);
+                len[k] += 1;
+                st->len[s] = len[k];
                 bump(&st->st.early_exits, 1);
                 bump(&st->st.exits_at_layer[e], 1);
                 bump(&st->st.steps, 1);
-                bump(&st->st.layer_passes, e);
+                ++n_steps_seen;
+                for (int j = 0; j < cps; ++j) nd.first_layer[k * cps + j] = INT_MAX;   // the sequence sits out the rest of the step
+                nd.head_mask &= ~(((1 << cps) - 1) << (k * cps));
             }
+            if (tape_i != st->tape_i) st->tape_i = tape_i;
+            if (hl_n != hl_n0) st->head_log_n = hl_n;
+            if (still) action = ACT_CONTINUE;
+            else bump(&st->st.layer_passes, e);   // the weights of layers 1..e were streamed once, for all the sequences
         }
         const bool prefilling = pf_end > 0;
         if (action != ACT_STOP && kind == CTRL_TOP && prefilling) {
-            // a pass over prompt positions [pf_pos, pf_pos + n) is complete at every layer
-            const int n = dprev.n_cols, end = pf_pos + n;
-            for (int l = 0; l < c.L; ++l) { fill_s[l] = end; c.fill[l] = end; }
+            // a pass over prompt positions [pf_pos, pf_pos + n) of the launch's one sequence is complete at every layer
+            const int s = seq0, n = dprev.n_cols, end = pf_pos + n;
+            for (int l = 0; l < L; ++l) { fill_s[l] = end; c.fill[(size_t)s * L + l] = end; }
             pf_pos = end;
             st->pf_pos = end;
             if (end >= pf_end) {   // KV cache <- LM(x) done: the full-depth argmax at the last prompt token is the first generated token
                 const int np = pf_end;
-                tok[np] = min(max(hr_s[n - 1].token, 0), c.vocab - 1);
-                len = np + 1; base = np; done = 1; pf_end = 0;
-                st->len[sq] = len;
-                st->base[sq] = base;
-                st->n_prompt[sq] = np;
-                st->done[sq] = 1;
+                c.tokens[(size_t)s * c.max_seq + np] = min(max(hr_s[n - 1].token, 0), c.vocab - 1);
+                len[0] = np + 1; base[0] = np; done[0] = 1; pf_end = 0;
+                st->len[s] = np + 1;
+                st->base[s] = np;
+                st->n_prompt[s] = np;
+                st->done[s] = 1;
                 st->pf_end = 0;
                 st->keep_rows = 1;
                 st->keep_row0 = n - 1;
-                verified = 1;
+                verified = s == 0;
             }
         }
+        // ---- verification (Eq. 2 at temperature zero) of every sequence whose newest token reached the last layer
         if (action != ACT_STOP && kind == CTRL_TOP && !prefilling) {
-            const int nrow = len - base;
-            long long rl = 0;
-            for (int l = 0; l < c.L; ++l) rl += len - fill_s[l];
-            bump(&st->st.row_layers, rl);
-            int bad = -1;
-            for (int j = 0; j + 1 < nrow; ++j)
-                if (hr_s[j].token != tok_s[j]) { bad = j; break; }
-            int new_base, keep;
-            if (bad < 0) {
-                bump(&st->st.accepted, nrow - 1);
-                tok[len] = min(max(hr_s[nrow - 1].token, 0), c.vocab - 1);
-                new_base = len;
-                keep = nrow;
-            } else {
-                bump(&st->st.accepted, bad);
-                bump(&st->st.rejected, 1);
-                bump(&st->st.discarded, nrow - 2 - bad);
-                new_base = base + bad + 1;
-                tok[new_base] = min(max(hr_s[bad].token, 0), c.vocab - 1);
-                keep = bad + 1;
+            for (int k = 0; k < nseq; ++k) {
+                const int s = seq0 + k, nrow = len[k] - base[k], c0 = k * cps;
+                if (nrow < 1 || nrow > cps || dprev.first_layer[c0 + nrow - 1] > L - 1) continue;   // left the step at an exit layer, or idle
+                int32_t *tok = c.tokens + (size_t)s * c.max_seq;
+                long long rl = 0;
+                for (int l = 0; l < L; ++l) rl += len[k] - fill_s[k * L + l];
+                bump(&st->st.row_layers, rl);
+                int bad = -1;
+                for (int j = 0; j + 1 < nrow; ++j)
+                    if (hr_s[c0 + j].token != tok_s[c0 + j]) { bad = j; break; }
+                int new_base, keep;
+                if (bad < 0) {
+                    bump(&st->st.accepted, nrow - 1);
+                    tok[len[k]] = min(max(hr_s[c0 + nrow - 1].token, 0), c.vocab - 1);
+                    new_base = len[k];
+                    keep = nrow;
+                } else {
+                    bump(&st->st.accepted, bad);
+                    bump(&st->st.rejected, 1);
+                    bump(&st->st.discarded, nrow - 2 - bad);
+                    new_base = base[k] + bad + 1;
+                    tok[new_base] = min(max(hr_s[c0 + bad].token, 0), c.vocab - 1);
+                    keep = bad + 1;
+                }
+                // Algorithm 1 runs "while t_i != [EOS]": the verified tokens of this step (positions base + 1 .. new_base,
+                // each equal to the full-depth argmax of the row before it) end the sequence at the first end-of-sequence
+                // token among them.  An early-predicted end-of-sequence token stops nothing until it is verified here.
+                int tgt = target[k];
+                if (eos0 >= 0) {
+                    for (int j = 0; j < keep; ++j)
+                        if (min(max(hr_s[c0 + j].token, 0), c.vocab - 1) == eos0) {
+                            if (base[k] + j + 2 <= tgt) { tgt = base[k] + j + 2; st->eos_hit[s] = 1; }
+                            break;
+                        }
+                }
+                int new_len = new_base + 1;
+                if (new_len > tgt) {
+                    bump(&st->st.truncated, new_len - tgt);
+                    new_len = tgt;
+                    new_base = new_len - 1;
+                }
+                keep = new_len - 1 - base[k];   // verified tokens that stay: their logit rows are the ones a capture keeps
+                for (int l = 0; l < L; ++l) { fill_s[k * L + l] = new_base; c.fill[(size_t)s * L + l] = new_base; }
+                len[k] = new_len; base[k] = new_base;
+                st->len[s] = new_len;
+                st->base[s] = new_base;
+                bump(&st->st.verify_steps, 1);
+                bump(&st->st.steps, 1);
+                if (new_len >= tgt) { done[k] = 1; st->done[s] = 1; }
+                if (s == 0) {
+                    st->keep_rows = keep;
+                    st->keep_row0 = 0;
+                    verified = 1;
+                }
             }
-            // Algorithm 1 runs "while t_i != [EOS]": the verified tokens of this step (positions base + 1 .. new_base,
-            // each equal to the full-depth argmax of the row before it) end the sequence at the first end-of-sequence
-            // token among them.  An early-predicted end-of-sequence token stops nothing until it is verified here.
-            int target = target0;
-            if (eos0 >= 0) {
-                for (int j = 0; j < keep; ++j)
-                    if (min(max(hr_s[j].token, 0), c.vocab - 1) == eos0) {
-                        if (base + j + 2 <= target) { target = base + j + 2; st->eos_hit[sq] = 1; }
-                        break;
-                    }
-            }
-            int new_len = new_base + 1;
-            if (new_len > target) {
-                bump(&st->st.truncated, new_len - target);
-                new_len = target;
-                new_base = new_len - 1;
-            }
-            keep = new_len - 1 - base;   // verified tokens that stay: their logit rows are the ones a capture keeps
-            for (int l = 0; l < c.L; ++l) { fill_s[l] = new_base; c.fill[l] = new_base; }
-            len = new_len; base = new_base;
-            st->len[sq] = len;
-            st->base[sq] = base;
-            bump(&st->st.verify_steps, 1);
-            bump(&st->st.steps, 1);
-            bump(&st->st.layer_passes, c.L);
-            if (new_len >= target) { done = 1; st->done[sq] = 1; }
-            st->keep_rows = keep;
-            st->keep_row0 = 0;
-            verified = 1;
         }
+        if (action != ACT_STOP && kind == CTRL_TOP && !prefilling) bump(&st->st.layer_passes, L);
         if (action == ACT_NEWSTEP) {
-            if (done) { action = ACT_STOP; st->n_done = 1; }
+            bool all_done = true;
+            for (int k = 0; k < nseq; ++k) all_done = all_done && done[k];
+            if (all_done) { action = ACT_STOP; st->n_done = 1; }
             else if (steps_started >= A.step_budget) action = ACT_STOP;
         }
-        if (action == ACT_NEWSTEP && pf_end > 0) {   // next pass over the prompt: up to eight positions, all from layer 1
+        if (action == ACT_NEWSTEP) {
             ++steps_started;
-            StepDesc nd;
-            nd.n_cols = min(MAX_COLS, pf_end - pf_pos);
-            nd.newest = nd.n_cols - 1;
-            nd.pmax = pf_pos + nd.n_cols - 1;
-            nd.head_ok = 0;
-            nd.fresh = (1 << nd.n_cols) - 1;
-            nd.run_final = pf_pos + nd.n_cols >= pf_end;
-            if (nd.n_cols < 1 || nd.pmax >= c.max_seq) {
-                atomicCAS(A.err, 0, ERR_BAD_STATE);
-                action = ACT_STOP;
-            }
-            for (int j = 0; j < MAX_COLS; ++j) {
-                nd.first_layer[j] = j < nd.n_cols ? 0 : INT_MAX;
-                nd.pos[j] = pf_pos + j;
-            }
-            pub->d = nd;
-        } else if (action == ACT_NEWSTEP) {
-            ++steps_started;
-            StepDesc nd;
-            nd.n_cols = len - base;
-            nd.newest = len - 1 - base;
-            nd.pmax = len - 1;
-            nd.fresh = 1 << (len - 1 - base);
-            nd.run_final = 1;
-            nd.head_ok = (len - 1 - base) < max_early0 && len < target0;
-            if (nd.n_cols < 1 || nd.n_cols > c.slots || nd.n_cols > MAX_COLS || len > c.max_seq || base < 0) {
-                atomicCAS(A.err, 0, ERR_BAD_STATE);
-                action = ACT_STOP;
-            }
-            for (int j = 0; j < MAX_COLS; ++j) {
-                int fl = INT_MAX;
-                const int pos = base + j;
-                if (j < nd.n_cols) {
-                    fl = 0;
-                    for (int l = 0; l < c.L; ++l) fl += fill_s[l] > pos;
+            nd.n_cols = 0; nd.newest_mask = 0; nd.head_mask = 0; nd.pmax = 0; nd.fresh = 0; nd.run_final = 1;
+            for (int j = 0; j < MAX_COLS; ++j) { nd.first_layer[j] = INT_MAX; nd.pos[j] = 0; nd.seq_pmax[j] = -1; }
+            if (pf_end > 0) {   // next pass over the prompt: up to eight positions, all from layer 1
+                const int n = min(MAX_COLS, pf_end - pf_pos);
+                nd.n_cols = n;
+                nd.newest_mask = 1 << (n - 1);
+                nd.pmax = pf_pos + n - 1;
+                nd.seq_pmax[0] = nd.pmax;
+                nd.fresh = (1 << n) - 1;
+                nd.run_final = pf_pos + n >= pf_end;
+                if (n < 1 || nd.pmax >= c.max_seq) {
+                    atomicCAS(A.err, 0, ERR_BAD_STATE);
+                    action = ACT_STOP;
                 }
-                nd.first_layer[j] = fl;
-                nd.pos[j] = pos;
+                for (int j = 0; j < n; ++j) { nd.first_layer[j] = 0; nd.pos[j] = pf_pos + j; }
+            } else {
+                for (int k = 0; k < nseq; ++k) {
+                    if (done[k]) continue;   // a sequence that has reached its target idles while the others go on
+                    const int nrow = len[k] - base[k], c0 = k * cps;
+                    if (nrow < 1 || nrow > cps || c0 + nrow > MAX_COLS || len[k] > c.max_seq || base[k] < 0) {
+                        atomicCAS(A.err, 0, ERR_BAD_STATE);
+                        action = ACT_STOP;
+                        break;
+                    }
+                    for (int j = 0; j < nrow; ++j) {
+                        const int pos = base[k] + j;
+                        int fl = 0;
+                        for (int l = 0; l < L; ++l) fl += fill_s[k * L + l] > pos;
+                        nd.first_layer[c0 + j] = fl;
+                        nd.pos[c0 + j] = pos;
+                    }
+                    const int cn = c0 + nrow - 1;
+                    nd.n_cols += nrow;
+                    nd.newest_mask |= 1 << cn;
+                    nd.fresh |= 1 << cn;
+                    if (nrow - 1 < max_early0 && len[k] < target[k]) nd.head_mask |= 1 << cn;
+                    nd.seq_pmax[k] = len[k] - 1;
+                    nd.pmax = max(nd.pmax, len[k] - 1);
+                }
             }
-            pub->d = nd;
         }
+        if (action == ACT_NEWSTEP || action == ACT_CONTINUE) pub->d = nd;
         pub->action = action;
         sm->bcast[0] = action;
         sm->bcast[3] = verified;
@@ -384,7 +423,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     bar_consumers();
     const int action = sm->bcast[0];
     // (c) logits of the verified rows (test hook), then the embedding of the next newest token
-    if (sq == 0 && kind == CTRL_TOP && c.capture && sm->bcast[3]) {
+    if (kind == CTRL_TOP && c.capture && sm->bcast[3]) {
         const int keep = st->keep_rows, at = st->capture_n;
         for (int j = 0; j < keep && at + j < st->capture_cap; ++j) {
             const float *src = c.logit_stage + (size_t)(st->keep_row0 + j) * c.vocab;
@@ -401,7 +440,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
         for (int col = 0; col < MAX_COLS; ++col) {
             if (!((nd.fresh >> col) & 1)) continue;
             const int pos = nd.pos[col];
-            const int tokid = min(max(c.tokens[pos], 0), c.vocab - 1);
+            const int tokid = min(max(c.tokens[(size_t)(seq0 + (nseq == 1 ? 0 : col / cps)) * c.max_seq + pos], 0), c.vocab - 1);
             const __nv_bfloat16 *erow = M.tok_embed + (size_t)tokid * c.d;
             for (int n0 = 0; n0 < c.d; n0 += 8 * CONS_THREADS) {   // eight loads of the embedding row and of the gain in flight per thread
                 float v[8], gn[8];
@@ -459,13 +498,15 @@ __device__ __forceinline__ int control_point(const MegaArgs &A, const Shared &S,
     // producer warp: same values), and checked before anything is indexed with it
     auto fetch = [&]() -> int {
         int act = aborted(S) ? ACT_STOP : *(volatile const int *)&pub->action;
-        if (act == ACT_NEWSTEP) {
+        if (act == ACT_NEWSTEP || act == ACT_CONTINUE) {   // a step that goes on may have lost the columns of sequences that left it
             const volatile int *src = reinterpret_cast<const volatile int *>(&pub->d);
             int *dst = reinterpret_cast<int *>(&d);
 #pragma unroll
             for (int i = 0; i < (int)(sizeof(StepDesc) / 4); ++i) dst[i] = src[i];
-            if (d.n_cols < 1 || d.n_cols > MAX_COLS || d.newest < 0 || d.newest >= MAX_COLS || d.pmax < 0 || d.pmax >= A.c.max_seq)
-                act = ACT_STOP;   // cannot happen unless memory was corrupted; never index with it
+            bool bad = d.n_cols < 1 || d.n_cols > MAX_COLS || d.pmax < 0 || d.pmax >= A.c.max_seq;
+#pragma unroll
+            for (int i = 0; i < MAX_COLS; ++i) bad = bad || d.pos[i] < 0 || d.pos[i] >= A.c.max_seq || d.seq_pmax[i] >= A.c.max_seq;
+            if (bad) act = ACT_STOP;   // cannot happen unless memory was corrupted; never index with it
         }
         // The two record slots alternate.  A role that fell two control points behind would find its slot
         // already rewritten for a later one: a record is used only if its number is still the expected one
@@ -513,6 +554,34 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// Attention work items of a launch that holds several sequences: sequence k of the launch (token columns
+// [k cps, (k + 1) cps); all eight in a prompt pass, which holds one sequence) contributes n_kv_heads x its
+// own number of 128-position chunks, and an item works on that sequence's columns and cache pages only.
+__device__ __forceinline__ unsigned seq_cols(const MegaArgs &A, int k) {
+    return A.nseq == 1 ? 0xffu : (((1u << A.c.slots) - 1u) << (k * A.c.slots));
+}
+__device__ __forceinline__ int seq_chunks(const MegaArgs &A, const StepDesc &d, unsigned mask, int k) {
+    return ((mask & seq_cols(A, k)) != 0 && d.seq_pmax[k] >= 0) ? d.seq_pmax[k] / ATT_CHUNK + 1 : 0;
+}
+__device__ __forceinline__ int attn_items(const MegaArgs &A, const StepDesc &d, unsigned mask) {
+    int n = 0;
+    for (int k = 0; k < A.nseq; ++k) n += A.c.nkv * seq_chunks(A, d, mask, k);
+    return n;
+}
+// item -> (sequence of the launch, kv head, chunk); nchunk = the sequence's chunk count
+__device__ __forceinline__ void attn_item(const MegaArgs &A, const StepDesc &d, unsigned mask, int item, int &k, int &kvh, int &j, int &nchunk) {
+    k = 0;
+    nchunk = seq_chunks(A, d, mask, 0);
+    while (k + 1 < A.nseq && item >= A.c.nkv * nchunk) {
+        item -= A.c.nkv * nchunk;
+        ++k;
+        nchunk = seq_chunks(A, d, mask, k);
+    }
+    nchunk = max(nchunk, 1);
+    kvh = min(item / nchunk, A.c.nkv - 1);
+    j = item - kvh * nchunk;
+}
+
 // K/V producer: for every work item of this CTA, the K and V page blocks of its sub-blocks.  The K and V
 // rows of the tokens of this pass were written into the cache by the QKV epilogues of other CTAs; a
 // work item whose positions include such a row is fetched only once the grid has passed the barrier
@@ -523,26 +592,29 @@ __device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S,
     const Ctx &c = A.c;
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31, cta = blockIdx.x, G = gridDim.x;
-    const int nchunk = d.pmax / ATT_CHUNK + 1, n_items = c.nkv * nchunk;
+    const int n_items = attn_items(A, d, mask);
     const uint32_t bytes = (uint32_t)(ATT_PAGE * c.hd * 2);
     const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
     bool synced = false;
     if (lane == 0) trace(S, EV_ATT, 8);
     for (int item = cta; item < n_items; item += G) {
-        const int kvh = item / nchunk, j = item - kvh * nchunk;
+        int k, kvh, j, nchunk;
+        attn_item(A, d, mask, item, k, kvh, j, nchunk);
+        const unsigned mk = mask & seq_cols(A, k);
+        const int32_t *pages = c.page_table + (size_t)(A.seq0 + k) * c.max_pages;
         const int p_base = j * ATT_CHUNK;
-        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.pmax - p_base) / ATT_PAGE + 1);
+        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[k] - p_base) / ATT_PAGE + 1);
         bool has_new = false;
 #pragma unroll
         for (int cc = 0; cc < MAX_COLS; ++cc)
-            has_new = has_new || (((mask >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK);
+            has_new = has_new || (((mk >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK);
         if (has_new && !synced) {
             grid_wait(S, A.grid_ctr, bar_target);
             fence_proxy_async();
             synced = true;
         }
         for (int sb = 0; sb < nsb; ++sb) {
-            const int page = c.page_table[(p_base + sb * ATT_PAGE) >> c.page_shift];
+            const int page = pages[(p_base + sb * ATT_PAGE) >> c.page_shift];
             for (int which = 0; which < 2; ++which) {
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
@@ -619,17 +691,17 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     constexpr int QV = 2 * KSQ * 64 / CONS_THREADS;        // 16-byte pieces of a kv head's query fragments per thread
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x, G = gridDim.x;
     const int group = c.group;
-    const int nchunk = d.pmax / ATT_CHUNK + 1, n_items = c.nkv * nchunk;
+    const int n_items = attn_items(A, d, mask);
     const int mt = warp >> 2, qr = warp & 3;
     (void)layer;
     // Merge of the chunk partials of one kv head into the O-projection's input (by a whole CTA).
-    auto merge_chunks = [&](int kvh) {
+    auto merge_chunks = [&](int kvh, unsigned mk) {   // mk: the active columns of the work item's sequence
         // Four features of one (column, q head) per thread and pass; the chunk partials are folded in
         // ascending order, eight at a time with all their loads in flight, by the usual running-max rule.
         const int nqc = MAX_COLS * group;
         for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
             const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = div_group(qcol, group), g = qcol - cc * group;
-            if (!((mask >> cc) & 1u)) continue;
+            if (!((mk >> cc) & 1u)) continue;
             const int h = kvh * group + g;
             const int nch = d.pos[cc] / ATT_CHUNK + 1;
             const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE;
@@ -671,9 +743,11 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     // designated CTAs do (see below).  Who merges does not change what is computed.
     const bool last_arriver_merges = n_items <= G;
     for (int item = cta; item < n_items; item += G) {
-        const int kvh = item / nchunk, j = item - kvh * nchunk;
+        int ks_, kvh, j, nchunk;
+        attn_item(A, d, mask, item, ks_, kvh, j, nchunk);
+        const unsigned mk = mask & seq_cols(A, ks_);   // the item's sequence: its columns only
         const int p_base = j * ATT_CHUNK;
-        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.pmax - p_base) / ATT_PAGE + 1);
+        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[ks_] - p_base) / ATT_PAGE + 1);
         // ---- the kv head's query fragments: one round trip to L2, then shared memory
         {
             const uint4 *src = reinterpret_cast<const uint4 *>(A.qfrag) + (size_t)kvh * (2 * KSQ * 64);
@@ -691,14 +765,14 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
 #pragma unroll
         for (int rh = 0; rh < 2; ++rh) {
             const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = div_group(qcol, group);
-            lim[rh] = (cc < MAX_COLS && ((mask >> cc) & 1u)) ? d.pos[cc] : -1;
+            lim[rh] = (cc < MAX_COLS && ((mk >> cc) & 1u)) ? d.pos[cc] : -1;
         }
         // a query tile none of whose 16 (column, q head) pairs is in use does no arithmetic (uniform per warp)
         bool tile_used = false;
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int cc = div_group(mt * 16 + q, group);
-            tile_used = tile_used || (cc < MAX_COLS && ((mask >> cc) & 1u));
+            tile_used = tile_used || (cc < MAX_COLS && ((mk >> cc) & 1u));
         }
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
         float o[NT][4];
@@ -828,7 +902,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
 #pragma unroll
             for (int rh = 0; rh < 2; ++rh) {
                 const int qcol = mt * 16 + (lane >> 2) + 8 * rh, cc = div_group(qcol, group), g = qcol - cc * group;
-                if (cc < MAX_COLS && ((mask >> cc) & 1u) && d.pos[cc] >= p_base) {
+                if (cc < MAX_COLS && ((mk >> cc) & 1u) && d.pos[cc] >= p_base) {
                     float *out = A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + j) * ATT_STRIDE;
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
@@ -843,17 +917,17 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
         if (last_arriver_merges) {
             if (tid == 0) {   // release this block's partials and acquire the others' in one step
                 unsigned old;
-                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + kvh) : "memory");
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + ks_ * c.nkv + kvh) : "memory");
                 sm->bcast[2] = (int)old;
             }
             bar_consumers();
             if (sm->bcast[2] == nchunk - 1) {
-                merge_chunks(kvh);
-                if (tid == 0) { A.attn_cnt[kvh] = 0u; trace(S, EV_COMBINE, kvh); }
+                merge_chunks(kvh, mk);
+                if (tid == 0) { A.attn_cnt[ks_ * c.nkv + kvh] = 0u; trace(S, EV_COMBINE, kvh); }
             }
         } else if (tid == 0) {
             __threadfence();
-            red_release_add(A.attn_cnt + kvh, 1u);
+            red_release_add(A.attn_cnt + ks_ * c.nkv + kvh, 1u);
         }
     }
     if (last_arriver_merges) return;
@@ -862,13 +936,15 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     // whichever CTA arrives last do it looks cheaper but piles up at long contexts: the CTA that
     // merges one head is late for its next item, so it is last again for the next head, and ends up
     // merging every head in turn while the rest of the grid waits.)
-    for (int kvh = 0; kvh < c.nkv; ++kvh) {
-        if ((G - 1 - kvh % G + G) % G != cta) continue;
-        if (tid == 0) grid_wait(S, A.attn_cnt + kvh, (unsigned)nchunk);
+    for (int hk = 0; hk < A.nseq * c.nkv; ++hk) {   // (sequence of the launch, kv head)
+        if ((G - 1 - hk % G + G) % G != cta) continue;
+        const int ks_ = hk / c.nkv, kvh = hk - ks_ * c.nkv, nchunk = seq_chunks(A, d, mask, ks_);
+        if (nchunk == 0) continue;
+        if (tid == 0) grid_wait(S, A.attn_cnt + hk, (unsigned)nchunk);
         bar_consumers();
         {
-            merge_chunks(kvh);
-            if (tid == 0) { A.attn_cnt[kvh] = 0u; trace(S, EV_COMBINE, kvh); }
+            merge_chunks(kvh, mask & seq_cols(A, ks_));
+            if (tid == 0) { A.attn_cnt[hk] = 0u; trace(S, EV_COMBINE, kvh); }
         }
         bar_consumers();   // the next head's wait must not start before every thread is done with this one
     }
@@ -909,9 +985,9 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     // then costs a round trip to L2 on the critical path.
     StepDesc &d = *reinterpret_cast<StepDesc *>(sm->desc[ROLE]);
     if (ROLE != 2 || threadIdx.x == 0) {
-        d.n_cols = 0; d.newest = 0; d.head_ok = 0; d.pmax = 0; d.fresh = 0; d.run_final = 1;
+        d.n_cols = 0; d.newest_mask = 0; d.head_mask = 0; d.pmax = 0; d.fresh = 0; d.run_final = 1;
 #pragma unroll
-        for (int i = 0; i < MAX_COLS; ++i) { d.first_layer[i] = INT_MAX; d.pos[i] = 0; }
+        for (int i = 0; i < MAX_COLS; ++i) { d.first_layer[i] = INT_MAX; d.pos[i] = 0; d.seq_pmax[i] = -1; }
     }
     if (ROLE == 2) bar_consumers(); else __syncwarp();
 
@@ -946,7 +1022,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
     };
     // head over E* with the fused (max, sum exp, argmax) reduction; X = final-normed residual (or T output)
     auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols) {
-        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head; g.part = nullptr; g.phase_id = bar_no + 1; g.columns(cols ? cols : 1u << d.newest);
+        Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head; g.part = nullptr; g.phase_id = bar_no + 1; g.columns(cols);
         x_ready();
         const unsigned vseq = bar_no + 1;
         if (ROLE == 2) {
@@ -1050,7 +1126,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                                 cp_async4(stash + (2 * q) * 32, cs);
                                 cp_async4(stash + (2 * q + 1) * 32, cs + 1);
                             }
-                            if (n0 >= qd) cp_async4(stash + (4 + q) * 32, c.page_table + (d.pos[cc] >> c.page_shift));
+                            if (n0 >= qd) cp_async4(stash + (4 + q) * 32, c.page_table + (size_t)(A.seq0 + (A.nseq == 1 ? 0 : cc / c.slots)) * c.max_pages + (d.pos[cc] >> c.page_shift));
                         }
                     }, [&](int tile, float (&acc)[1][4]) {
                         if (!have_r) { vec_wait(S, vseq); r0 = sm->vec[c0]; r1 = sm->vec[c0 + 1]; have_r = true; }
@@ -1223,10 +1299,11 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                 phase_barrier(8);
             }
             // ---- intermediate head (Section 2.1) and the early-prediction rule (Eq. 1)
-            if (l + 1 < L && A.exit_at[l + 1] != 0 && d.head_ok) {
+            const unsigned hcols = (unsigned)d.head_mask & mask;   // newest tokens that reached this layer and may exit early
+            if (l + 1 < L && A.exit_at[l + 1] != 0 && hcols != 0) {
                 const MegaLayer &hl = M.layer[l + 1];
                 if (hl.wT) {
-                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_d; g.part = nullptr; g.phase_id = bar_no + 1; g.columns(1u << d.newest);
+                    Gemm g; g.W = hl.wT; g.X = reinterpret_cast<const uint4 *>(A.XF); g.N = d_model; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_d; g.part = nullptr; g.phase_id = bar_no + 1; g.columns(hcols);
                     x_ready();
                     const unsigned vseq = bar_no + 1;
                     if (ROLE == 2) {
@@ -1244,9 +1321,9 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                     } else if (ROLE == 1) gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { rstd_produce(sm, A.ssq_a, ntd, d_model, c.eps, vseq); });
                     else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
                     phase_barrier(10);
-                    head_phase(A.XT, nullptr, hl.head_scale, 0u);
+                    head_phase(A.XT, nullptr, hl.head_scale, hcols);
                 } else {
-                    head_phase(A.XF, A.ssq_a, hl.head_scale, 0u);
+                    head_phase(A.XF, A.ssq_a, hl.head_scale, hcols);
                 }
                 action = control_point<ROLE>(A, S, CTRL_HEAD, l + 1, pub_no, d, steps_started);
                 book_control();
@@ -1284,8 +1361,7 @@ __global__ void k_repack_qkv(const __nv_bfloat16 *__restrict__ wq, const __nv_bf
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) d4[i] = s4[i];
 }
 
-// Arms the prompt passes of the persistent kernel for one sequence (KV cache <- LM(x), first line of Algorithm 1);
-// c.fill points at that sequence's fill levels.
+// Arms the prompt passes of the persistent kernel for one sequence (KV cache <- LM(x), first line of Algorithm 1).
 __global__ void k_prefill_arm(Ctx c, int seq, int n_prompt) {
     DevState *st = c.st;
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
@@ -1297,7 +1373,7 @@ __global__ void k_prefill_arm(Ctx c, int seq, int n_prompt) {
     st->base[seq] = 0;
     st->tape_n = 0;
     st->tape_i = 0;
-    for (int l = 0; l < c.L; ++l) c.fill[l] = 0;
+    for (int l = 0; l < c.L; ++l) c.fill[(size_t)seq * c.L + l] = 0;
 }
 
 template <int HD>

@@ -418,3 +418,62 @@ def test_batch_of_ragged_sequences_on_the_persistent_path():
     assert list(st.emitted[:3]) == [n, k + 1, n] and st.finished == 1
     assert np.array_equal(e[0], singles[0]) and np.array_equal(e[2], singles[2])
     assert np.array_equal(e[1][:k + 1], singles[1][:k + 1]) and (e[1][k + 1:] == eos).all()
+
+
+@pytest.mark.parametrize("max_early,batch", [(1, 4), (3, 3), (0, 8)])
+def test_sequences_sharing_one_weight_stream(max_early, batch):
+    """Sessions whose sequences fit the kernel's eight token columns together (batch x (max_early + 1) <= 8, or
+    groups of 8 / (max_early + 1)): every launch decodes the group in lock-step over one pass of the weights.  Each
+    sequence still equals its own single-sequence run bit for bit: plain, adaptive (decisions differ per sequence),
+    and with an end-of-sequence token that stops one sequence while the others run on."""
+    cfg = gqa()
+    pair = Pair(cfg)
+    lens = [5, 19, 70, 33, 8, 41, 12, 27][:batch]
+    prompts = [synth.make_prompt(cfg, n=n, seq=i).numpy() for i, n in enumerate(lens)]
+    n = 24
+    singles = []
+    for p in prompts:
+        S = session(pair)
+        S.prefill(p)
+        one = binding.Stats()
+        singles.append(S.plain_decode(n, one)[0])
+
+    def fresh():
+        B = binding.Session(pair.gm, batch, 256, 64, max_early)
+        assert B.get_path() == 1
+        for i, p in enumerate(prompts):
+            B.prefill(p, seq=i)
+        return B
+
+    st = binding.Stats()
+    out = fresh().plain_decode(n, st)
+    for i in range(batch):
+        assert np.array_equal(out[i], singles[i]), i
+    assert st.path == 1 and list(st.emitted[:batch]) == [n] * batch
+    # one pass of the weights per step for the whole group, not one per sequence
+    group = min(batch, 8 // (max_early + 1))
+    launches_groups = -(-batch // group)
+    assert st.layer_passes == launches_groups * one.layer_passes
+    if max_early == 0:
+        return
+    A = fresh()
+    st = binding.Stats()
+    a1 = A.adaptive_decode(10, 0.3, cfg.exit_layers, max_early, st)
+    a2 = A.adaptive_decode(n - 10, 0.0, cfg.exit_layers, max_early, st)
+    assert np.array_equal(np.concatenate([a1, a2], axis=1), out) and st.early_exits > 0
+    for i in range(batch):
+        ln, fill = A.state(i)
+        assert ln == lens[i] + n and (fill == lens[i] + n - 1).all()
+    k = next(j for j in range(3, n) if singles[1][j] not in singles[1][:j]
+             and all(singles[1][j] not in singles[o] for o in range(batch) if o != 1))
+    eos = int(singles[1][k])
+    E = fresh()
+    st = binding.Stats()
+    e = E.adaptive_decode(n, 0.3, cfg.exit_layers, max_early, st, eos_id=eos)
+    want = [n] * batch
+    want[1] = k + 1
+    assert list(st.emitted[:batch]) == want and st.finished == 1
+    for i in range(batch):
+        if i != 1:
+            assert np.array_equal(e[i], singles[i]), i
+    assert np.array_equal(e[1][:k + 1], singles[1][:k + 1]) and (e[1][k + 1:] == eos).all()
