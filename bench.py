@@ -138,7 +138,7 @@ class Bench:
     """One model, one session, timed decode runs of it."""
 
     def __init__(self, cfg, torch, binding, synth, sizes, warm, dist=None, resid_scale=None, logit_scale=None,
-                 dense_T=False, launch_steps=0, seed=1234):
+                 dense_T=False, launch_steps=0, seed=1234, max_early=-1):
         import dataclasses
         self.torch, self.binding, self.dist = torch, binding, dist
         if resid_scale is not None:
@@ -156,9 +156,15 @@ class Bench:
             self.prompts = [synth.make_prompt(cfg, seed=5678).numpy()]
         self.gen_len = sum(sizes)
         max_seq = max(len(p) for p in self.prompts) + max(self.gen_len, max(sizes) * max(warm, 1)) + 16
-        self.sess = binding.Session(self.model, self.batch, max_seq, 64, 5)
+        # A sequence holds max_early + 1 of the persistent kernel's eight token columns.  One sequence: the paper's
+        # setting of up to five early-predicted tokens.  A batch: as many as still let all its sequences share every
+        # pass over the weights.
+        self.max_early = max_early if max_early >= 0 else (5 if self.batch == 1 else max(0, 8 // self.batch - 1))
+        self.sess = binding.Session(self.model, self.batch, max_seq, 64, self.max_early)
         if launch_steps > 0 and self.sess.get_path() == 1:
             self.sess.set_launch_steps(launch_steps)
+        # launches a decode call needs for the batch (each streams the weights for its own sequences)
+        self.groups = -(-self.batch // max(1, 8 // (self.max_early + 1))) if self.sess.get_path() == 1 else 1
         m = max(sizes)
         self.out = np.empty((self.batch, m), dtype=np.int32)
         try:
@@ -166,7 +172,8 @@ class Bench:
         except Exception:
             pass
         self.prompt_bytes = sum(4 * len(p) for p in self.prompts)
-        self.ctx_sum = sum(len(p) for p in self.prompts) + self.batch * self.gen_len / 2
+        # cached positions one layer pass reads: those of the sequences that share the pass
+        self.ctx_sum = (sum(len(p) for p in self.prompts) + self.batch * self.gen_len / 2) / self.groups
 
     def register_heads(self, scale, dense_T=False):
         torch = self.torch
@@ -201,7 +208,7 @@ class Bench:
         for n in sizes:
             o = self.out[:, :n] if n == self.out.shape[1] else np.empty((self.batch, n), dtype=np.int32)
             if mode == "adaptive":
-                sess.adaptive_decode(n, threshold, exit_layers, 5, st, out=o)
+                sess.adaptive_decode(n, threshold, exit_layers, self.max_early, st, out=o)
             else:
                 sess.plain_decode(n, st, out=o)
             toks.append(o.copy())
@@ -226,7 +233,7 @@ class Bench:
         for n in sizes:
             o = self.out[:, :n] if n == self.out.shape[1] else np.empty((self.batch, n), dtype=np.int32)
             if mode == "adaptive":
-                sess.adaptive_decode(n, self.cfg.threshold, self.cfg.exit_layers, 5, st, out=o)
+                sess.adaptive_decode(n, self.cfg.threshold, self.cfg.exit_layers, self.max_early, st, out=o)
             else:
                 sess.plain_decode(n, st, out=o)
         self.barrier()
@@ -269,7 +276,7 @@ def run_ours(args):
     gen_len = args.gen_len if args.gen_len > 0 else cfg.gen_len
     sizes = step_sizes(gen_len, K)
     warm = [sizes[0]] * max(Wm, 1)
-    B = Bench(cfg, torch, binding, synth, sizes, max(Wm, 1), dist, launch_steps=args.launch_steps)
+    B = Bench(cfg, torch, binding, synth, sizes, max(Wm, 1), dist, launch_steps=args.launch_steps, max_early=args.max_early)
     path = B.sess.get_path()
 
     if args.plain_only or args.adaptive_only:
@@ -331,10 +338,12 @@ def run_ours(args):
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": f"{cfg.name}-shaped decoder bs{cfg.batch}, {prompt_desc}, "
                                f"{gen_len} greedy tokens each, exits {list(cfg.exit_layers)}, gamma {cfg.threshold}, "
-                               f"tied head logit scale {cfg.logit_scale}, max_early 5, o/down scale {cfg.resid_scale}",
+                               f"tied head logit scale {cfg.logit_scale}, max_early {B.max_early}, o/down scale {cfg.resid_scale}",
                    "tokens_per_step": sizes[0], "last_step_tokens": sizes[-1], "l2": "inputs_larger_than_l2 (weights stream >> 126 MB)",
-                   "decode_path": ("persistent kernel" + (", sequences decoded one after another (each streams the weights for itself)"
-                                                           if cfg.batch > 1 else "")) if path == 1 else "one kernel per operation",
+                   "decode_path": ("persistent kernel" + ("" if cfg.batch == 1 else
+                                                           ", all sequences share every pass over the weights" if B.groups == 1 else
+                                                           f", sequences in {B.groups} groups, each group streams the weights for itself"))
+                                  if path == 1 else "one kernel per operation",
                    "parallelism": "replicas" if world > 1 else "single"},
         "e2e": {"value": whole_job_tokens_per_s(n_tok, world, a_wall), "unit": UNIT,
                 "h2d_bytes_per_step": int(64 + 4 * 16 + 4 * len(cfg.exit_layers)),
@@ -508,6 +517,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--max-early", type=int, default=-1,
+                    help="early-predicted tokens a sequence may hold (default: 5 for one sequence, 8 // batch - 1 for a batch)")
     ap.add_argument("--workload", default="8b", choices=["tiny", "1b", "8b", "8b-long", "13b"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
