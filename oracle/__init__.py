@@ -20,6 +20,9 @@ _SRC = os.path.join(_HERE, "adadecode_oracle.c")
 _LIB = None
 
 
+NU = 8   # random numbers per sequence position of a sampling decode call
+
+
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (OpenMP across mat-vec output rows)."""
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
@@ -83,6 +86,8 @@ def _lib():
         L.orc_adaptive_decode.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_int, C.c_int,
                                           C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_int32),
                                           C.POINTER(Stats)]
+        L.orc_sampling_decode.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p, C.c_int, C.c_int,
+                                          C.c_void_p, C.c_int, C.c_void_p, C.POINTER(C.c_int32), C.POINTER(Stats)]
         _LIB = L
     return _LIB
 
@@ -177,6 +182,7 @@ class Model:
 class Session:
     def __init__(self, model: Model, max_seq: int):
         self.model = model
+        self.max_seq = max_seq
         self.h = _lib().orc_session_create(model.h, max_seq)
         if not self.h:
             raise MemoryError("orc_session_create")
@@ -268,6 +274,24 @@ class Session:
                                         out.ctypes.data, C.byref(got), C.byref(stats) if stats is not None else None)
         if rc:
             raise RuntimeError(f"orc_adaptive_decode -> {rc}")
+        self.emitted = got.value
+        return out
+
+    def sampling_decode(self, n: int, temperature: float, gamma: float, exit_layers: Sequence[int], max_early: int,
+                        uniforms: np.ndarray, stats: Optional[Stats] = None, eos_id: int = -1) -> np.ndarray:
+        """Algorithm 1 with sampled tokens (Eq. 1) and the acceptance test and resampling of Eq. 2.
+        `uniforms[pos][k]`, float64 in [0, 1), k < NU: the random numbers of the token at sequence position pos
+        ([0] draw at the last layer, [1] acceptance test, [2] resampling, [3 + e] draw at the e-th exit layer)."""
+        out = np.empty(n, dtype=np.int32)
+        got = C.c_int32(0)
+        ex = np.ascontiguousarray(np.asarray(exit_layers, dtype=np.int32))
+        u = np.ascontiguousarray(np.asarray(uniforms, dtype=np.float64))
+        assert u.ndim == 2 and u.shape[1] == NU and u.shape[0] >= self.max_seq
+        rc = _lib().orc_sampling_decode(self.h, n, temperature, gamma, ex.ctypes.data, len(ex), max_early,
+                                        u.ctypes.data, eos_id, out.ctypes.data, C.byref(got),
+                                        C.byref(stats) if stats is not None else None)
+        if rc:
+            raise RuntimeError(f"orc_sampling_decode -> {rc}")
         self.emitted = got.value
         return out
 

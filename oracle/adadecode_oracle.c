@@ -9,7 +9,10 @@
  *       Section 2.2 "output parity", Table 2 "Vanilla Decoding");
  *   (3) Algorithm 1 (adaptive layer parallelism) with the early-prediction rule of Eq. 1, the
  *       lightweight head E^(i) = E* T^(i) of Section 2.1, and the verification rule of Eq. 2 in
- *       its greedy (temperature 0, Appendix D) form, including KV-cache rollback.
+ *       its greedy (temperature 0, Appendix D) form, including KV-cache rollback;
+ *   (4) the same algorithm with sampled tokens: Eq. 1 with a draw from the head's distribution and Eq. 2 with
+ *       its acceptance probability and the resampling from Normalize(max(0, p* - q)) (orc_sampling_decode,
+ *       at the end of the file; every random number is an input).
  *
  * Only tests, the smoke check and the benchmark's CPU-baseline leg may call this file.  It
  * shares no code with the CUDA library and never calls it.  All floating point is IEEE double;
@@ -21,7 +24,9 @@
  * Pins (tests that do not run the CUDA path): an independent NumPy restatement of the decoder,
  * closed forms (zero weights, identity head), incremental == from-scratch recompute, brute force
  * over every exit-decision tape (output equals plain greedy), the gamma = 0 / gamma = 1 end
- * points of Section 4.4, the worked schedule of Figure 2, the cap of Appendix D.
+ * points of Section 4.4, the worked schedule of Figure 2, the cap of Appendix D; for the sampled form the
+ * closed-form law of a verified token (chi-square over seeded runs, with planted wrong rules rejected),
+ * gamma = 0 = plain sampling, vanishing temperature = greedy, no exit layers = numpy's inverse CDF.
  * Parity unpinned: the exit and rejection RATES on random weights (they are properties of the
  * synthetic model, not values the paper fixes); they are reported, never asserted.
  */
@@ -641,5 +646,192 @@ int orc_adaptive_decode(orc_session *s, int n, double gamma, const int32_t *exit
     }
 done:
     free(P); free(Pn); free(H); free(z); free(argm);
+    return rc;
+}
+
+/* ---------------------------------------------------------------- Algorithm 1 with sampling */
+
+#define ORC_NU 8 /* uniforms per sequence position: [0] draw at the last layer, [1] acceptance test of Eq. 2,
+                    [2] resampling after a rejection, [3 + e] draw at the e-th exit layer of the call (e < 5) */
+
+/* softmax(z / temperature) into p */
+static void softmax_t(const double *z, int V, double temperature, double *p) {
+    double zmax = z[0], den = 0.0;
+    for (int t = 1; t < V; ++t) if (z[t] > zmax) zmax = z[t];
+    for (int t = 0; t < V; ++t) { p[t] = exp((z[t] - zmax) / temperature); den += p[t]; }
+    for (int t = 0; t < V; ++t) p[t] /= den;
+}
+
+/* Inverse-CDF draw in vocabulary order from the non-negative weights w: the first token whose running
+   sum exceeds u x (sum of all weights); the last token of non-zero weight if rounding leaves none. */
+static int draw(const double *w, int V, double u) {
+    double total = 0.0, run = 0.0;
+    int last = 0;
+    for (int t = 0; t < V; ++t) total += w[t];
+    for (int t = 0; t < V; ++t) {
+        if (w[t] > 0.0) last = t;
+        run += w[t];
+        if (run > u * total) return t;
+    }
+    return last;
+}
+
+/*
+ * Algorithm 1 with a sampled next token instead of the greedy one.
+ *
+ *   Eq. 1: at an exit layer the newest token's successor is DRAWN from the head's distribution
+ *          q = softmax(head logits / temperature); the draw t is emitted early iff q(t) > gamma,
+ *          otherwise it is thrown away and the token climbs on.
+ *   Eq. 2: at the last layer every early-predicted token t (drawn from q at its exit layer) is accepted
+ *          with probability min{1, p*(t) / q(t)}, p* = softmax(final logits / temperature) of the row
+ *          before it, in sequence order; the first rejected one is replaced by a draw from
+ *          Normalize(max(0, p* - q)), the K/V of everything from its position on is dropped and
+ *          generation resumes from the replacement.  If all are accepted the next token is drawn from
+ *          p* of the newest row.
+ *
+ * Every random number is an input: u[pos * ORC_NU + k] belongs to the token at sequence position pos.
+ * A position that is drawn again after a rollback uses its numbers again: they are independent of the
+ * event that caused the rollback (the acceptance test of an earlier position).
+ *
+ * gamma = 0 makes every consulted head emit its draw, which is speculative sampling with the head as
+ * the draft distribution: the verified tokens are then distributed exactly as plain sampling from p*.
+ * For gamma > 0 the draft is used only where q(t) > gamma and the law of a verified token is
+ *   P(v) = sum_i prod_{j<i}(1 - Q_j) [ 1{q_i(v) > gamma} min(q_i(v), p*(v)) + R_i res_i(v) ] + prod_j (1 - Q_j) p*(v),
+ * Q_i = sum_{q_i(t) > gamma} q_i(t), R_i = sum_{q_i(t) > gamma} max(0, q_i(t) - p*(t)), res_i = Normalize(max(0, p* - q_i)),
+ * which the tests compute independently and compare with the frequencies this function produces.
+ */
+int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma, const int32_t *exit_layers, int n_exit,
+                        int max_early, const double *u, int eos_id, int32_t *out, int32_t *n_out, orc_stats *st) {
+    const orc_config *c = &s->m->c;
+    const int L = c->n_layers, d = c->d_model, V = c->vocab;
+    if (max_early < 0 || max_early > ORC_MAX_INFLIGHT) return -5;
+    if (s->n_inflight) return -3;
+    if (!(temperature > 0.0) || n_exit > ORC_NU - 3 || !u) return -7;
+    for (int e = 0; e < n_exit; ++e) {
+        if (exit_layers[e] < 1 || exit_layers[e] >= L || !s->m->has_head[exit_layers[e]]) return -6;
+        if (e && exit_layers[e] <= exit_layers[e - 1]) return -6;
+    }
+    int target_len = s->n_prompt + s->n_reported + n;
+    if (target_len + 1 > s->max_seq) return -4;
+    if (eos_id >= 0 && s->len >= 1 && s->len <= target_len && s->tokens[s->len - 1] == eos_id) target_len = s->len;
+
+    int32_t(*P)[ORC_MAX_INFLIGHT + 1] = calloc(L + 1, sizeof(*P));
+    int32_t *Pn = (int32_t *)calloc(L + 1, sizeof(int32_t));
+    double *H = (double *)malloc(sizeof(double) * (ORC_MAX_INFLIGHT + 1) * d);
+    double *z = (double *)malloc(sizeof(double) * V);
+    double *pstar = (double *)malloc(sizeof(double) * V), *res = (double *)malloc(sizeof(double) * V);
+    double *Q = (double *)malloc(sizeof(double) * (size_t)(max_early + 1) * V); /* q of every early token in flight */
+    int rc = 0;
+    int64_t step_no = st ? st->steps : 0;
+
+    while (!(s->n_inflight == 0 && s->len >= target_len)) {
+        const int pos_new = s->len - 1;
+        double *h_new = s->inflight_h + (size_t)s->n_inflight * d;
+        embed(s->m, s->tokens[pos_new], h_new);
+        int exited = 0;
+        for (int l = 1; l <= L && !exited; ++l) {
+            P[l][Pn[l]++] = pos_new;
+            int n_rows = Pn[l], pos0 = P[l][0];
+            for (int r = 0; r < n_rows; ++r) {
+                if (P[l][r] != pos0 + r) { rc = -20; goto done; }
+                int slot = P[l][r] == pos_new ? s->n_inflight : P[l][r] - s->inflight_pos[0];
+                if (slot < 0 || slot > s->n_inflight) { rc = -21; goto done; }
+                if (slot < s->n_inflight && (s->inflight_pos[slot] != P[l][r] || s->inflight_depth[slot] != l - 1)) { rc = -22; goto done; }
+                memcpy(H + (size_t)r * d, s->inflight_h + (size_t)slot * d, sizeof(double) * d);
+            }
+            rc = layer_forward(s, l - 1, pos0, n_rows, H);
+            if (rc) goto done;
+            for (int r = 0; r < n_rows; ++r) {
+                int slot = P[l][r] == pos_new ? s->n_inflight : P[l][r] - s->inflight_pos[0];
+                memcpy(s->inflight_h + (size_t)slot * d, H + (size_t)r * d, sizeof(double) * d);
+                if (slot < s->n_inflight) s->inflight_depth[slot] = l;
+            }
+            if (st) st->row_layers += n_rows;
+            if (l < L) Pn[l] = 0;
+
+            int exit_idx = -1;
+            for (int e = 0; e < n_exit; ++e) if (exit_layers[e] == l) exit_idx = e;
+            if (l < L && exit_idx >= 0 && s->n_inflight < max_early && s->len < target_len) {
+                /* Eq. 1: t ~ q, emitted iff q(t) > gamma */
+                double pbest;
+                double *q = Q + (size_t)s->n_inflight * V;
+                head_eval(s->m, l, h_new, &pbest, z);
+                softmax_t(z, V, temperature, q);
+                const int tok = draw(q, V, u[(size_t)s->len * ORC_NU + 3 + exit_idx]);
+                if (st) st->head_evals++;
+                if (s->head_sink) {
+                    if (s->head_n < s->head_cap) {
+                        double *hs = s->head_sink + 4 * (size_t)s->head_n;
+                        hs[0] = (double)step_no; hs[1] = l; hs[2] = tok; hs[3] = q[tok];
+                    }
+                    s->head_n++;
+                }
+                if (q[tok] > gamma) {
+                    s->tokens[s->len++] = tok;
+                    for (int l2 = l + 1; l2 <= L; ++l2) P[l2][Pn[l2]++] = pos_new;
+                    s->inflight_pos[s->n_inflight] = pos_new;
+                    s->inflight_depth[s->n_inflight] = l;
+                    s->n_inflight++;
+                    if (st) { st->early_exits++; st->exits_at_layer[l]++; }
+                    exited = 1;
+                }
+            }
+            if (l == L) {
+                /* Eq. 2: row r holds the token at position pos0 + r; the token after it (position pos0 + r + 1) was
+                   drawn from Q[r] when row r left at its exit layer */
+                int first_bad = -1;
+                for (int r = 0; r + 1 < n_rows && first_bad < 0; ++r) {
+                    const int pos_t = pos0 + r + 1, t = s->tokens[pos_t];
+                    const double *q = Q + (size_t)r * V;
+                    final_logits(s->m, H + (size_t)r * d, z);
+                    softmax_t(z, V, temperature, pstar);
+                    record_logits(s, z);
+                    if (u[(size_t)pos_t * ORC_NU + 1] * q[t] < pstar[t]) continue; /* accepted with probability min{1, p*(t)/q(t)} */
+                    first_bad = r;
+                    double mass = 0.0;
+                    for (int v = 0; v < V; ++v) { res[v] = pstar[v] > q[v] ? pstar[v] - q[v] : 0.0; mass += res[v]; }
+                    s->tokens[pos_t] = draw(mass > 0.0 ? res : pstar, V, u[(size_t)pos_t * ORC_NU + 2]);
+                    if (st) {
+                        st->accepted += r;
+                        st->rejected += 1;
+                        st->discarded += (n_rows - 1) - r - 1;
+                    }
+                    s->len = pos_t + 1;
+                    for (int l2 = 0; l2 < L; ++l2) if (s->kv_len[l2] > pos_t) s->kv_len[l2] = pos_t;
+                }
+                if (first_bad < 0) {
+                    if (st) st->accepted += n_rows - 1;
+                    final_logits(s->m, H + (size_t)(n_rows - 1) * d, z);
+                    softmax_t(z, V, temperature, pstar);
+                    record_logits(s, z);
+                    s->tokens[s->len] = draw(pstar, V, u[(size_t)s->len * ORC_NU + 0]);
+                    s->len++;
+                }
+                Pn[L] = 0;
+                s->n_inflight = 0;
+                if (st) st->verify_steps++;
+                if (eos_id >= 0)
+                    for (int q2 = pos0 + 1; q2 < s->len; ++q2)
+                        if (s->tokens[q2] == eos_id) { if (q2 + 1 < target_len) target_len = q2 + 1; break; }
+            }
+        }
+        if (st) st->steps++;
+        step_no++;
+        for (int l2 = 1; l2 < L; ++l2) if (s->kv_len[l2] > s->kv_len[l2 - 1]) { rc = -23; goto done; }
+    }
+    if (s->len > target_len) {
+        if (st) st->truncated += s->len - target_len;
+        s->len = target_len;
+        for (int l2 = 0; l2 < L; ++l2) if (s->kv_len[l2] > target_len - 1) s->kv_len[l2] = target_len - 1;
+    }
+    {
+        int got = s->len - (s->n_prompt + s->n_reported);
+        if (got > n) got = n;
+        report(s, got, out);
+        for (int i = got; i < n; ++i) out[i] = eos_id;
+        if (n_out) *n_out = got;
+    }
+done:
+    free(P); free(Pn); free(H); free(z); free(pstar); free(res); free(Q);
     return rc;
 }
