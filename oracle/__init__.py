@@ -87,7 +87,8 @@ def _lib():
                                           C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_int32),
                                           C.POINTER(Stats)]
         L.orc_sampling_decode.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p, C.c_int, C.c_int,
-                                          C.c_void_p, C.c_int, C.c_void_p, C.POINTER(C.c_int32), C.POINTER(Stats)]
+                                          C.c_void_p, C.c_int, C.c_void_p, C.POINTER(C.c_int32), C.POINTER(Stats),
+                                          C.POINTER(C.c_double)]
         _LIB = L
     return _LIB
 
@@ -287,12 +288,14 @@ class Session:
         ex = np.ascontiguousarray(np.asarray(exit_layers, dtype=np.int32))
         u = np.ascontiguousarray(np.asarray(uniforms, dtype=np.float64))
         assert u.ndim == 2 and u.shape[1] == NU and u.shape[0] >= self.max_seq
+        margin = C.c_double(1.0)
         rc = _lib().orc_sampling_decode(self.h, n, temperature, gamma, ex.ctypes.data, len(ex), max_early,
                                         u.ctypes.data, eos_id, out.ctypes.data, C.byref(got),
-                                        C.byref(stats) if stats is not None else None)
+                                        C.byref(stats) if stats is not None else None, C.byref(margin))
         if rc:
             raise RuntimeError(f"orc_sampling_decode -> {rc}")
         self.emitted = got.value
+        self.min_margin = margin.value   # smallest distance (in probability) of any random decision of the call from flipping
         return out
 
     def __del__(self):

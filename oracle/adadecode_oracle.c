@@ -664,14 +664,23 @@ static void softmax_t(const double *z, int V, double temperature, double *p) {
 
 /* Inverse-CDF draw in vocabulary order from the non-negative weights w: the first token whose running
    sum exceeds u x (sum of all weights); the last token of non-zero weight if rounding leaves none. */
-static int draw(const double *w, int V, double u) {
+static int draw(const double *w, int V, double u, double *margin) {
     double total = 0.0, run = 0.0;
     int last = 0;
     for (int t = 0; t < V; ++t) total += w[t];
     for (int t = 0; t < V; ++t) {
         if (w[t] > 0.0) last = t;
         run += w[t];
-        if (run > u * total) return t;
+        if (run > u * total) {
+            /* how far u is from the two ends of the token's interval of the CDF: a caller comparing with a
+               lower-precision implementation can tell a decision that rounding could flip */
+            if (margin) {
+                double lo = u - (run - w[t]) / total, hi = run / total - u;
+                if (t > 0 && lo < *margin) *margin = lo;
+                if (hi < *margin) *margin = hi;
+            }
+            return t;
+        }
     }
     return last;
 }
@@ -701,7 +710,8 @@ static int draw(const double *w, int V, double u) {
  * which the tests compute independently and compare with the frequencies this function produces.
  */
 int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma, const int32_t *exit_layers, int n_exit,
-                        int max_early, const double *u, int eos_id, int32_t *out, int32_t *n_out, orc_stats *st) {
+                        int max_early, const double *u, int eos_id, int32_t *out, int32_t *n_out, orc_stats *st,
+                        double *min_margin /* nullable: smallest distance, in probability, of any decision from flipping */) {
     const orc_config *c = &s->m->c;
     const int L = c->n_layers, d = c->d_model, V = c->vocab;
     if (max_early < 0 || max_early > ORC_MAX_INFLIGHT) return -5;
@@ -723,6 +733,7 @@ int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma,
     double *Q = (double *)malloc(sizeof(double) * (size_t)(max_early + 1) * V); /* q of every early token in flight */
     int rc = 0;
     int64_t step_no = st ? st->steps : 0;
+    double margin = 1.0;
 
     while (!(s->n_inflight == 0 && s->len >= target_len)) {
         const int pos_new = s->len - 1;
@@ -757,7 +768,8 @@ int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma,
                 double *q = Q + (size_t)s->n_inflight * V;
                 head_eval(s->m, l, h_new, &pbest, z);
                 softmax_t(z, V, temperature, q);
-                const int tok = draw(q, V, u[(size_t)s->len * ORC_NU + 3 + exit_idx]);
+                const int tok = draw(q, V, u[(size_t)s->len * ORC_NU + 3 + exit_idx], &margin);
+                if (fabs(q[tok] - gamma) < margin) margin = fabs(q[tok] - gamma);
                 if (st) st->head_evals++;
                 if (s->head_sink) {
                     if (s->head_n < s->head_cap) {
@@ -786,11 +798,15 @@ int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma,
                     final_logits(s->m, H + (size_t)r * d, z);
                     softmax_t(z, V, temperature, pstar);
                     record_logits(s, z);
+                    {
+                        const double gap = fabs(u[(size_t)pos_t * ORC_NU + 1] - pstar[t] / q[t]);
+                        if (pstar[t] < q[t] && gap < margin) margin = gap;
+                    }
                     if (u[(size_t)pos_t * ORC_NU + 1] * q[t] < pstar[t]) continue; /* accepted with probability min{1, p*(t)/q(t)} */
                     first_bad = r;
                     double mass = 0.0;
                     for (int v = 0; v < V; ++v) { res[v] = pstar[v] > q[v] ? pstar[v] - q[v] : 0.0; mass += res[v]; }
-                    s->tokens[pos_t] = draw(mass > 0.0 ? res : pstar, V, u[(size_t)pos_t * ORC_NU + 2]);
+                    s->tokens[pos_t] = draw(mass > 0.0 ? res : pstar, V, u[(size_t)pos_t * ORC_NU + 2], &margin);
                     if (st) {
                         st->accepted += r;
                         st->rejected += 1;
@@ -804,7 +820,7 @@ int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma,
                     final_logits(s->m, H + (size_t)(n_rows - 1) * d, z);
                     softmax_t(z, V, temperature, pstar);
                     record_logits(s, z);
-                    s->tokens[s->len] = draw(pstar, V, u[(size_t)s->len * ORC_NU + 0]);
+                    s->tokens[s->len] = draw(pstar, V, u[(size_t)s->len * ORC_NU + 0], &margin);
                     s->len++;
                 }
                 Pn[L] = 0;
@@ -832,6 +848,7 @@ int orc_sampling_decode(orc_session *s, int n, double temperature, double gamma,
         if (n_out) *n_out = got;
     }
 done:
+    if (min_margin) *min_margin = margin;
     free(P); free(Pn); free(H); free(z); free(pstar); free(res); free(Q);
     return rc;
 }

@@ -2,6 +2,7 @@
 oracle) and small conveniences.  Nothing here is imported by the oracle or the CUDA path."""
 
 import numpy as np
+from scipy import stats as sps
 import torch
 
 from paper_2506_03700_b200 import synth
@@ -73,3 +74,51 @@ def make_oracle(cfg, seed=1234, tied=True, jitter=0.05, heads=True, scale=None, 
         for l in cfg.exit_layers:
             m.set_head(l, None, cfg.logit_scale if scale is None else scale)
     return w, m
+
+
+# ---- sampled decoding: the closed-form law of a verified token, from the oracle's forward pass alone
+
+def tempered(p, temperature):
+    w = np.power(p, 1.0 / temperature)
+    return w / w.sum()
+
+
+def head_and_final_distributions(cfg, m, tokens, temperature):
+    """q_i (one per exit layer) and p* for the successor of tokens[-1], from the oracle's forward pass only."""
+    qs = []
+    for l in cfg.exit_layers:
+        h = m.hidden_after(tokens, l)
+        _, _, probs = m.head_eval(l, h, want_probs=True)
+        qs.append(tempered(np.asarray(probs), temperature))
+    z = m.full_logits(tokens)[-1]
+    p = np.exp((z - z.max()) / temperature)
+    return qs, p / p.sum()
+
+
+def law_of_a_verified_token(qs, pstar, gamma):
+    """Law of the verified successor when every exit head is consulted in turn (derivation: a head's draw t is
+    used iff q(t) > gamma, then accepted with probability min(1, p*(t)/q(t)) or replaced by a draw from the
+    normalised positive part of p* - q; if no head emits, the token is drawn from p*)."""
+    out = np.zeros_like(pstar)
+    reach = 1.0
+    for q in qs:
+        emit = q > gamma
+        acc = np.where(emit, np.minimum(q, pstar), 0.0)
+        rej_mass = np.where(emit, q - np.minimum(q, pstar), 0.0).sum()
+        res = np.maximum(0.0, pstar - q)
+        res = res / res.sum() if res.sum() > 0 else pstar
+        out += reach * (acc + rej_mass * res)
+        reach *= 1.0 - q[emit].sum()
+    return out + reach * pstar
+
+
+def chi2_ok(counts, law, alpha=1e-4):
+    n = counts.sum()
+    exp = law * n
+    big = exp >= 5
+    obs = np.append(counts[big], counts[~big].sum())
+    ex = np.append(exp[big], exp[~big].sum())
+    if ex[-1] == 0:
+        obs, ex = obs[:-1], ex[:-1]
+    stat = ((obs - ex) ** 2 / ex).sum()
+    return stat <= sps.chi2.ppf(1 - alpha, len(ex) - 1), stat

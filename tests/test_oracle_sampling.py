@@ -12,7 +12,7 @@ from scipy import stats as sps
 
 import oracle
 from paper_2506_03700_b200 import synth
-from helpers import make_oracle
+from helpers import make_oracle, head_and_final_distributions as _distributions, law_of_a_verified_token as _law, chi2_ok as _chi2_ok
 
 
 def _mini(**kw):
@@ -20,52 +20,6 @@ def _mini(**kw):
                 resid_scale=1.0, exit_layers=(1, 2), logit_scale=3.0, sigma=0.25)
     base.update(kw)
     return synth.small_config(name="mini-sampling", **base)
-
-
-def _tempered(p, temperature):
-    w = np.power(p, 1.0 / temperature)
-    return w / w.sum()
-
-
-def _distributions(cfg, m, tokens, temperature):
-    """q_i (one per exit layer) and p* for the successor of tokens[-1], from the oracle's forward pass only."""
-    qs = []
-    for l in cfg.exit_layers:
-        h = m.hidden_after(tokens, l)
-        _, _, probs = m.head_eval(l, h, want_probs=True)
-        qs.append(_tempered(np.asarray(probs), temperature))
-    z = m.full_logits(tokens)[-1]
-    p = np.exp((z - z.max()) / temperature)
-    return qs, p / p.sum()
-
-
-def _law(qs, pstar, gamma):
-    """Law of the verified successor when every exit head is consulted in turn (derivation: a head's draw t is
-    used iff q(t) > gamma, then accepted with probability min(1, p*(t)/q(t)) or replaced by a draw from the
-    normalised positive part of p* - q; if no head emits, the token is drawn from p*)."""
-    out = np.zeros_like(pstar)
-    reach = 1.0
-    for q in qs:
-        emit = q > gamma
-        acc = np.where(emit, np.minimum(q, pstar), 0.0)
-        rej_mass = np.where(emit, q - np.minimum(q, pstar), 0.0).sum()
-        res = np.maximum(0.0, pstar - q)
-        res = res / res.sum() if res.sum() > 0 else pstar
-        out += reach * (acc + rej_mass * res)
-        reach *= 1.0 - q[emit].sum()
-    return out + reach * pstar
-
-
-def _chi2_ok(counts, law, alpha=1e-4):
-    n = counts.sum()
-    exp = law * n
-    big = exp >= 5
-    obs = np.append(counts[big], counts[~big].sum())
-    ex = np.append(exp[big], exp[~big].sum())
-    if ex[-1] == 0:
-        obs, ex = obs[:-1], ex[:-1]
-    stat = ((obs - ex) ** 2 / ex).sum()
-    return stat <= sps.chi2.ppf(1 - alpha, len(ex) - 1), stat
 
 
 def _sample_second_token(cfg, m, prompt, temperature, gamma, runs, seed, exit_layers=None, max_early=3):
