@@ -163,6 +163,27 @@ int ada_plain_decode(ada_session *s, int32_t n_tokens, int32_t eos_id, int32_t *
 int ada_adaptive_decode(ada_session *s, int32_t n_tokens, float threshold, const int32_t *exit_layers,
                         int32_t n_exit_layers, int32_t max_early, int32_t eos_id, int32_t *out_host, ada_stats *stats);
 
+/* Algorithm 1 with SAMPLED tokens (Eq. 1: "any sampling strategy can be employed"; here: the softmax of the head's logits
+ * over `temperature` > 0) and the stochastic form of Eq. 2.  At an exit layer the successor t of the newest token is
+ * drawn from the head's distribution q and emitted early iff q(t) > threshold.  At the last layer every early-predicted
+ * token, in sequence order, is accepted with probability min{1, p*(t) / q(t)} (p* = the full model's distribution at
+ * the same temperature); the first one that is not is replaced by a draw from Normalize(max(0, p* - q)), the K/V of
+ * everything from its position on is dropped and generation resumes from the replacement; if all are accepted the next
+ * token is drawn from p*.  n_exit_layers = 0 is plain sampling.  Draws are inverse-CDF draws in vocabulary order.
+ *
+ * Every random number is an input (nothing is generated inside the library): uniforms_host[batch][n_pos][8], fp32 in
+ * [0, 1), row j of a sequence belonging to the token at sequence position first_pos + j (prompt included):
+ * [0] its draw at the last layer, [1] its acceptance test, [2] its resampling, [3 + e] its draw at the e-th exit layer
+ * of the call (at most 5 exit layers).  A position drawn again after a rollback uses its numbers again.  Rows must cover
+ * every position from each sequence's current length to one past the call's last token; ADA_EINVAL otherwise.
+ * With threshold 0 the verified tokens are distributed exactly as plain sampling; for threshold > 0 the draft is
+ * consulted only where q(t) > threshold and the law differs slightly from p* (the paper states the rule, not this
+ * consequence).  The first token after the prompt is the prompt pass's argmax.  Persistent decode path only
+ * (ADA_EUNSUPPORTED otherwise); end-of-sequence handling, return layout and statistics as for ada_adaptive_decode. */
+int ada_sampling_decode(ada_session *s, int32_t n_tokens, float temperature, float threshold, const int32_t *exit_layers,
+                        int32_t n_exit_layers, int32_t max_early, int32_t eos_id, const float *uniforms_host,
+                        int32_t first_pos, int32_t n_pos, int32_t *out_host, ada_stats *stats);
+
 /* ---- test hooks --------------------------------------------------------------------------- */
 
 /* Record the final-layer logits of every verified generated token of sequence 0 into dev_buf

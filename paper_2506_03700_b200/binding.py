@@ -22,6 +22,8 @@ ADA_MAX_BATCH = 16
 ERRORS = {0: "ADA_OK", -1: "ADA_EINVAL", -2: "ADA_ESTATE", -3: "ADA_ECAPACITY", -4: "ADA_ECUDA",
           -5: "ADA_ETIMEOUT", -6: "ADA_EUNSUPPORTED"}
 
+SAMPLE_NU = 8   # random numbers per sequence position of a sampling decode call
+
 EXPORTS = [
     "ada_strerror", "ada_last_cuda_error", "ada_model_create", "ada_model_set_tensor", "ada_model_set_exit_head",
     "ada_model_finalize", "ada_model_destroy", "ada_session_scratch_bytes", "ada_kv_page_bytes",
@@ -30,7 +32,7 @@ EXPORTS = [
     "ada_debug_set_exit_tape", "ada_debug_get_state", "ada_debug_read_kv", "ada_debug_set_path",
     "ada_debug_profile", "ada_debug_profile_read", "ada_debug_gemm", "ada_debug_gemm_plan", "ada_debug_gemm_work_bytes", "ada_debug_get_path", "ada_debug_set_launch_steps", "ada_debug_trace", "ada_gemm_noalloc",
     "ada_model_arena_bytes", "ada_model_set_arena", "ada_debug_set_wait_limit", "ada_debug_set_prefill",
-    "ada_debug_dense_gemm", "ada_debug_dense_gemm_work_bytes",
+    "ada_debug_dense_gemm", "ada_debug_dense_gemm_work_bytes", "ada_sampling_decode",
 ]
 
 
@@ -108,6 +110,7 @@ def load() -> C.CDLL:
         L.ada_prefill.argtypes = [vp, i32, vp, i32]
         L.ada_plain_decode.argtypes = [vp, i32, i32, vp, C.POINTER(Stats)]
         L.ada_adaptive_decode.argtypes = [vp, i32, C.c_float, vp, i32, i32, i32, vp, C.POINTER(Stats)]
+        L.ada_sampling_decode.argtypes = [vp, i32, C.c_float, C.c_float, vp, i32, i32, i32, vp, i32, i32, vp, C.POINTER(Stats)]
         L.ada_debug_capture_logits.argtypes = [vp, vp, i32]
         L.ada_debug_logits_captured.argtypes = [vp, C.POINTER(i32)]
         L.ada_debug_capture_heads.argtypes = [vp, vp, i32, C.POINTER(i32)]
@@ -297,6 +300,20 @@ class Session:
         _ck(load().ada_adaptive_decode(self.h, n_tokens, threshold, ex.ctypes.data if len(ex) else None, len(ex),
                                        max_early, eos_id, out.ctypes.data, C.byref(stats) if stats is not None else None),
             "ada_adaptive_decode")
+        return out
+
+    def sampling_decode(self, n_tokens: int, temperature: float, threshold: float, exit_layers: Sequence[int],
+                        max_early: int, uniforms: np.ndarray, first_pos: int = 0, stats: Optional[Stats] = None,
+                        out: Optional[np.ndarray] = None, eos_id: int = -1) -> np.ndarray:
+        """`uniforms`: float32 [batch][n_pos][SAMPLE_NU], row j = the random numbers of sequence position first_pos + j."""
+        out = np.empty((self.batch, n_tokens), dtype=np.int32) if out is None else out
+        ex = np.ascontiguousarray(np.asarray(exit_layers, dtype=np.int32))
+        u = np.ascontiguousarray(uniforms, dtype=np.float32)
+        if u.ndim != 3 or u.shape[0] != self.batch or u.shape[2] != SAMPLE_NU:
+            raise ValueError("uniforms must be [batch][n_pos][%d]" % SAMPLE_NU)
+        _ck(load().ada_sampling_decode(self.h, n_tokens, temperature, threshold, ex.ctypes.data if len(ex) else None, len(ex),
+                                       max_early, eos_id, u.ctypes.data, first_pos, u.shape[1], out.ctypes.data,
+                                       C.byref(stats) if stats is not None else None), "ada_sampling_decode")
         return out
 
     # ---- test hooks

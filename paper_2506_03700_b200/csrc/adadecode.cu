@@ -142,6 +142,8 @@ struct ada_session {
     CUtensorMap *maps_dev = nullptr;      // [6 L + 2]: wqkv, wo, wgu, wup, wdown per layer, lm_head, then T per 1-based layer
     mg::MegaModel *mm_dev = nullptr;
     int *exit_at_dev = nullptr;
+    bool sampling = false;   // the call in progress draws its tokens (ada_sampling_decode)
+    float inv_temp = 1.0f;
     int steps_per_launch = 256;
     unsigned long long wait_ns = st::WAIT_NS_DEFAULT;
     // dense prompt pass (tcgen05 GEMMs over blocks of up to 128 positions)
@@ -176,7 +178,7 @@ namespace {
 struct Layout {
     size_t st, rt, fill, tokens, page_table, head_res, resid, xn, qkv, q, attn_out, gu, hact, rope_cs, attn_part,
         head_part, logit_stage, head_log, t_out, pf_hi, pf_lo, pf_err, pf_part, maps, mm, exit_at, xa, xb, xo, xh, xf, xt, ssq_a, ssq_b, qfrag, attn_cnt, rope_freq, part,
-        grid_ctr, pub, err, total;
+        grid_ctr, pub, err, q_stage, qinfo, uniforms, total;
 };
 
 bool model_fits_persistent(const ada_config &g);
@@ -244,6 +246,11 @@ Layout make_layout(const ada_config &g, int batch, int max_seq, int max_early, i
         L.grid_ctr = take(256);
         L.pub = take(sizeof(mg::Pub) * 2);
         L.err = take(256);
+        // sampled decoding: the logits and normalisers of the intermediate head that drew each token in flight, and the
+        // random numbers of every sequence position
+        L.q_stage = take(sizeof(float) * (size_t)batch * st::MAX_COLS * g.vocab);
+        L.qinfo = take(sizeof(float4) * (size_t)batch * st::MAX_COLS);
+        L.uniforms = take(sizeof(float) * (size_t)batch * max_seq * mg::SAMPLE_NU);
     }
     L.total = o;
     return L;
@@ -697,6 +704,11 @@ int setup_persistent(ada_session *S, const Layout &lay) {
     a.nseq = 1;
     a.wait_ns = S->wait_ns;
     a.store_logits = 0;
+    a.sampling = 0;
+    a.inv_temp = 1.0f;
+    a.uniforms = (const float *)(b + lay.uniforms);
+    a.q_stage = (float *)(b + lay.q_stage);
+    a.qinfo = (float4 *)(b + lay.qinfo);
     a.trace = st::Trace{nullptr, nullptr, 0};
     a.trace_step0 = a.trace_step1 = 0;
     S->mega = true;
@@ -718,7 +730,7 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
     if (!plain) {
         for (int i = 0; i < n_exit; ++i) {
             const int e = exit_layers[i];
-            ex[e] = 1;
+            ex[e] = 1 + i;
             M.layer[e].has_head = 1;
             M.layer[e].head_scale = m->head_scale[e];
             M.layer[e].wT = nullptr;
@@ -748,6 +760,8 @@ int run_persistent(ada_session *S, const int32_t *exit_layers, int n_exit, bool 
         a.step_budget = S->steps_per_launch;
         a.wait_ns = S->wait_ns;
         a.store_logits = (S->capture_dev && sq == 0) ? 1 : 0;
+        a.sampling = S->sampling ? 1 : 0;
+        a.inv_temp = S->sampling ? S->inv_temp : 1.0f;
         CK(cudaMemsetAsync(&S->c.st->n_done, 0, sizeof(int32_t), S->stream));
         for (long long guard = 0;; ++guard) {
             if (guard > (1ll << 24)) return ADA_ETIMEOUT;
@@ -1307,6 +1321,30 @@ int ada_adaptive_decode(ada_session *S, int32_t n_tokens, float threshold, const
                         int32_t n_exit_layers, int32_t max_early, int32_t eos_id, int32_t *out_host, ada_stats *stats) {
     if (!S || n_exit_layers < 0 || (n_exit_layers > 0 && !exit_layers)) return ADA_EINVAL;
     return decode(S, n_tokens, threshold, exit_layers, n_exit_layers, max_early, eos_id, out_host, stats);
+}
+
+int ada_sampling_decode(ada_session *S, int32_t n_tokens, float temperature, float threshold, const int32_t *exit_layers,
+                        int32_t n_exit_layers, int32_t max_early, int32_t eos_id, const float *uniforms_host, int32_t first_pos,
+                        int32_t n_pos, int32_t *out_host, ada_stats *stats) {
+    if (!S || n_exit_layers < 0 || (n_exit_layers > 0 && !exit_layers) || !uniforms_host) return ADA_EINVAL;
+    if (!(temperature > 0.0f) || first_pos < 0 || n_pos < 1 || first_pos + (int64_t)n_pos > S->max_seq) return ADA_EINVAL;
+    if (n_exit_layers > mg::SAMPLE_NU - 3) return ADA_ECAPACITY;
+    if (!(S->mega && S->path == 1) || S->m->cfg.vocab > mg::DRAW_MAX_VOCAB) return ADA_EUNSUPPORTED;
+    // every position the call may draw, test or resample must have its random numbers
+    for (int s = 0; s < S->batch; ++s) {
+        if (!S->prefilled[s]) return ADA_ESTATE;
+        if (S->finished[s]) continue;
+        if (S->h_len[s] < first_pos || S->h_prompt[s] + S->h_reported[s] + n_tokens + 1 > first_pos + n_pos) return ADA_EINVAL;
+    }
+    float *dev = const_cast<float *>(S->margs.uniforms);
+    for (int s = 0; s < S->batch; ++s)
+        CK(cudaMemcpyAsync(dev + ((size_t)s * S->max_seq + first_pos) * mg::SAMPLE_NU, uniforms_host + (size_t)s * n_pos * mg::SAMPLE_NU,
+                           sizeof(float) * (size_t)n_pos * mg::SAMPLE_NU, cudaMemcpyHostToDevice, S->stream));
+    S->sampling = true;
+    S->inv_temp = 1.0f / temperature;
+    const int rc = decode(S, n_tokens, threshold, exit_layers, n_exit_layers, max_early, eos_id, out_host, stats);
+    S->sampling = false;
+    return rc;
 }
 
 int ada_debug_set_wait_limit(ada_session *S, uint64_t ns) {

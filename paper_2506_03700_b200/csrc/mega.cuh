@@ -73,7 +73,7 @@ struct MegaModel {
 struct MegaArgs {
     Ctx c;
     const MegaModel *mm;
-    const int *exit_at;        // [L + 1]: 1 if this call consults the head after 1-based layer e
+    const int *exit_at;        // [L + 1]: 1 + the index of 1-based layer e among the call's exit layers if the call consults its head, else 0
     __nv_bfloat16 *XA, *XB, *XO, *XH, *XF, *XT;   // GEMM inputs in fragment layout (see stream.cuh)
     float *ssq_a, *ssq_b;      // [d/16][8] partial sums of squares of the residual (per 16-feature tile, per column)
     uint32_t *qfrag;           // [nkv][2][hd/16][32][8]: rotated, scaled queries as tensor-core A fragments (bf16 high parts, then low parts)
@@ -90,6 +90,12 @@ struct MegaArgs {
                                // token columns [k slots, (k + 1) slots), slots = max_early + 1, nseq slots <= 8; they share every weight stream
     unsigned long long wait_ns;   // a single device-side wait gives up after this long
     int store_logits;
+    // Sampled decoding (Eq. 1 with a drawn token, Eq. 2 with its acceptance test and the resampling): off = greedy
+    int sampling;
+    float inv_temp;            // 1 / temperature: every head's logits are multiplied by it
+    const float *uniforms;     // [batch][max_seq][SAMPLE_NU]: the random numbers of the token at each sequence position
+    float *q_stage;            // [batch][8][vocab]: logits of the intermediate head that drew the token after position p, slot p % 8
+    float4 *qinfo;             // [batch][8]: (max logit, sum of exp, probability of the drawn token) of that head
     Trace trace;               // test hook: event trace of the steps [trace_step0, trace_step1) of this launch
     int trace_step0, trace_step1;
 };
@@ -178,6 +184,199 @@ __device__ __forceinline__ HeadResult merge_head(const float *head_part, int G, 
     return hr;
 }
 
+// ---------------------------------------------------------------- sampling (CTA 0, consumer warps)
+
+// Random numbers per sequence position: [0] draw at the last layer, [1] acceptance test of Eq. 2, [2] resampling after a
+// rejection, [3 + e] draw at the e-th exit layer of the call.
+constexpr int SAMPLE_NU = 8;
+constexpr int DRAW_CHUNK = 128;                 // vocabulary entries per partial sum
+constexpr int DRAW_OFFSET = 12288;              // the draw's buffers sit in the consumers' scratch behind the control point's copies
+constexpr int DRAW_MAX_CHUNKS = (SCRATCH_BYTES - DRAW_OFFSET - 4 * (CONS_THREADS + DRAW_CHUNK + 8)) / 4;
+constexpr int DRAW_MAX_VOCAB = DRAW_MAX_CHUNKS * DRAW_CHUNK;
+
+// Weights the draw is made from, in vocabulary order: exp(z - m) (a head's distribution up to its normaliser), or, with
+// zq set, the positive part of exp(z - m) / s - exp(zq - mq) / sq (the distribution Eq. 2 resamples from, up to its normaliser).
+struct DrawSrc {
+    const float *z; float m, inv_s;
+    const float *zq; float mq, inv_sq;
+    __device__ __forceinline__ float weight(int v) const {
+        const float a = __expf(__ldcg(z + v) - m);
+        if (!zq) return a;
+        return fmaxf(0.f, a * inv_s - __expf(__ldcg(zq + v) - mq) * inv_sq);
+    }
+};
+
+// Inverse-CDF draw by the consumer warps of one CTA: the first token, in vocabulary order, whose running sum of weights
+// exceeds u x (sum of all weights); the last token of non-zero weight if rounding leaves none.  Returns the token to every
+// thread (-1 if all weights are zero), with the sum of all weights and the drawn token's weight.  Partial sums per 128
+// entries in a fixed order, so the result does not depend on timing.
+__device__ __forceinline__ int block_draw(Smem *sm, const DrawSrc &src, int V, float u, float &total, float &w_tok) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    float *psum = reinterpret_cast<float *>(sm->scratch + DRAW_OFFSET);   // [CONS_THREADS]
+    float *wbuf = psum + CONS_THREADS;                                     // [DRAW_CHUNK]
+    float *res = wbuf + DRAW_CHUNK;                                        // token, its weight
+    float *csum = res + 8;                                                 // [chunks]
+    const int n_chunks = (V + DRAW_CHUNK - 1) / DRAW_CHUNK;
+    // pass 1: the sum of every chunk (warp w takes chunks w, w + 8, ...; eight chunks' loads in flight)
+    for (int c0 = warp; c0 < n_chunks; c0 += CONS_WARPS * 8) {
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int ch = c0 + j * CONS_WARPS;
+            float a = 0.f;
+            if (ch < n_chunks) {
+#pragma unroll
+                for (int it = 0; it < DRAW_CHUNK / 32; ++it) {
+                    const int v = ch * DRAW_CHUNK + it * 32 + lane;
+                    a += v < V ? src.weight(v) : 0.f;
+                }
+            }
+            acc[j] = a;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float a = acc[j];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+            const int ch = c0 + j * CONS_WARPS;
+            if (lane == 0 && ch < n_chunks) csum[ch] = a;
+        }
+    }
+    bar_consumers();
+    const int cpt = (n_chunks + CONS_THREADS - 1) / CONS_THREADS;   // chunks per thread of the second level
+    {
+        float a = 0.f;
+        for (int j = 0; j < cpt; ++j) {
+            const int ch = tid * cpt + j;
+            a += ch < n_chunks ? csum[ch] : 0.f;
+        }
+        psum[tid] = a;
+    }
+    bar_consumers();
+    // every thread walks the same two levels to the chunk that holds the crossing
+    total = 0.f;
+    for (int i = 0; i < CONS_THREADS; ++i) total += psum[i];
+    w_tok = 0.f;
+    if (!(total > 0.f)) return -1;
+    const float target = u * total;
+    float base = 0.f;
+    int t_at = -1;
+    for (int i = 0; i < CONS_THREADS; ++i) {
+        if (base + psum[i] > target) { t_at = i; break; }
+        base += psum[i];
+    }
+    int ch_at = -1;
+    bool take_last = false;
+    if (t_at >= 0) {
+        for (int j = 0; j < cpt; ++j) {
+            const int ch = t_at * cpt + j;
+            if (ch >= n_chunks) break;
+            if (base + csum[ch] > target) { ch_at = ch; break; }
+            base += csum[ch];
+        }
+    }
+    if (ch_at < 0) {   // rounding left no crossing: the last chunk of non-zero weight, its last such token
+        take_last = true;
+        for (int ch = n_chunks - 1; ch >= 0; --ch)
+            if (csum[ch] > 0.f) { ch_at = ch; break; }
+        if (ch_at < 0) return -1;
+    }
+    // pass 2: locate the token inside the chunk
+    if (warp == 0) {
+#pragma unroll
+        for (int it = 0; it < DRAW_CHUNK / 32; ++it) {
+            const int v = ch_at * DRAW_CHUNK + it * 32 + lane;
+            wbuf[it * 32 + lane] = v < V ? src.weight(v) : 0.f;
+        }
+        __syncwarp();
+        if (lane == 0) {
+            float run = base;
+            int tok = -1, last = -1;
+            for (int i = 0; i < DRAW_CHUNK; ++i) {
+                const float w = wbuf[i];
+                if (w > 0.f) last = i;
+                run += w;
+                if (!take_last && run > target) { tok = i; break; }
+            }
+            if (tok < 0) tok = last < 0 ? 0 : last;
+            res[0] = __int_as_float(ch_at * DRAW_CHUNK + tok);
+            res[1] = wbuf[tok];
+        }
+    }
+    bar_consumers();
+    const int tok = __float_as_int(res[0]);
+    w_tok = res[1];
+    bar_consumers();   // the buffers may be rewritten by the next draw
+    return tok;
+}
+
+struct SampleArgs {
+    const float *uniforms; float *q_stage; float4 *qinfo; const float *logit_stage; HeadResult *head_res; DevState *st;
+    int vocab, max_seq, cps, L, seq0, nseq, exit_idx;
+};
+
+// Sampled decoding at a control point (its own function: its registers must not weigh on the streaming loops).
+// After an intermediate head (Eq. 1): the newest token's successor is drawn from the head's distribution q; its
+// probability q(t) is what the threshold test sees.  After the final head (Eq. 2): every early-predicted token t, in
+// sequence order, is accepted with probability min{1, p*(t) / q(t)} -- the result stands in the column's head result as
+// the token itself, so that the comparison of the bookkeeping accepts it -- and the first one that is not is replaced by
+// a draw from Normalize(max(0, p* - q)); if all are accepted the next token is drawn from p* of the newest column.
+__device__ __noinline__ void sample_stage(SampleArgs a, Smem *sm, bool after_head, const StepDesc *dprev, unsigned head_cols) {
+    const int tid = threadIdx.x, V = a.vocab, cps = a.cps;
+    HeadResult *hr_s = reinterpret_cast<HeadResult *>(sm->scratch + 8192);
+    const int *tok_s = reinterpret_cast<const int *>(sm->scratch + 8192 + sizeof(HeadResult) * MAX_COLS);
+    auto unif = [&](int s, int pos, int which) { return a.uniforms[((size_t)s * a.max_seq + pos) * SAMPLE_NU + which]; };
+    if (after_head) {
+        for (int col = 0; col < MAX_COLS; ++col) {
+            if (!((head_cols >> col) & 1u)) continue;
+            const int s = a.seq0 + (a.nseq == 1 ? 0 : col / cps), pos = dprev->pos[col], slot = s * MAX_COLS + (pos & 7);
+            DrawSrc src{a.q_stage + (size_t)slot * V, hr_s[col].zmax, 0.f, nullptr, 0.f, 0.f};
+            float total, wt;
+            const int tok = block_draw(sm, src, V, unif(s, pos + 1, 3 + a.exit_idx), total, wt);
+            if (tid == 0) {
+                hr_s[col].token = max(tok, 0);
+                hr_s[col].p = tok < 0 ? 0.f : wt / total;
+                a.head_res[col] = hr_s[col];
+                a.qinfo[slot] = make_float4(hr_s[col].zmax, total, hr_s[col].p, 0.f);
+            }
+        }
+    } else {
+        for (int k = 0; k < a.nseq; ++k) {
+            const int s = a.seq0 + k, ln = a.st->len[s], bs = a.st->base[s], nrow = ln - bs, c0 = k * cps;
+            if (nrow < 1 || nrow > cps || dprev->first_layer[c0 + nrow - 1] > a.L - 1) continue;
+            bool rejected = false;
+            for (int r = 0; r + 1 < nrow && !rejected; ++r) {
+                const int col = c0 + r, pos_t = bs + r + 1, t = min(max(tok_s[col], 0), V - 1), slot = s * MAX_COLS + ((bs + r) & 7);
+                const float *zs = a.logit_stage + (size_t)col * V;
+                const float4 qi = a.qinfo[slot];
+                const float ps = __expf(__ldcg(zs + t) - hr_s[col].zmax) / hr_s[col].sumexp;
+                if (unif(s, pos_t, 1) * qi.z < ps) {   // accepted; every thread evaluates the same numbers
+                    if (tid == 0) hr_s[col].token = t;
+                    continue;
+                }
+                rejected = true;
+                DrawSrc src{zs, hr_s[col].zmax, 1.f / hr_s[col].sumexp, a.q_stage + (size_t)slot * V, qi.x, 1.f / qi.y};
+                float total, wt;
+                int tok = block_draw(sm, src, V, unif(s, pos_t, 2), total, wt);
+                if (tok < 0) {   // p* nowhere above q (they are equal up to rounding): draw from p*
+                    DrawSrc plain{zs, hr_s[col].zmax, 0.f, nullptr, 0.f, 0.f};
+                    tok = block_draw(sm, plain, V, unif(s, pos_t, 2), total, wt);
+                }
+                if (tid == 0) hr_s[col].token = max(tok, 0);
+            }
+            if (!rejected) {
+                const int col = c0 + nrow - 1;
+                DrawSrc src{a.logit_stage + (size_t)col * V, hr_s[col].zmax, 0.f, nullptr, 0.f, 0.f};
+                float total, wt;
+                const int tok = block_draw(sm, src, V, unif(s, ln, 0), total, wt);
+                if (tid == 0) hr_s[col].token = max(tok, 0);
+            }
+        }
+    }
+    __threadfence_block();
+    bar_consumers();
+}
+
 // ---------------------------------------------------------------- control point (CTA 0, consumer warps)
 
 // Applies the outcome of the step that just ended (Eq. 1 after a head; verification and rollback,
@@ -220,6 +419,12 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     }
     __threadfence_block();
     bar_consumers();
+    // (a') sampled decoding replaces the tokens and probabilities the bookkeeping below works with
+    if (A.sampling && kind != CTRL_START && !(kind == CTRL_TOP && st->pf_end > 0)) {
+        SampleArgs sa{A.uniforms, A.q_stage, A.qinfo, c.logit_stage, c.head_res, st, c.vocab, c.max_seq, cps, L, seq0, nseq,
+                      kind == CTRL_HEAD ? A.exit_at[e] - 1 : 0};
+        sample_stage(sa, sm, kind == CTRL_HEAD, &dprev, head_cols);
+    }
     // (b) bookkeeping, one thread.  Every scalar it may need is read up front (the loads overlap);
     // counters are bumped by reductions, which do not wait for memory.
     if (tid == 0) {
@@ -1021,7 +1226,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
         }
     };
     // head over E* with the fused (max, sum exp, argmax) reduction; X = final-normed residual (or T output)
-    auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols) {
+    auto head_phase = [&](const __nv_bfloat16 *X, const float *ssq, float scale, unsigned cols, bool inter) {
         Gemm g; g.W = M.lm_head; g.X = reinterpret_cast<const uint4 *>(X); g.N = c.vocab; g.K = d_model; g.pair = 1; g.half = 0; g.ctas = n_head; g.part = nullptr; g.phase_id = bar_no + 1; g.columns(cols);
         x_ready();
         const unsigned vseq = bar_no + 1;
@@ -1029,6 +1234,17 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
             Msa run[2];
             run[0].m = run[1].m = -INFINITY; run[0].s = run[1].s = 0.f; run[0].i = run[1].i = INT_MAX;
             const int c0 = 2 * (lane & 3);
+            // sampled decoding: logits over the temperature; they are kept, the final head's by column, an intermediate
+            // head's by the position of its row (the verification of the token drawn from them needs them again)
+            if (A.sampling) scale *= A.inv_temp;
+            float *zrow[2] = {nullptr, nullptr};
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int col = c0 + q;
+                if (!((cols >> col) & 1u)) continue;
+                if (A.sampling && inter) zrow[q] = A.q_stage + ((size_t)(A.seq0 + (A.nseq == 1 ? 0 : col / c.slots)) * MAX_COLS + (d.pos[col] & 7)) * c.vocab;
+                else if (A.sampling || A.store_logits) zrow[q] = c.logit_stage + (size_t)col * c.vocab;
+            }
             float r0 = scale, r1 = scale;
             bool have_r = ssq == nullptr;
             gemm_consume<1>(S, g, blockIdx.x, G, r, [&](int tile, float (&acc)[1][4]) {
@@ -1038,7 +1254,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                     const int n = tile * 16 + (lane >> 2) + (i >> 1) * 8;
                     if (n < c.vocab) {
                         const float z = acc[0][i] * ((i & 1) ? r1 : r0);
-                        if (A.store_logits && ((cols >> (c0 + (i & 1))) & 1u)) c.logit_stage[(size_t)(c0 + (i & 1)) * c.vocab + n] = z;
+                        if (zrow[i & 1]) zrow[i & 1][n] = z;
                         Msa one; one.m = z; one.s = 1.f; one.i = n;
                         run[i & 1] = msa_merge(run[i & 1], one);
                     }
@@ -1321,9 +1537,9 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                     } else if (ROLE == 1) gemm_produce_x(S, g, blockIdx.x, G, r, pol, [&]() { rstd_produce(sm, A.ssq_a, ntd, d_model, c.eps, vseq); });
                     else gemm_phase<ROLE, 1>(S, g, r, pol, NoEpi());
                     phase_barrier(10);
-                    head_phase(A.XT, nullptr, hl.head_scale, hcols);
+                    head_phase(A.XT, nullptr, hl.head_scale, hcols, true);
                 } else {
-                    head_phase(A.XF, A.ssq_a, hl.head_scale, hcols);
+                    head_phase(A.XF, A.ssq_a, hl.head_scale, hcols, true);
                 }
                 action = control_point<ROLE>(A, S, CTRL_HEAD, l + 1, pub_no, d, steps_started);
                 book_control();
@@ -1332,7 +1548,7 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
         }
         if (!restart) {
             // ---- final head for every column, then verification (Eq. 2 at temperature zero) in the control point
-            if (d.run_final) head_phase(A.XF, A.ssq_a, 1.0f, active_mask(d, L - 1));
+            if (d.run_final) head_phase(A.XF, A.ssq_a, 1.0f, active_mask(d, L - 1), false);
             action = control_point<ROLE>(A, S, CTRL_TOP, 0, pub_no, d, steps_started);
             book_control();
         }
