@@ -190,7 +190,7 @@ class Bench:
             self.dist.barrier()
         self.torch.cuda.synchronize()
 
-    def timed(self, mode, sizes=None, threshold=None, exit_layers=None):
+    def timed(self, mode, sizes=None, threshold=None, exit_layers=None, temperature=1.0):
         """Prefill (untimed), then one decode call per entry of `sizes`.  Returns device ms (CUDA events on
         the session stream around the calls), wall ms around the same calls, stats, tokens [batch][sum]."""
         torch, sess, cfg = self.torch, self.sess, self.cfg
@@ -209,6 +209,9 @@ class Bench:
             o = self.out[:, :n] if n == self.out.shape[1] else np.empty((self.batch, n), dtype=np.int32)
             if mode == "adaptive":
                 sess.adaptive_decode(n, threshold, exit_layers, self.max_early, st, out=o)
+            elif mode == "sampling":
+                # every random number is an input of the call: rows for all positions, drawn on the host (seeded)
+                sess.sampling_decode(n, temperature, threshold, exit_layers, self.max_early, self.uniforms(), 0, st, out=o)
             else:
                 sess.plain_decode(n, st, out=o)
             toks.append(o.copy())
@@ -216,6 +219,12 @@ class Bench:
         self.barrier()
         wall_ms = (time.perf_counter() - t0) * 1e3
         return ev0.elapsed_time(ev1), wall_ms, st, np.concatenate(toks, axis=1)
+
+    def uniforms(self):
+        if getattr(self, "_uniforms", None) is None:
+            rng = np.random.default_rng(4321)
+            self._uniforms = rng.random((self.batch, self.sess.max_seq_len, self.binding.SAMPLE_NU), dtype=np.float32)
+        return self._uniforms
 
     def e2e(self, mode, sizes=None):
         """The same steps end to end through the C ABI with host buffers: every step's timed region holds the
@@ -422,6 +431,15 @@ def extras(args, B, p_tok, torch, binding, synth) -> dict:
         B.register_heads(cfg.logit_scale, dense_T=True)
         out["dense_head_transformation"] = run()
         B.register_heads(cfg.logit_scale)
+    if B.sess.get_path() == 1:
+        # sampled decoding (Eq. 1 with a drawn token, Eq. 2 with acceptance test and resampling) at temperature 1:
+        # plain sampling (no exit layers) and the adaptive form; the time over plain greedy decoding is what the draws cost
+        sm = {}
+        for name, ex in (("plain_sampling", ()), ("adaptive_sampling", cfg.exit_layers)):
+            ms, _, st, tok = B.timed("sampling", sz, cfg.threshold, ex, temperature=1.0)
+            sm[name] = {"tokens_per_s": n * cfg.batch / (ms * 1e-3), "early_exit_rate": st.early_exits / max(1, st.steps),
+                        "rejection_rate": st.rejected / max(1, st.accepted + st.rejected), "time_vs_plain_greedy": ms / p_ms}
+        out["sampled_decoding_temperature_1"] = sm
     if args.workload == "8b" and not args.no_regime:
         out["confident_head_regime"] = confident_regime(args, cfg, torch, binding, synth)
     if args.workload == "8b-long" and not args.no_regime:
