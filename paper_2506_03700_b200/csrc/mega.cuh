@@ -210,7 +210,7 @@ struct DrawSrc {
 // exceeds u x (sum of all weights); the last token of non-zero weight if rounding leaves none.  Returns the token to every
 // thread (-1 if all weights are zero), with the sum of all weights and the drawn token's weight.  Partial sums per 128
 // entries in a fixed order, so the result does not depend on timing.
-__device__ __forceinline__ int block_draw(Smem *sm, const DrawSrc &src, int V, float u, float &total, float &w_tok) {
+__device__ __noinline__ int block_draw(Smem *sm, const DrawSrc &src, int V, float u, float &total, float &w_tok) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     float *psum = reinterpret_cast<float *>(sm->scratch + DRAW_OFFSET);   // [CONS_THREADS]
     float *wbuf = psum + CONS_THREADS;                                     // [DRAW_CHUNK]
