@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 # from the ncu captures summarised in profiles/ (1B-shaped launches; traffic grows in proportion to the
 # bytes streamed, so a ratio carries over to the larger shapes), keyed by decoding mode.  None = not
 # captured for the kernel as it stands.
-DRAM_TRAFFIC_RATIO = {"plain": None, "adaptive": None}
+DRAM_TRAFFIC_RATIO = {"plain": 0.9962, "adaptive": 0.9977}   # profiles/k_decode_persistent_1b_dram_traffic_ncu.md
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -291,13 +291,16 @@ def run_ours(args):
     if args.plain_only or args.adaptive_only:
         # profiling aid: one mode only, so that every launch of the persistent kernel moves a known number of bytes
         mode = "plain" if args.plain_only else "adaptive"
-        B.timed(mode, warm)
+        _, _, wst, _ = B.timed(mode, warm)
         ms, wall, st, tok = B.timed(mode)
         if rank == 0:
+            # the warm-up's own counters too: a capture of every launch of the process is compared with the sum of both
             print(json.dumps({"mode": mode + "_only", "tokens_per_s": gen_len * cfg.batch / (ms * 1e-3), "decode_ms": st.decode_ms,
                               "launches": int(st.kernel_launches), "layer_passes": int(st.layer_passes),
                               "head_evals": int(st.head_evals), "verify_steps": int(st.verify_steps),
-                              "algorithmic_bytes": byte_model(cfg, st, B.ctx_sum)}))
+                              "algorithmic_bytes": byte_model(cfg, st, B.ctx_sum),
+                              "warmup_launches": int(wst.kernel_launches),
+                              "warmup_algorithmic_bytes": byte_model(cfg, wst, sum(len(q) for q in B.prompts) / B.groups + sum(warm) / 2)}))
         if dist is not None:
             dist.destroy_process_group()
         return
