@@ -787,10 +787,50 @@ __device__ __forceinline__ void attn_item(const MegaArgs &A, const StepDesc &d, 
     j = item - kvh * nchunk;
 }
 
-// K/V producer: for every work item of this CTA, the K and V page blocks of its sub-blocks.  The K and V
-// rows of the tokens of this pass were written into the cache by the QKV epilogues of other CTAs; a
-// work item whose positions include such a row is fetched only once the grid has passed the barrier
-// that ends the QKV phase (`bar_target`).  Every other item reads rows of earlier passes only and is
+// Query tiles (16 (column, q head) pairs each) that hold a pair of the columns mk: bit t = tile t.
+__device__ __forceinline__ unsigned seq_tiles(const MegaArgs &A, unsigned mk) {
+    unsigned t = 0;
+#pragma unroll
+    for (int cc = 0; cc < MAX_COLS; ++cc)
+        if ((mk >> cc) & 1u) t |= (1u << ((cc * A.c.group) >> 4)) | (1u << ((cc * A.c.group + A.c.group - 1) >> 4));
+    return t & 3u;
+}
+// The consumers are two groups of four warps.  Where an item's queries span both tiles, group t works on tile t
+// of the same item.  Where every sequence's queries fit one tile (plain decoding; few columns; one q head per kv
+// head) the second group would idle: the groups then take DIFFERENT items, two per round, which halves the rounds
+// of a CTA that owns several items.  Which warps compute an item never changes what is computed.
+__device__ __forceinline__ bool attn_dual(const MegaArgs &A, unsigned mask) {
+    bool dual = true;
+    for (int k = 0; k < A.nseq; ++k) {
+        const unsigned t = seq_tiles(A, mask & seq_cols(A, k));
+        dual = dual && t != 3u;
+    }
+    return dual;
+}
+// One item of a round as every role sees it.
+struct AttnItem {
+    int k, kvh, j, nchunk, nsb, p_base, qt;   // sequence of the launch, kv head, chunk, the sequence's chunks, 64-position sub-blocks, first position, query tile
+    unsigned mk;                              // the sequence's active columns
+    bool have;
+};
+__device__ __forceinline__ AttnItem attn_item_of(const MegaArgs &A, const StepDesc &d, unsigned mask, int item, int n_items, bool dual, int grp) {
+    AttnItem it;
+    it.have = item < n_items;
+    it.k = it.kvh = it.j = it.nsb = it.p_base = it.qt = 0; it.nchunk = 1; it.mk = 0;
+    if (!it.have) return it;
+    attn_item(A, d, mask, item, it.k, it.kvh, it.j, it.nchunk);
+    it.mk = mask & seq_cols(A, it.k);
+    it.p_base = it.j * ATT_CHUNK;
+    it.nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[it.k] - it.p_base) / ATT_PAGE + 1);
+    it.qt = dual ? ((seq_tiles(A, it.mk) & 1u) ? 0 : 1) : grp;
+    return it;
+}
+
+// K/V producer: for every work item of this CTA, the K and V page blocks of its sub-blocks, in the order the
+// consumers walk them: per round (one item, or two in the dual arrangement) sub-block by sub-block, K of every
+// item of the round, then V.  The K and V rows of the tokens of this pass were written into the cache by the QKV
+// epilogues of other CTAs; an item whose positions include such a row is fetched only once the grid has passed
+// the barrier that ends the QKV phase (`bar_target`).  Every other item reads rows of earlier passes only and is
 // fetched as soon as ring slots are free, i.e. while the QKV product is still streaming.
 __device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, unsigned mask, unsigned bar_target,
                                              Rings &r, uint64_t pol) {
@@ -798,40 +838,44 @@ __device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S,
     Smem *sm = S.sm;
     const int lane = threadIdx.x & 31, cta = blockIdx.x, G = gridDim.x;
     const int n_items = attn_items(A, d, mask);
+    const bool dual = attn_dual(A, mask);
+    const int per_round = dual ? 2 : 1;
     const uint32_t bytes = (uint32_t)(ATT_PAGE * c.hd * 2);
     const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
     bool synced = false;
     if (lane == 0) trace(S, EV_ATT, 8);
-    for (int item = cta; item < n_items; item += G) {
-        int k, kvh, j, nchunk;
-        attn_item(A, d, mask, item, k, kvh, j, nchunk);
-        const unsigned mk = mask & seq_cols(A, k);
-        const int32_t *pages = c.page_table + (size_t)(A.seq0 + k) * c.max_pages;
-        const int p_base = j * ATT_CHUNK;
-        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[k] - p_base) / ATT_PAGE + 1);
+    for (int it0 = cta; it0 < n_items; it0 += G * per_round) {
+        AttnItem it[2];
+        it[0] = attn_item_of(A, d, mask, it0, n_items, dual, 0);
+        it[1] = attn_item_of(A, d, mask, dual ? it0 + G : n_items, n_items, dual, 1);
         bool has_new = false;
 #pragma unroll
-        for (int cc = 0; cc < MAX_COLS; ++cc)
-            has_new = has_new || (((mk >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK);
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+            for (int cc = 0; cc < MAX_COLS; ++cc)
+                has_new = has_new || (it[g].have && ((it[g].mk >> cc) & 1u) && d.pos[cc] >= it[g].p_base && d.pos[cc] < it[g].p_base + ATT_CHUNK);
         if (has_new && !synced) {
             grid_wait(S, A.grid_ctr, bar_target);
             fence_proxy_async();
             synced = true;
         }
-        for (int sb = 0; sb < nsb; ++sb) {
-            const int page = pages[(p_base + sb * ATT_PAGE) >> c.page_shift];
-            for (int which = 0; which < 2; ++which) {
-                const int slot = r.xi % NX;
-                mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
-                if (lane == 0 && !aborted(S)) {
-                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + which) * c.nkv + kvh) * ((size_t)ATT_PAGE * c.hd);
-                    mbar_expect_tx(&sm->x_full[slot], bytes);
-                    bulk_g2s(sm->x[slot], pool + blk, bytes, &sm->x_full[slot], pol);
-                    trace(S, EV_ATT, 9 + 16 * (2 * sb + which));
+        const int nsb = max(it[0].nsb, it[1].nsb);
+        for (int sb = 0; sb < nsb; ++sb)
+            for (int which = 0; which < 2; ++which)
+                for (int g = 0; g < per_round; ++g) {
+                    if (!it[g].have || sb >= it[g].nsb) continue;
+                    const int32_t *pages = c.page_table + (size_t)(A.seq0 + it[g].k) * c.max_pages;
+                    const int page = pages[(it[g].p_base + sb * ATT_PAGE) >> c.page_shift];
+                    const int slot = r.xi % NX;
+                    mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
+                    if (lane == 0 && !aborted(S)) {
+                        const size_t blk = ((((size_t)page * c.L + layer) * 2 + which) * c.nkv + it[g].kvh) * ((size_t)ATT_PAGE * c.hd);
+                        mbar_expect_tx(&sm->x_full[slot], bytes);
+                        bulk_g2s(sm->x[slot], pool + blk, bytes, &sm->x_full[slot], pol);
+                        trace(S, EV_ATT, 9 + 16 * (2 * sb + which));
+                    }
+                    ++r.xi;
                 }
-                ++r.xi;
-            }
-        }
     }
 }
 
@@ -893,7 +937,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     AttnSmem<HD> *as = reinterpret_cast<AttnSmem<HD> *>(sm->scratch);
     constexpr int KSQ = HD / 16, NT = HD / 8;
     constexpr int ATT_STRIDE = HD + 4;                     // floats per chunk partial: output, max, sum, padding (16-byte rows)
-    constexpr int QV = 2 * KSQ * 64 / CONS_THREADS;        // 16-byte pieces of a kv head's query fragments per thread
+    constexpr int QV = KSQ * 64 / (CONS_THREADS / 2);      // 16-byte pieces of one query tile's fragments per thread of a warp group
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x, G = gridDim.x;
     const int group = c.group;
     const int n_items = attn_items(A, d, mask);
@@ -947,138 +991,162 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     // With at most one work item per CTA the CTA that completes a head last merges it at once; with more,
     // designated CTAs do (see below).  Who merges does not change what is computed.
     const bool last_arriver_merges = n_items <= G;
-    for (int item = cta; item < n_items; item += G) {
-        int ks_, kvh, j, nchunk;
-        attn_item(A, d, mask, item, ks_, kvh, j, nchunk);
-        const unsigned mk = mask & seq_cols(A, ks_);   // the item's sequence: its columns only
-        const int p_base = j * ATT_CHUNK;
-        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[ks_] - p_base) / ATT_PAGE + 1);
-        // ---- the kv head's query fragments: one round trip to L2, then shared memory
+    // Rounds: one item whose two query tiles go to the two warp groups, or (every sequence's queries in one tile) two
+    // items, one per group.  Every warp walks the ring stages of the whole round in order and releases each of them;
+    // it multiplies only those of its own group's item.
+    const bool dual = attn_dual(A, mask);
+    const int per_round = dual ? 2 : 1;
+    for (int it0 = cta; it0 < n_items; it0 += G * per_round) {
+        AttnItem itg[2];
+        itg[0] = attn_item_of(A, d, mask, it0, n_items, dual, 0);
+        itg[1] = attn_item_of(A, d, mask, dual ? it0 + G : it0, n_items, dual, 1);
+        const AttnItem me = itg[mt];
+        const int kvh = me.kvh, j = me.j, p_base = me.p_base, qt = me.qt;
+        const unsigned mk = me.mk;   // the item's sequence: its columns only
+        // ---- query tile qt of the item's kv head, by this warp group: one round trip to L2, then shared memory
         {
-            const uint4 *src = reinterpret_cast<const uint4 *>(A.qfrag) + (size_t)kvh * (2 * KSQ * 64);
+            const uint4 *src = reinterpret_cast<const uint4 *>(A.qfrag) + (size_t)kvh * (2 * KSQ * 64) + (size_t)qt * (KSQ * 64);
+            const int gt = tid & (CONS_THREADS / 2 - 1);
             uint4 v[QV];
 #pragma unroll
-            for (int u = 0; u < QV; ++u) v[u] = __ldcg(src + tid + u * CONS_THREADS);
-            bar_consumers();   // the previous item is done with the shared buffers
+            for (int u = 0; u < QV; ++u) v[u] = me.have ? __ldcg(src + gt + u * (CONS_THREADS / 2)) : make_uint4(0u, 0u, 0u, 0u);
+            bar_consumers();   // the previous round is done with the shared buffers
 #pragma unroll
-            for (int u = 0; u < QV; ++u) reinterpret_cast<uint4 *>(&as->qfrag[0][0][0][0])[tid + u * CONS_THREADS] = v[u];
+            for (int u = 0; u < QV; ++u) reinterpret_cast<uint4 *>(&as->qfrag[mt][0][0][0])[gt + u * (CONS_THREADS / 2)] = v[u];
         }
         bar_consumers();
         if (tid == 0) trace(S, EV_ATT, 2);   // queries ready
-        // ---- per-warp online softmax state: rows (lane/4) and (lane/4)+8 of query tile mt
+        // ---- per-warp online softmax state: rows (lane/4) and (lane/4)+8 of query tile qt
         int lim[2];
 #pragma unroll
         for (int rh = 0; rh < 2; ++rh) {
-            const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = div_group(qcol, group);
-            lim[rh] = (cc < MAX_COLS && ((mk >> cc) & 1u)) ? d.pos[cc] : -1;
+            const int qcol = qt * 16 + (lane >> 2) + rh * 8, cc = div_group(qcol, group);
+            lim[rh] = (me.have && cc < MAX_COLS && ((mk >> cc) & 1u)) ? d.pos[cc] : -1;
         }
         // a query tile none of whose 16 (column, q head) pairs is in use does no arithmetic (uniform per warp)
         bool tile_used = false;
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
-            const int cc = div_group(mt * 16 + q, group);
+            const int cc = div_group(qt * 16 + q, group);
             tile_used = tile_used || (cc < MAX_COLS && ((mk >> cc) & 1u));
         }
+        tile_used = tile_used && me.have;
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
         float o[NT][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) o[nt][i] = 0.f;
+        const int nsb = max(itg[0].nsb, dual ? itg[1].nsb : 0);
         for (int sb = 0; sb < nsb; ++sb) {
             const int p0 = p_base + sb * ATT_PAGE;
+            const bool act = me.have && sb < me.nsb;   // this warp's item has this sub-block
             float s[2][4];
-            {   // ---- K block
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s[nt][i] = -INFINITY;
+#pragma unroll 1
+            for (int g = 0; g < per_round; ++g) {   // ---- K block(s)
+                if (!itg[g].have || sb >= itg[g].nsb) continue;
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
                 if (tid == 0) trace(S, EV_ATT, 3 + 16 * sb);   // K block landed
-                const unsigned char *kb = sm->x[slot];
-                float sh[2][4], sl[2][4];
+                if (!dual || g == mt) {
+                    const unsigned char *kb = sm->x[slot];
+                    float sh[2][4], sl[2][4];
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+                    for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) { sh[nt][i] = 0.f; sl[nt][i] = 0.f; }
-                const int id = lane >> 3;
-                const int pl = 16 * qr + (lane & 7) + 8 * (id >> 1);
-                const unsigned char *krow = kb + pl * (HD * 2);
-                if (tile_used)
+                        for (int i = 0; i < 4; ++i) { sh[nt][i] = 0.f; sl[nt][i] = 0.f; }
+                    const int id = lane >> 3;
+                    const int pl = 16 * qr + (lane & 7) + 8 * (id >> 1);
+                    const unsigned char *krow = kb + pl * (HD * 2);
+                    if (tile_used)
 #pragma unroll
-                for (int k0 = 0; k0 < KSQ; k0 += 4) {   // four k-steps of loads in flight, then their multiply-adds
-                    uint4 qh[4], ql[4];
-                    uint32_t kf[4][4];
+                    for (int k0 = 0; k0 < KSQ; k0 += 4) {   // four k-steps of loads in flight, then their multiply-adds
+                        uint4 qh[4], ql[4];
+                        uint32_t kf[4][4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int ks = k0 + u;
-                        qh[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][0]);
-                        ql[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][4]);
-                        ldmatrix_x4(kf[u], krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
+                        for (int u = 0; u < 4; ++u) {
+                            const int ks = k0 + u;
+                            qh[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][0]);
+                            ql[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][4]);
+                            ldmatrix_x4(kf[u], krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const uint32_t ah[4] = {qh[u].x, qh[u].y, qh[u].z, qh[u].w}, al[4] = {ql[u].x, ql[u].y, ql[u].z, ql[u].w};
+                            mma16816(sh[0], ah, kf[u][0], kf[u][1]);
+                            mma16816(sh[1], ah, kf[u][2], kf[u][3]);
+                            mma16816(sl[0], al, kf[u][0], kf[u][1]);
+                            mma16816(sl[1], al, kf[u][2], kf[u][3]);
+                        }
                     }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint32_t ah[4] = {qh[u].x, qh[u].y, qh[u].z, qh[u].w}, al[4] = {ql[u].x, ql[u].y, ql[u].z, ql[u].w};
-                        mma16816(sh[0], ah, kf[u][0], kf[u][1]);
-                        mma16816(sh[1], ah, kf[u][2], kf[u][3]);
-                        mma16816(sl[0], al, kf[u][0], kf[u][1]);
-                        mma16816(sl[1], al, kf[u][2], kf[u][3]);
-                    }
+                    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int pos = p0 + 16 * qr + 8 * nt + 2 * (lane & 3) + (i & 1);
+                            s[nt][i] = pos <= lim[i >> 1] ? sh[nt][i] + sl[nt][i] : -INFINITY;
+                        }
                 }
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int pos = p0 + 16 * qr + 8 * nt + 2 * (lane & 3) + (i & 1);
-                        s[nt][i] = pos <= lim[i >> 1] ? sh[nt][i] + sl[nt][i] : -INFINITY;
-                    }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->x_empty[slot]);
                 ++r.xi;
             }
             // ---- online softmax over this warp's 16 positions
-            uint32_t ph[4], plo[4];
+            uint32_t ph[4] = {0u, 0u, 0u, 0u}, plo[4] = {0u, 0u, 0u, 0u};
+            if (act) {
 #pragma unroll
-            for (int rh = 0; rh < 2; ++rh) {
-                float mx = fmaxf(fmaxf(s[0][2 * rh], s[0][2 * rh + 1]), fmaxf(s[1][2 * rh], s[1][2 * rh + 1]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float mn = fmaxf(m_run[rh], mx);
-                float corr = 1.f, p[4] = {0.f, 0.f, 0.f, 0.f};
-                if (mn != -INFINITY) {
-                    corr = __expf(m_run[rh] - mn);
-                    p[0] = __expf(s[0][2 * rh] - mn); p[1] = __expf(s[0][2 * rh + 1] - mn);
-                    p[2] = __expf(s[1][2 * rh] - mn); p[3] = __expf(s[1][2 * rh + 1] - mn);
+                for (int rh = 0; rh < 2; ++rh) {
+                    float mx = fmaxf(fmaxf(s[0][2 * rh], s[0][2 * rh + 1]), fmaxf(s[1][2 * rh], s[1][2 * rh + 1]));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float mn = fmaxf(m_run[rh], mx);
+                    float corr = 1.f, p[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (mn != -INFINITY) {
+                        corr = __expf(m_run[rh] - mn);
+                        p[0] = __expf(s[0][2 * rh] - mn); p[1] = __expf(s[0][2 * rh + 1] - mn);
+                        p[2] = __expf(s[1][2 * rh] - mn); p[3] = __expf(s[1][2 * rh + 1] - mn);
+                    }
+                    m_run[rh] = mn;
+                    l_run[rh] = l_run[rh] * corr + ((p[0] + p[1]) + (p[2] + p[3]));
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) { o[nt][2 * rh] *= corr; o[nt][2 * rh + 1] *= corr; }
+                    // A fragment of P: a0/a1 = n-tile 0 (rows r / r+8), a2/a3 = n-tile 1
+                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
+                    ph[rh] = *reinterpret_cast<const uint32_t *>(&h0);
+                    ph[2 + rh] = *reinterpret_cast<const uint32_t *>(&h1);
+                    plo[rh] = pack_bf16(p[0] - __low2float(h0), p[1] - __high2float(h0));
+                    plo[2 + rh] = pack_bf16(p[2] - __low2float(h1), p[3] - __high2float(h1));
                 }
-                m_run[rh] = mn;
-                l_run[rh] = l_run[rh] * corr + ((p[0] + p[1]) + (p[2] + p[3]));
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) { o[nt][2 * rh] *= corr; o[nt][2 * rh + 1] *= corr; }
-                // A fragment of P: a0/a1 = n-tile 0 (rows r / r+8), a2/a3 = n-tile 1
-                const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
-                ph[rh] = *reinterpret_cast<const uint32_t *>(&h0);
-                ph[2 + rh] = *reinterpret_cast<const uint32_t *>(&h1);
-                plo[rh] = pack_bf16(p[0] - __low2float(h0), p[1] - __high2float(h0));
-                plo[2 + rh] = pack_bf16(p[2] - __low2float(h1), p[3] - __high2float(h1));
             }
-            {   // ---- V block
+#pragma unroll 1
+            for (int g = 0; g < per_round; ++g) {   // ---- V block(s)
+                if (!itg[g].have || sb >= itg[g].nsb) continue;
                 const int slot = r.xi % NX;
                 mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
                 if (tid == 0) trace(S, EV_ATT, 4 + 16 * sb);   // V block landed
-                const unsigned char *vb = sm->x[slot];
-                const int id = lane >> 3;
-                const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
-                const unsigned char *vrow = vb + pl * (HD * 2);
-                if (tile_used)
+                if (!dual || g == mt) {
+                    const unsigned char *vb = sm->x[slot];
+                    const int id = lane >> 3;
+                    const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
+                    const unsigned char *vrow = vb + pl * (HD * 2);
+                    if (tile_used)
 #pragma unroll
-                for (int n0 = 0; n0 < NT / 2; n0 += 4) {
-                    uint32_t vf[4][4];
+                    for (int n0 = 0; n0 < NT / 2; n0 += 4) {
+                        uint32_t vf[4][4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) ldmatrix_x4_trans(vf[u], vrow + ((((2 * (n0 + u)) | (id >> 1)) ^ (pl & 7)) << 4));
+                        for (int u = 0; u < 4; ++u) ldmatrix_x4_trans(vf[u], vrow + ((((2 * (n0 + u)) | (id >> 1)) ^ (pl & 7)) << 4));
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int np = n0 + u;
-                        mma16816(o[2 * np], ph, vf[u][0], vf[u][1]);
-                        mma16816(o[2 * np + 1], ph, vf[u][2], vf[u][3]);
-                        mma16816(o[2 * np], plo, vf[u][0], vf[u][1]);
-                        mma16816(o[2 * np + 1], plo, vf[u][2], vf[u][3]);
+                        for (int u = 0; u < 4; ++u) {
+                            const int np = n0 + u;
+                            mma16816(o[2 * np], ph, vf[u][0], vf[u][1]);
+                            mma16816(o[2 * np + 1], ph, vf[u][2], vf[u][3]);
+                            mma16816(o[2 * np], plo, vf[u][0], vf[u][1]);
+                            mma16816(o[2 * np + 1], plo, vf[u][2], vf[u][3]);
+                        }
                     }
                 }
                 __syncwarp();
@@ -1086,7 +1154,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 ++r.xi;
             }
         }
-        // ---- row sums over the quad, then merge the four position quarters of each query tile:
+        // ---- row sums over the quad, then merge the four position quarters of each warp group:
         //      (q0 + q1) and (q2 + q3), then the two halves
 #pragma unroll
         for (int rh = 0; rh < 2; ++rh) {
@@ -1106,8 +1174,8 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
             // ---- chunk partial (unnormalised output, max, sum) of every valid (column, q head)
 #pragma unroll
             for (int rh = 0; rh < 2; ++rh) {
-                const int qcol = mt * 16 + (lane >> 2) + 8 * rh, cc = div_group(qcol, group), g = qcol - cc * group;
-                if (cc < MAX_COLS && ((mk >> cc) & 1u) && d.pos[cc] >= p_base) {
+                const int qcol = qt * 16 + (lane >> 2) + 8 * rh, cc = div_group(qcol, group), g = qcol - cc * group;
+                if (me.have && cc < MAX_COLS && ((mk >> cc) & 1u) && d.pos[cc] >= p_base) {
                     float *out = A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + j) * ATT_STRIDE;
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
@@ -1116,23 +1184,27 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
                 }
             }
         }
-        // ---- this item's partials are complete: count it (a release that returns nothing, so nobody waits for it)
-        if (tid == 0) trace(S, EV_ITEM, item);
+        // ---- the round's partials are complete: count its items (a release that returns nothing, so nobody waits for it)
+        if (tid == 0) trace(S, EV_ITEM, it0);
         bar_consumers();
-        if (last_arriver_merges) {
+        if (last_arriver_merges) {   // at most one item per CTA: the round holds item it0 alone
+            const int cnt = itg[0].k * c.nkv + itg[0].kvh;
             if (tid == 0) {   // release this block's partials and acquire the others' in one step
                 unsigned old;
-                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + ks_ * c.nkv + kvh) : "memory");
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + cnt) : "memory");
                 sm->bcast[2] = (int)old;
             }
             bar_consumers();
-            if (sm->bcast[2] == nchunk - 1) {
-                merge_chunks(kvh, mk);
-                if (tid == 0) { A.attn_cnt[ks_ * c.nkv + kvh] = 0u; trace(S, EV_COMBINE, kvh); }
+            if (sm->bcast[2] == itg[0].nchunk - 1) {
+                merge_chunks(itg[0].kvh, itg[0].mk);
+                if (tid == 0) { A.attn_cnt[cnt] = 0u; trace(S, EV_COMBINE, itg[0].kvh); }
             }
-        } else if (tid == 0) {
-            __threadfence();
-            red_release_add(A.attn_cnt + ks_ * c.nkv + kvh, 1u);
+        } else if (tid == 0 || (dual && tid == CONS_THREADS / 2)) {
+            const AttnItem &mine = itg[tid == 0 ? 0 : 1];
+            if (mine.have) {
+                __threadfence();
+                red_release_add(A.attn_cnt + mine.k * c.nkv + mine.kvh, 1u);
+            }
         }
     }
     if (last_arriver_merges) return;
@@ -1141,8 +1213,7 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
     // whichever CTA arrives last do it looks cheaper but piles up at long contexts: the CTA that
     // merges one head is late for its next item, so it is last again for the next head, and ends up
     // merging every head in turn while the rest of the grid waits.)
-    for (int hk = 0; hk < A.nseq * c.nkv; ++hk) {   // (sequence of the launch, kv head)
-        if ((G - 1 - hk % G + G) % G != cta) continue;
+    for (int hk = G - 1 - cta; hk < A.nseq * c.nkv; hk += G) {   // (sequence of the launch, kv head) pairs of this CTA
         const int ks_ = hk / c.nkv, kvh = hk - ks_ * c.nkv, nchunk = seq_chunks(A, d, mask, ks_);
         if (nchunk == 0) continue;
         if (tid == 0) grid_wait(S, A.attn_cnt + hk, (unsigned)nchunk);
