@@ -879,6 +879,50 @@ __device__ __forceinline__ void attn_produce(const MegaArgs &A, const Shared &S,
     }
 }
 
+// The producer of a phase in which no CTA owns more than one item (see attn_consume_single).
+__device__ __forceinline__ void attn_produce_single(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, unsigned mask, unsigned bar_target,
+                                             Rings &r, uint64_t pol) {
+    const Ctx &c = A.c;
+    Smem *sm = S.sm;
+    const int lane = threadIdx.x & 31, cta = blockIdx.x, G = gridDim.x;
+    const int n_items = attn_items(A, d, mask);
+    const uint32_t bytes = (uint32_t)(ATT_PAGE * c.hd * 2);
+    const __nv_bfloat16 *pool = reinterpret_cast<const __nv_bfloat16 *>(c.kv_pool);
+    bool synced = false;
+    if (lane == 0) trace(S, EV_ATT, 8);
+    for (int item = cta; item < n_items; item += G) {
+        int k, kvh, j, nchunk;
+        attn_item(A, d, mask, item, k, kvh, j, nchunk);
+        const unsigned mk = mask & seq_cols(A, k);
+        const int32_t *pages = c.page_table + (size_t)(A.seq0 + k) * c.max_pages;
+        const int p_base = j * ATT_CHUNK;
+        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[k] - p_base) / ATT_PAGE + 1);
+        bool has_new = false;
+#pragma unroll
+        for (int cc = 0; cc < MAX_COLS; ++cc)
+            has_new = has_new || (((mk >> cc) & 1u) && d.pos[cc] >= p_base && d.pos[cc] < p_base + ATT_CHUNK);
+        if (has_new && !synced) {
+            grid_wait(S, A.grid_ctr, bar_target);
+            fence_proxy_async();
+            synced = true;
+        }
+        for (int sb = 0; sb < nsb; ++sb) {
+            const int page = pages[(p_base + sb * ATT_PAGE) >> c.page_shift];
+            for (int which = 0; which < 2; ++which) {
+                const int slot = r.xi % NX;
+                mbar_wait(S, &sm->x_empty[slot], ((r.xi / NX) & 1) ^ 1);
+                if (lane == 0 && !aborted(S)) {
+                    const size_t blk = ((((size_t)page * c.L + layer) * 2 + which) * c.nkv + kvh) * ((size_t)ATT_PAGE * c.hd);
+                    mbar_expect_tx(&sm->x_full[slot], bytes);
+                    bulk_g2s(sm->x[slot], pool + blk, bytes, &sm->x_full[slot], pol);
+                    trace(S, EV_ATT, 9 + 16 * (2 * sb + which));
+                }
+                ++r.xi;
+            }
+        }
+    }
+}
+
 // Merge (max, sum, unnormalised output) of another warp, read from shared memory, into this warp's.
 template <int NT, int HD>
 __device__ __forceinline__ void attn_merge_from(float (&o)[NT][4], float (&m_run)[2], float (&l_run)[2], const float (*so)[HD],
@@ -928,6 +972,261 @@ __device__ __forceinline__ void attn_merge_to(const float (&o)[NT][4], const flo
 // general integer division (some thirty of those sat on the critical path of every attention item)
 __device__ __forceinline__ int div_group(int x, int group) {
     return group == 4 ? x >> 2 : group == 2 ? x >> 1 : group == 1 ? x : (x * 43) >> 7;
+}
+
+// The same for a phase in which no CTA owns more than one item (contexts up to about 128 positions x CTAs / kv heads:
+// the common case of short and medium contexts): one item, its two query tiles on the two warp groups, merged by
+// whichever CTA completes a head last.  Kept as a path of its own: the general form below, with its rounds of two
+// items, costs this case 2-4 % of the step.
+template <int HD>
+__device__ __forceinline__ void attn_consume_single(const MegaArgs &A, const Shared &S, const StepDesc &d, int layer, unsigned mask, Rings &r) {
+    const Ctx &c = A.c;
+    Smem *sm = S.sm;
+    AttnSmem<HD> *as = reinterpret_cast<AttnSmem<HD> *>(sm->scratch);
+    constexpr int KSQ = HD / 16, NT = HD / 8;
+    constexpr int ATT_STRIDE = HD + 4;                     // floats per chunk partial: output, max, sum, padding (16-byte rows)
+    constexpr int QV = 2 * KSQ * 64 / CONS_THREADS;        // 16-byte pieces of a kv head's query fragments per thread
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x, G = gridDim.x;
+    const int group = c.group;
+    const int n_items = attn_items(A, d, mask);
+    const int mt = warp >> 2, qr = warp & 3;
+    (void)layer;
+    // Merge of the chunk partials of one kv head into the O-projection's input (by a whole CTA).
+    auto merge_chunks = [&](int kvh, unsigned mk) {   // mk: the active columns of the work item's sequence
+        // Four features of one (column, q head) per thread and pass; the chunk partials are folded in
+        // ascending order, eight at a time with all their loads in flight, by the usual running-max rule.
+        const int nqc = MAX_COLS * group;
+        for (int idx = tid; idx < nqc * (HD / 4); idx += CONS_THREADS) {
+            const int qcol = idx / (HD / 4), dim = (idx - qcol * (HD / 4)) * 4, cc = div_group(qcol, group), g = qcol - cc * group;
+            if (!((mk >> cc) & 1u)) continue;
+            const int h = kvh * group + g;
+            const int nch = d.pos[cc] / ATT_CHUNK + 1;
+            const float *part = A.attn_part + (((size_t)cc * c.nq + h) * c.n_chunks) * ATT_STRIDE;
+            float Mx = -INFINITY, den = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k0 = 0; k0 < nch; k0 += 8) {
+                float2 ml[8];
+                float4 ov[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const bool ok = k0 + u < nch;
+                    const float *pk = part + (size_t)(k0 + u) * ATT_STRIDE;
+                    ml[u] = ok ? __ldcg(reinterpret_cast<const float2 *>(pk + HD)) : make_float2(-INFINITY, 0.f);
+                    ov[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(pk + dim)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float Mn = Mx;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, ml[u].x);
+                if (Mn == -INFINITY) continue;
+                const float sc = Mx == -INFINITY ? 0.f : __expf(Mx - Mn);
+                den *= sc; acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (ml[u].x != -INFINITY) {
+                        const float w = __expf(ml[u].x - Mn);
+                        den += ml[u].y * w;
+                        acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
+                    }
+                }
+                Mx = Mn;
+            }
+            xfrag_store(A.XO, h * HD + dim, cc, acc.x / den);
+            xfrag_store(A.XO, h * HD + dim + 1, cc, acc.y / den);
+            xfrag_store(A.XO, h * HD + dim + 2, cc, acc.z / den);
+            xfrag_store(A.XO, h * HD + dim + 3, cc, acc.w / den);
+        }
+    };
+    // With at most one work item per CTA the CTA that completes a head last merges it at once; with more,
+    // designated CTAs do (see below).  Who merges does not change what is computed.
+    const bool last_arriver_merges = true;   // at most one item per CTA (the caller's condition)
+    for (int item = cta; item < n_items; item += G) {
+        int ks_, kvh, j, nchunk;
+        attn_item(A, d, mask, item, ks_, kvh, j, nchunk);
+        const unsigned mk = mask & seq_cols(A, ks_);   // the item's sequence: its columns only
+        const int p_base = j * ATT_CHUNK;
+        const int nsb = min(ATT_CHUNK / ATT_PAGE, (d.seq_pmax[ks_] - p_base) / ATT_PAGE + 1);
+        // ---- the kv head's query fragments: one round trip to L2, then shared memory
+        {
+            const uint4 *src = reinterpret_cast<const uint4 *>(A.qfrag) + (size_t)kvh * (2 * KSQ * 64);
+            uint4 v[QV];
+#pragma unroll
+            for (int u = 0; u < QV; ++u) v[u] = __ldcg(src + tid + u * CONS_THREADS);
+            bar_consumers();   // the previous item is done with the shared buffers
+#pragma unroll
+            for (int u = 0; u < QV; ++u) reinterpret_cast<uint4 *>(&as->qfrag[0][0][0][0])[tid + u * CONS_THREADS] = v[u];
+        }
+        bar_consumers();
+        if (tid == 0) trace(S, EV_ATT, 2);   // queries ready
+        // ---- per-warp online softmax state: rows (lane/4) and (lane/4)+8 of query tile mt
+        int lim[2];
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+            const int qcol = mt * 16 + (lane >> 2) + rh * 8, cc = div_group(qcol, group);
+            lim[rh] = (cc < MAX_COLS && ((mk >> cc) & 1u)) ? d.pos[cc] : -1;
+        }
+        // a query tile none of whose 16 (column, q head) pairs is in use does no arithmetic (uniform per warp)
+        bool tile_used = false;
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int cc = div_group(mt * 16 + q, group);
+            tile_used = tile_used || (cc < MAX_COLS && ((mk >> cc) & 1u));
+        }
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float o[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[nt][i] = 0.f;
+        for (int sb = 0; sb < nsb; ++sb) {
+            const int p0 = p_base + sb * ATT_PAGE;
+            float s[2][4];
+            {   // ---- K block
+                const int slot = r.xi % NX;
+                mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                if (tid == 0) trace(S, EV_ATT, 3 + 16 * sb);   // K block landed
+                const unsigned char *kb = sm->x[slot];
+                float sh[2][4], sl[2][4];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { sh[nt][i] = 0.f; sl[nt][i] = 0.f; }
+                const int id = lane >> 3;
+                const int pl = 16 * qr + (lane & 7) + 8 * (id >> 1);
+                const unsigned char *krow = kb + pl * (HD * 2);
+                if (tile_used)
+#pragma unroll
+                for (int k0 = 0; k0 < KSQ; k0 += 4) {   // four k-steps of loads in flight, then their multiply-adds
+                    uint4 qh[4], ql[4];
+                    uint32_t kf[4][4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int ks = k0 + u;
+                        qh[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][0]);
+                        ql[u] = *reinterpret_cast<const uint4 *>(&as->qfrag[mt][ks][lane][4]);
+                        ldmatrix_x4(kf[u], krow + ((((2 * ks) | (id & 1)) ^ (pl & 7)) << 4));
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t ah[4] = {qh[u].x, qh[u].y, qh[u].z, qh[u].w}, al[4] = {ql[u].x, ql[u].y, ql[u].z, ql[u].w};
+                        mma16816(sh[0], ah, kf[u][0], kf[u][1]);
+                        mma16816(sh[1], ah, kf[u][2], kf[u][3]);
+                        mma16816(sl[0], al, kf[u][0], kf[u][1]);
+                        mma16816(sl[1], al, kf[u][2], kf[u][3]);
+                    }
+                }
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int pos = p0 + 16 * qr + 8 * nt + 2 * (lane & 3) + (i & 1);
+                        s[nt][i] = pos <= lim[i >> 1] ? sh[nt][i] + sl[nt][i] : -INFINITY;
+                    }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->x_empty[slot]);
+                ++r.xi;
+            }
+            // ---- online softmax over this warp's 16 positions
+            uint32_t ph[4], plo[4];
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                float mx = fmaxf(fmaxf(s[0][2 * rh], s[0][2 * rh + 1]), fmaxf(s[1][2 * rh], s[1][2 * rh + 1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float mn = fmaxf(m_run[rh], mx);
+                float corr = 1.f, p[4] = {0.f, 0.f, 0.f, 0.f};
+                if (mn != -INFINITY) {
+                    corr = __expf(m_run[rh] - mn);
+                    p[0] = __expf(s[0][2 * rh] - mn); p[1] = __expf(s[0][2 * rh + 1] - mn);
+                    p[2] = __expf(s[1][2 * rh] - mn); p[3] = __expf(s[1][2 * rh + 1] - mn);
+                }
+                m_run[rh] = mn;
+                l_run[rh] = l_run[rh] * corr + ((p[0] + p[1]) + (p[2] + p[3]));
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) { o[nt][2 * rh] *= corr; o[nt][2 * rh + 1] *= corr; }
+                // A fragment of P: a0/a1 = n-tile 0 (rows r / r+8), a2/a3 = n-tile 1
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
+                ph[rh] = *reinterpret_cast<const uint32_t *>(&h0);
+                ph[2 + rh] = *reinterpret_cast<const uint32_t *>(&h1);
+                plo[rh] = pack_bf16(p[0] - __low2float(h0), p[1] - __high2float(h0));
+                plo[2 + rh] = pack_bf16(p[2] - __low2float(h1), p[3] - __high2float(h1));
+            }
+            {   // ---- V block
+                const int slot = r.xi % NX;
+                mbar_wait(S, &sm->x_full[slot], (r.xi / NX) & 1);
+                if (tid == 0) trace(S, EV_ATT, 4 + 16 * sb);   // V block landed
+                const unsigned char *vb = sm->x[slot];
+                const int id = lane >> 3;
+                const int pl = 16 * qr + (lane & 7) + 8 * (id & 1);
+                const unsigned char *vrow = vb + pl * (HD * 2);
+                if (tile_used)
+#pragma unroll
+                for (int n0 = 0; n0 < NT / 2; n0 += 4) {
+                    uint32_t vf[4][4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) ldmatrix_x4_trans(vf[u], vrow + ((((2 * (n0 + u)) | (id >> 1)) ^ (pl & 7)) << 4));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int np = n0 + u;
+                        mma16816(o[2 * np], ph, vf[u][0], vf[u][1]);
+                        mma16816(o[2 * np + 1], ph, vf[u][2], vf[u][3]);
+                        mma16816(o[2 * np], plo, vf[u][0], vf[u][1]);
+                        mma16816(o[2 * np + 1], plo, vf[u][2], vf[u][3]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->x_empty[slot]);
+                ++r.xi;
+            }
+        }
+        // ---- row sums over the quad, then merge the four position quarters of each query tile:
+        //      (q0 + q1) and (q2 + q3), then the two halves
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+            l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 1);
+            l_run[rh] += __shfl_xor_sync(0xffffffffu, l_run[rh], 2);
+        }
+        if (tid == 0) trace(S, EV_ATT, 5);   // sub-blocks done
+        bar_consumers();   // every warp is done with the query fragments, whose space the merge reuses
+        if (qr & 1) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        bar_consumers();
+        if (!(qr & 1)) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        bar_consumers();
+        if (qr == 2) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+        bar_consumers();
+        if (qr == 0) {
+            attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+            // ---- chunk partial (unnormalised output, max, sum) of every valid (column, q head)
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const int qcol = mt * 16 + (lane >> 2) + 8 * rh, cc = div_group(qcol, group), g = qcol - cc * group;
+                if (cc < MAX_COLS && ((mk >> cc) & 1u) && d.pos[cc] >= p_base) {
+                    float *out = A.attn_part + (((size_t)cc * c.nq + kvh * group + g) * c.n_chunks + j) * ATT_STRIDE;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        *reinterpret_cast<float2 *>(out + nt * 8 + 2 * (lane & 3)) = make_float2(o[nt][2 * rh], o[nt][2 * rh + 1]);
+                    if ((lane & 3) == 0) *reinterpret_cast<float2 *>(out + HD) = make_float2(m_run[rh], l_run[rh]);
+                }
+            }
+        }
+        // ---- this item's partials are complete: count it (a release that returns nothing, so nobody waits for it)
+        if (tid == 0) trace(S, EV_ITEM, item);
+        bar_consumers();
+        if (last_arriver_merges) {
+            if (tid == 0) {   // release this block's partials and acquire the others' in one step
+                unsigned old;
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(A.attn_cnt + ks_ * c.nkv + kvh) : "memory");
+                sm->bcast[2] = (int)old;
+            }
+            bar_consumers();
+            if (sm->bcast[2] == nchunk - 1) {
+                merge_chunks(kvh, mk);
+                if (tid == 0) { A.attn_cnt[ks_ * c.nkv + kvh] = 0u; trace(S, EV_COMBINE, kvh); }
+            }
+        } else if (tid == 0) {
+            __threadfence();
+            red_release_add(A.attn_cnt + ks_ * c.nkv + kvh, 1u);
+        }
+    }
 }
 
 template <int HD>
@@ -1465,8 +1764,14 @@ __device__ __forceinline__ void run(const MegaArgs &A, Shared &S) {
                 phase_barrier(2);
             }
             // ---- attention (work items that hold no row of this pass are fetched before the QKV phase has ended)
-            if (ROLE == 1) attn_produce(A, S, d, l, mask, bar_no * (unsigned)G, r, pol);
-            if (ROLE == 2) attn_consume<HD>(A, S, d, l, mask, r);
+            if (ROLE == 1) {
+                if (attn_items(A, d, mask) <= G) attn_produce_single(A, S, d, l, mask, bar_no * (unsigned)G, r, pol);
+                else attn_produce(A, S, d, l, mask, bar_no * (unsigned)G, r, pol);
+            }
+            if (ROLE == 2) {
+                if (attn_items(A, d, mask) <= G) attn_consume_single<HD>(A, S, d, l, mask, r);
+                else attn_consume<HD>(A, S, d, l, mask, r);
+            }
             phase_barrier(4);
             // ---- O projection + residual; prepares the FFN input
             {

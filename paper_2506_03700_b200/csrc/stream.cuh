@@ -684,15 +684,13 @@ __device__ __forceinline__ void gemm_consume(const Shared &S, const Gemm &g, int
         if (KS > 1) bar_consumers();
     };
     {
-        // one call site for both kinds of plan: the group's code (main loop, reduction, epilogue) exists once per
-        // product, which keeps the kernel's instruction footprint down
         const Plan pl = make_plan(g, cta, G);
-        const int n_groups = pl.split ? (pl.n > 0 ? 1 : 0) : (pl.t1 - pl.t0 + CONS_WARPS - 1) / CONS_WARPS;
-        const int ksp = (pl.split && pl.s0_own_k0 > 0) ? group_ks(make_plan(g, cta - 1, G).n) : 0;
-        for (int gi = 0; gi < n_groups; ++gi) {
-            const int g0 = pl.split ? pl.ta : pl.t0 + gi * CONS_WARPS;
-            group(g0, pl.split ? pl.n : min(CONS_WARPS, pl.t1 - g0), pl.split ? pl.s0_own_k0 : 0, pl.split ? pl.s0_pub_k1 : 0,
-                  pl.split ? pl.sl_k1 : nch, ksp, gi + 1 == n_groups);
+        if (pl.split) {
+            const int ksp = pl.s0_own_k0 > 0 ? group_ks(make_plan(g, cta - 1, G).n) : 0;
+            if (pl.n > 0) group(pl.ta, pl.n, pl.s0_own_k0, pl.s0_pub_k1, pl.sl_k1, ksp, true);
+        } else {
+            for (int g0 = pl.t0; g0 < pl.t1; g0 += CONS_WARPS)
+                group(g0, min(CONS_WARPS, pl.t1 - g0), 0, 0, nch, 0, g0 + CONS_WARPS >= pl.t1);
         }
     }
 }
