@@ -163,3 +163,28 @@ def test_law_of_a_verified_token_on_the_gpu(gamma):
     assert st.early_exits > 0 and st.rejected > 0 and st.accepted > 0
     # the wrong rule a plausible mistake would implement (accept every early token) is told apart at this sample size
     assert not chi2_ok(counts, qs[0], alpha=1e-6)[0]
+
+
+def test_same_numbers_same_decisions_for_every_sequence_of_a_batch():
+    """Three sequences in one launch (one weight stream), each with its own prompt and its own random numbers: each
+    equals the oracle's run of that sequence alone.  (The chi-square test cannot see a mix-up of the sequences' random
+    numbers: any uniform number gives the right law.)"""
+    cfg = hd128(logit_scale=2.0, resid_scale=0.1)
+    pair = Pair(cfg)
+    batch, n, max_seq, max_early = 3, 12, 64, 1
+    prompts = [synth.make_prompt(cfg, n=m, seq=i).numpy() for i, m in enumerate((9, 21, 14))]
+    us, wants, sts = [], [], []
+    for i, p in enumerate(prompts):
+        u, want, ost, _ = _numbers_with_margin(pair, p, n, 0.25, 0.2, cfg.exit_layers, max_early, max_seq, seed0=1000 * i)
+        us.append(u); wants.append(want); sts.append(ost)
+    S = binding.Session(pair.gm, batch, max_seq, 64, max_early)
+    assert S.get_path() == 1
+    for i, p in enumerate(prompts):
+        S.prefill(p, seq=i)
+    st = binding.Stats()
+    got = S.sampling_decode(n, 0.25, 0.2, cfg.exit_layers, max_early, np.stack(us), 0, st)
+    for i in range(batch):
+        assert np.array_equal(got[i], wants[i]), (i, got[i], wants[i])
+    for f in ("head_evals", "early_exits", "accepted", "rejected", "discarded"):
+        assert getattr(st, f) == sum(getattr(o, f) for o in sts), f
+    assert st.early_exits > 0 and st.accepted > 0
