@@ -199,11 +199,12 @@ constexpr int DRAW_MAX_VOCAB = DRAW_MAX_CHUNKS * DRAW_CHUNK;
 struct DrawSrc {
     const float *z; float m, inv_s;
     const float *zq; float mq, inv_sq;
-    __device__ __forceinline__ float weight(int v) const {
-        const float a = __expf(__ldcg(z + v) - m);
+    __device__ __forceinline__ float weight_of(float zv, float qv) const {   // from the loaded logits (-inf: outside the vocabulary)
+        const float a = __expf(zv - m);
         if (!zq) return a;
-        return fmaxf(0.f, a * inv_s - __expf(__ldcg(zq + v) - mq) * inv_sq);
+        return fmaxf(0.f, a * inv_s - __expf(qv - mq) * inv_sq);
     }
+    __device__ __forceinline__ float weight(int v) const { return weight_of(__ldcg(z + v), zq ? __ldcg(zq + v) : 0.f); }
 };
 
 // Inverse-CDF draw by the consumer warps of one CTA: the first token, in vocabulary order, whose running sum of weights
@@ -218,19 +219,42 @@ __device__ __noinline__ int block_draw(Smem *sm, const DrawSrc &src, int V, floa
     float *csum = res + 8;                                                 // [chunks]
     const int n_chunks = (V + DRAW_CHUNK - 1) / DRAW_CHUNK;
     // pass 1: the sum of every chunk (warp w takes chunks w, w + 8, ...; eight chunks' loads in flight)
-    for (int c0 = warp; c0 < n_chunks; c0 += CONS_WARPS * 8) {
+    const bool vec = (V & 3) == 0;   // rows start on 16-byte boundaries: one 16-byte load per lane and chunk
+    for (int c0 = warp; vec && c0 < n_chunks; c0 += CONS_WARPS * 8) {
+        float4 zv[8], qv[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int v = (c0 + j * CONS_WARPS) * DRAW_CHUNK + 4 * lane;
+            const bool in = v < V;   // V is a multiple of 4: the four entries are inside together
+            zv[j] = in ? __ldcg(reinterpret_cast<const float4 *>(src.z + v)) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            qv[j] = (src.zq && in) ? __ldcg(reinterpret_cast<const float4 *>(src.zq + v)) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float a = (src.weight_of(zv[j].x, qv[j].x) + src.weight_of(zv[j].y, qv[j].y)) + (src.weight_of(zv[j].z, qv[j].z) + src.weight_of(zv[j].w, qv[j].w));
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+            const int ch = c0 + j * CONS_WARPS;
+            if (lane == 0 && ch < n_chunks) csum[ch] = a;
+        }
+    }
+    for (int c0 = warp; !vec && c0 < n_chunks; c0 += CONS_WARPS * 8) {
+        // all 32 (or 64) loads of the lane first, then the arithmetic: one round trip to L2 per eight chunks, not one per entry
+        float zv[8][DRAW_CHUNK / 32], qv[8][DRAW_CHUNK / 32];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int it = 0; it < DRAW_CHUNK / 32; ++it) {
+                const int v = (c0 + j * CONS_WARPS) * DRAW_CHUNK + it * 32 + lane;
+                zv[j][it] = v < V ? __ldcg(src.z + v) : -INFINITY;
+                qv[j][it] = (src.zq && v < V) ? __ldcg(src.zq + v) : -INFINITY;
+            }
         float acc[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const int ch = c0 + j * CONS_WARPS;
             float a = 0.f;
-            if (ch < n_chunks) {
 #pragma unroll
-                for (int it = 0; it < DRAW_CHUNK / 32; ++it) {
-                    const int v = ch * DRAW_CHUNK + it * 32 + lane;
-                    a += v < V ? src.weight(v) : 0.f;
-                }
-            }
+            for (int it = 0; it < DRAW_CHUNK / 32; ++it) a += src.weight_of(zv[j][it], qv[j][it]);
             acc[j] = a;
         }
 #pragma unroll
@@ -310,9 +334,163 @@ __device__ __noinline__ int block_draw(Smem *sm, const DrawSrc &src, int V, floa
     return tok;
 }
 
+// The same draw from a head's distribution exp(z - m), using what the head product already left behind: CTA b of the
+// grid has published (max, sum of exp, argmax) of its own rows of the vocabulary, [16 t0(b), 16 t1(b)), a contiguous range in
+// CTA order.  The running sum over the CTAs finds the CTA whose range holds the crossing; only that range's logits
+// (vocabulary / grid entries) are read again.  Two round trips to L2 instead of a pass over the whole vocabulary by one CTA.
+__device__ __noinline__ int block_draw_head(Smem *sm, const float *z, float m, const float *head_part, int col, int G, int V, float u,
+                                            float &total, float &w_tok) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    float *psum = reinterpret_cast<float *>(sm->scratch + DRAW_OFFSET);   // second-level sums, then the located range
+    float *wbuf = psum + CONS_THREADS;
+    float *res = wbuf + DRAW_CHUNK;
+    float *csum = res + 8;
+    const int T = (V + 15) / 16;
+    // (1) running sum over the CTAs' sums, by warp 0: lane l holds CTAs [l per, (l + 1) per)
+    if (warp == 0) {
+        const int per = (G + 31) / 32;
+        float loc = 0.f;
+        for (int k = 0; k < per; ++k) {
+            const int b = lane * per + k;
+            if (b < G) {
+                const float4 v = __ldcg(reinterpret_cast<const float4 *>(head_part + ((size_t)b * MAX_COLS + col) * 4));
+                loc += (v.x == -INFINITY) ? 0.f : v.y * __expf(v.x - m);
+            }
+        }
+        float inc = loc;   // inclusive scan over the lanes
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float o = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += o;
+        }
+        const float tot = __shfl_sync(0xffffffffu, inc, 31);
+        const float target = u * tot;
+        const unsigned hit = __ballot_sync(0xffffffffu, inc > target);
+        int l_at = hit ? __ffs(hit) - 1 : -1;
+        bool take_last = false;
+        if (l_at < 0) {   // rounding left no crossing: the last lane of non-zero sum
+            const unsigned pos = __ballot_sync(0xffffffffu, loc > 0.f);
+            l_at = pos ? 31 - __clz(pos) : -1;
+            take_last = true;
+        }
+        if (lane == (l_at < 0 ? 0 : l_at)) {
+            int b_at = -1;
+            float base = inc - loc;
+            if (l_at >= 0) {
+                float run = base;
+                int last_b = -1;
+                for (int k = 0; k < per; ++k) {   // the lane walks its CTAs again (the same values, from L2)
+                    const int b = lane * per + k;
+                    if (b >= G) break;
+                    const float4 v = __ldcg(reinterpret_cast<const float4 *>(head_part + ((size_t)b * MAX_COLS + col) * 4));
+                    const float wv = (v.x == -INFINITY) ? 0.f : v.y * __expf(v.x - m);
+                    if (wv > 0.f) last_b = b;
+                    if (!take_last && run + wv > target) { b_at = b; base = run; break; }
+                    run += wv;
+                }
+                if (b_at < 0) { b_at = last_b; take_last = true; base = 0.f; }
+            }
+            res[0] = __int_as_float(b_at);
+            res[1] = base;
+            res[2] = tot;
+            res[3] = take_last ? 1.f : 0.f;
+        }
+    }
+    bar_consumers();
+    const int b_at = __float_as_int(res[0]);
+    const float base = res[1];
+    total = res[2];
+    const bool take_last = res[3] != 0.f;
+    w_tok = 0.f;
+    if (b_at < 0 || !(total > 0.f)) { bar_consumers(); return -1; }
+    const float target = u * total;
+    int t0, t1;
+    cta_tile_range(T, b_at, G, t0, t1);
+    const int v0 = t0 * 16, v1 = min(V, t1 * 16), n_sub = (v1 - v0 + DRAW_CHUNK - 1) / DRAW_CHUNK;
+    // (2) sums of the 128-entry pieces of that range (one per warp and turn)
+    for (int sub = warp; sub < n_sub; sub += CONS_WARPS) {
+        float a = 0.f;
+#pragma unroll
+        for (int it = 0; it < DRAW_CHUNK / 32; ++it) {
+            const int v = v0 + sub * DRAW_CHUNK + it * 32 + lane;
+            a += v < v1 ? __expf(__ldcg(z + v) - m) : 0.f;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+        if (lane == 0) csum[sub] = a;
+    }
+    bar_consumers();
+    // (3) the piece that holds the crossing, then the entry inside it (warp 0; entries in vocabulary order)
+    if (warp == 0) {
+        float run = base;
+        int sub_at = -1;
+        bool tl = take_last;
+        for (int sub = 0; sub < n_sub; ++sub) {
+            if (!tl && run + csum[sub] > target) { sub_at = sub; break; }
+            run += csum[sub];
+        }
+        if (sub_at < 0) {
+            tl = true;
+            for (int sub = n_sub - 1; sub >= 0; --sub)
+                if (csum[sub] > 0.f) { sub_at = sub; break; }
+        }
+        int tok = -1;
+        float wt = 0.f;
+        if (sub_at >= 0) {
+            // lane l holds the entries [4 l, 4 l + 4) of the piece
+            float wv[4], loc = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int v = v0 + sub_at * DRAW_CHUNK + 4 * lane + i;
+                wv[i] = v < v1 ? __expf(__ldcg(z + v) - m) : 0.f;
+                loc += wv[i];
+            }
+            float inc = loc;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float o = __shfl_up_sync(0xffffffffu, inc, off);
+                if (lane >= off) inc += o;
+            }
+            const float before = run + inc - loc;
+            int my = -1;
+            float r2 = before;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                r2 += wv[i];
+                if (my < 0 && !tl && r2 > target) my = i;
+            }
+            const unsigned hit = __ballot_sync(0xffffffffu, my >= 0);
+            int l_at, i_at;
+            if (hit) {
+                l_at = __ffs(hit) - 1;
+                i_at = __shfl_sync(0xffffffffu, my, l_at);
+            } else {   // the last entry of non-zero weight
+                int lastp = -1;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) if (wv[i] > 0.f) lastp = i;
+                const unsigned pos = __ballot_sync(0xffffffffu, lastp >= 0);
+                l_at = pos ? 31 - __clz(pos) : 0;
+                i_at = max(__shfl_sync(0xffffffffu, lastp, l_at), 0);
+            }
+            float wsel = wv[0];
+#pragma unroll
+            for (int i = 1; i < 4; ++i) if (i == i_at) wsel = wv[i];
+            wt = __shfl_sync(0xffffffffu, wsel, l_at);
+            tok = v0 + sub_at * DRAW_CHUNK + 4 * l_at + i_at;
+        }
+        if (lane == 0) { res[4] = __int_as_float(tok); res[5] = wt; }
+    }
+    bar_consumers();
+    const int tok = __float_as_int(res[4]);
+    w_tok = res[5];
+    bar_consumers();   // the buffers may be rewritten by the next draw
+    return tok;
+}
+
 struct SampleArgs {
     const float *uniforms; float *q_stage; float4 *qinfo; const float *logit_stage; HeadResult *head_res; DevState *st;
     int vocab, max_seq, cps, L, seq0, nseq, exit_idx;
+    const float *head_part; int G;   // the grid's per-CTA (max, sum of exp, argmax) of the head just evaluated
 };
 
 // Sampled decoding at a control point (its own function: its registers must not weigh on the streaming loops).
@@ -330,9 +508,8 @@ __device__ __noinline__ void sample_stage(SampleArgs a, Smem *sm, bool after_hea
         for (int col = 0; col < MAX_COLS; ++col) {
             if (!((head_cols >> col) & 1u)) continue;
             const int s = a.seq0 + (a.nseq == 1 ? 0 : col / cps), pos = dprev->pos[col], slot = s * MAX_COLS + (pos & 7);
-            DrawSrc src{a.q_stage + (size_t)slot * V, hr_s[col].zmax, 0.f, nullptr, 0.f, 0.f};
             float total, wt;
-            const int tok = block_draw(sm, src, V, unif(s, pos + 1, 3 + a.exit_idx), total, wt);
+            const int tok = block_draw_head(sm, a.q_stage + (size_t)slot * V, hr_s[col].zmax, a.head_part, col, a.G, V, unif(s, pos + 1, 3 + a.exit_idx), total, wt);
             if (tid == 0) {
                 hr_s[col].token = max(tok, 0);
                 hr_s[col].p = tok < 0 ? 0.f : wt / total;
@@ -366,9 +543,8 @@ __device__ __noinline__ void sample_stage(SampleArgs a, Smem *sm, bool after_hea
             }
             if (!rejected) {
                 const int col = c0 + nrow - 1;
-                DrawSrc src{a.logit_stage + (size_t)col * V, hr_s[col].zmax, 0.f, nullptr, 0.f, 0.f};
                 float total, wt;
-                const int tok = block_draw(sm, src, V, unif(s, ln, 0), total, wt);
+                const int tok = block_draw_head(sm, a.logit_stage + (size_t)col * V, hr_s[col].zmax, a.head_part, col, a.G, V, unif(s, ln, 0), total, wt);
                 if (tid == 0) hr_s[col].token = max(tok, 0);
             }
         }
@@ -422,7 +598,7 @@ __device__ __forceinline__ void control_cta0(const MegaArgs &A, Smem *sm, int ki
     // (a') sampled decoding replaces the tokens and probabilities the bookkeeping below works with
     if (A.sampling && kind != CTRL_START && !(kind == CTRL_TOP && st->pf_end > 0)) {
         SampleArgs sa{A.uniforms, A.q_stage, A.qinfo, c.logit_stage, c.head_res, st, c.vocab, c.max_seq, cps, L, seq0, nseq,
-                      kind == CTRL_HEAD ? A.exit_at[e] - 1 : 0};
+                      kind == CTRL_HEAD ? A.exit_at[e] - 1 : 0, A.head_part, G};
         sample_stage(sa, sm, kind == CTRL_HEAD, &dprev, head_cols);
     }
     // (b) bookkeeping, one thread.  Every scalar it may need is read up front (the loads overlap);
