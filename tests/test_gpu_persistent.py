@@ -477,3 +477,31 @@ def test_sequences_sharing_one_weight_stream(max_early, batch):
         if i != 1:
             assert np.array_equal(e[i], singles[i]), i
     assert np.array_equal(e[1][:k + 1], singles[1][:k + 1]) and (e[1][k + 1:] == eos).all()
+
+
+def test_both_attention_arrangements_agree_with_more_items_than_ctas():
+    """Four q heads per kv head at a context of 9700 positions: 2 x 76 work items, more than the GPU has SMs.  Plain
+    decoding (one column: every query in the first tile, the two warp groups take different items) and adaptive decoding
+    with forced exits (up to six columns: both query tiles in use, the groups share an item) must give the same tokens
+    and the same final-logit bits: which warps compute an item does not change its arithmetic."""
+    cfg = gqa(n_layers=2, exit_layers=(1,))
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n_prompt = 128 * (sms // 2 + 2) - 28
+    assert 2 * (n_prompt // 128 + 1) > sms
+    pair = Pair(cfg)
+    prompt = synth.make_prompt(cfg, n=n_prompt).numpy()
+    n = 14
+    P = session(pair, max_seq=n_prompt + 64)
+    P.capture_logits(n + 4)
+    P.prefill(prompt)
+    out = P.plain_decode(n)[0]
+    lg = P.captured_logits()[:n].clone()
+    for tape in ([1] * 32, [1, 1, 0, 1, 1, 1, 1, 0] * 4):
+        A = session(pair, max_seq=n_prompt + 64)
+        A.capture_logits(n + 8)
+        A.prefill(prompt)
+        A.set_exit_tape(tape)
+        st = binding.Stats()
+        assert np.array_equal(A.adaptive_decode(n, 0.5, cfg.exit_layers, 5, st)[0], out)
+        assert torch.equal(A.captured_logits()[:n], lg)
+        assert st.early_exits >= 5
