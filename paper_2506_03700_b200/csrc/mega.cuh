@@ -1363,14 +1363,15 @@ __device__ __forceinline__ void attn_consume_single(const MegaArgs &A, const Sha
         }
         if (tid == 0) trace(S, EV_ATT, 5);   // sub-blocks done
         bar_consumers();   // every warp is done with the query fragments, whose space the merge reuses
-        if (qr & 1) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        // (a query tile without a query in use skips the merge: its warps only keep the barriers)
+        if ((qr & 1) && tile_used) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
         bar_consumers();
-        if (!(qr & 1)) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        if (!(qr & 1) && tile_used) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
         bar_consumers();
-        if (qr == 2) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+        if (qr == 2 && tile_used) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
         bar_consumers();
         if (qr == 0) {
-            attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+            if (tile_used) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
             // ---- chunk partial (unnormalised output, max, sum) of every valid (column, q head)
 #pragma unroll
             for (int rh = 0; rh < 2; ++rh) {
@@ -1638,14 +1639,15 @@ __device__ __forceinline__ void attn_consume(const MegaArgs &A, const Shared &S,
         }
         if (tid == 0) trace(S, EV_ATT, 5);   // sub-blocks done
         bar_consumers();   // every warp is done with the query fragments, whose space the merge reuses
-        if (qr & 1) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        // (a query tile without a query in use skips the merge: its warps only keep the barriers)
+        if ((qr & 1) && tile_used) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
         bar_consumers();
-        if (!(qr & 1)) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
+        if (!(qr & 1) && tile_used) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][qr >> 1], as->ml[mt][qr >> 1], lane);
         bar_consumers();
-        if (qr == 2) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+        if (qr == 2 && tile_used) attn_merge_to<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
         bar_consumers();
         if (qr == 0) {
-            attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
+            if (tile_used) attn_merge_from<NT, HD>(o, m_run, l_run, as->o[mt][0], as->ml[mt][0], lane);
             // ---- chunk partial (unnormalised output, max, sum) of every valid (column, q head)
 #pragma unroll
             for (int rh = 0; rh < 2; ++rh) {
