@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 # from the ncu captures summarised in profiles/ (1B-shaped launches; traffic grows in proportion to the
 # bytes streamed, so a ratio carries over to the larger shapes), keyed by decoding mode.  None = not
 # captured for the kernel as it stands.
-DRAM_TRAFFIC_RATIO = {"plain": 0.9962, "adaptive": 0.9976}   # profiles/k_decode_persistent_1b_dram_traffic_ncu.md
+DRAM_TRAFFIC_RATIO = {"plain": 0.9961, "adaptive": 0.9976}   # profiles/k_decode_persistent_1b_dram_traffic_ncu.md
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
