@@ -464,6 +464,21 @@ def second_model_run(args, cfg, torch, binding, synth, resid_scale, n_tok) -> di
     d.update({"o_down_scale": resid_scale, "tokens": n, "plain_tokens_per_s": n * cfg.batch / (p_ms * 1e-3),
               "speedup_vs_plain": p_ms / a_ms, "byte_model_speedup": byte_model_speedup(cfg, a_st, p_st, B2.ctx_sum),
               "distinct_tokens": len(set(p_tok[0].tolist())), "exits_at_layer": a_st.as_dict()["exits_at_layer"]})
+    if B2.sess.get_path() == 1:
+        # the same with sampled tokens: plain sampling against the adaptive form with Eq. 2 in full, at a low and at a
+        # moderate temperature (a shorter run each)
+        n_s = min(n, 512)
+        sz_s = step_sizes(n_s, max(1, min(args.steps, n_s)))
+        sm = {}
+        for T in (0.2, 0.7):
+            r = {}
+            for name, ex in (("plain_sampling", ()), ("adaptive_sampling", cfg.exit_layers)):
+                ms, _, st, _ = B2.timed("sampling", sz_s, cfg.threshold, ex, temperature=T)
+                r[name] = {"tokens_per_s": n_s * cfg.batch / (ms * 1e-3), "early_exit_rate": st.early_exits / max(1, st.steps),
+                           "rejection_rate": st.rejected / max(1, st.accepted + st.rejected)}
+            r["speedup_vs_plain_sampling"] = r["adaptive_sampling"]["tokens_per_s"] / r["plain_sampling"]["tokens_per_s"]
+            sm[str(T)] = r
+        d["sampled_decoding_by_temperature"] = sm
     del B2
     torch.cuda.empty_cache()
     return d
